@@ -1,0 +1,20 @@
+"""B200-native N-way Adasum combine (arXiv 2006.02924): hand-written sm_100a kernels behind a
+C-ABI library, with a thin Python binding.
+
+``workloads`` (synthetic inputs) imports without the native library; every compute entry point
+lives in ``binding`` and raises if the library has not been built.
+"""
+
+_BINDING_NAMES = (
+    "adasum_reduce", "adasum_pair", "adasum_workspace_bytes", "adasum_status_string",
+    "adasum_shutdown", "AdasumError",
+)
+
+
+def __getattr__(name):
+    if name in _BINDING_NAMES or name == "binding":
+        import importlib
+
+        binding = importlib.import_module(__name__ + ".binding")
+        return binding if name == "binding" else getattr(binding, name)
+    raise AttributeError(name)
