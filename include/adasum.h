@@ -1,0 +1,177 @@
+/*
+ * adasum.h — C ABI of the B200 (sm_100a) N-way Adasum combine.
+ *
+ * The operation (arXiv 2006.02924, Section 3 and Section 3.4; Algorithm 1 for the order):
+ *
+ *     Adasum(a, b) = (1 - a.b / (2 |a|^2)) a  +  (1 - a.b / (2 |b|^2)) b
+ *
+ * applied recursively over a binary tree whose first level pairs workers (2i, 2i+1), whose
+ * second level pairs the results of blocks of two, and so on, independently for every tensor
+ * (layer) of a fused gradient buffer (Section 3.6, Section 4.4.3).  |g|^2 is the squared L2
+ * norm.  An operand whose squared norm is exactly zero contributes nothing and leaves the
+ * other operand unchanged.  If the operand count at a level is odd, the last operand is
+ * carried to the next level unchanged (the paper itself only treats powers of two).
+ *
+ * All N worker buffers live in the memory of ONE GPU.  Dot products and norms are accumulated
+ * in fp32 inside blocks of at most a few thousand elements per thread block and in fp64 across
+ * blocks (Section 4.4.1 asks for accumulation wider than the gradient type); all coefficient
+ * arithmetic is fp64 on the device; intermediates between levels and the output are fp32.
+ *
+ * Conventions for every entry point:
+ *   - plain C, no exceptions; every call returns a status, and on any status other than
+ *     ADASUM_OK nothing has been launched unless stated otherwise;
+ *   - "device" pointers are CUDA device addresses on the current device, "host" pointers are
+ *     ordinary host memory that is only read during the call;
+ *   - the caller owns every buffer; inputs are never written; `out` and `workspace` must not
+ *     overlap any input or each other;
+ *   - calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL = legacy
+ *     default stream) and never synchronise it;
+ *   - the library allocates nothing per call.  The first call with a tensor-offset table it
+ *     has not seen on the current device builds a small segment table on the device
+ *     (cudaMalloc plus a blocking copy); later calls with the same table reuse it.  Up to 64
+ *     tables are kept; beyond that the oldest is freed.  adasum_shutdown() frees them all.
+ *     That first call must therefore not be made while the stream is being captured into a
+ *     CUDA graph;
+ *   - results are deterministic: the same inputs, sizes and flags give the same bits.
+ */
+#ifndef ADASUM_H_
+#define ADASUM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Element type of the worker gradients.  The output is fp32 for every input type. */
+typedef enum {
+    ADASUM_F32 = 0,
+    ADASUM_F16 = 1,   /* IEEE binary16 */
+    ADASUM_BF16 = 2
+} adasum_dtype_t;
+
+typedef enum {
+    ADASUM_OK = 0,
+    ADASUM_ERR_NULL = 1,        /* a required pointer is NULL */
+    ADASUM_ERR_ARG = 2,         /* N < 1, num_tensors < 0, bad flags, misaligned out, overlap */
+    ADASUM_ERR_OFFSETS = 3,     /* offsets[0] != 0 or decreasing offsets */
+    ADASUM_ERR_DTYPE = 4,       /* unknown dtype */
+    ADASUM_ERR_WORKSPACE = 5,   /* workspace NULL or smaller than adasum_workspace_bytes() */
+    ADASUM_ERR_CUDA = 6,        /* a CUDA runtime call or a launch failed (see adasum_last_error) */
+    ADASUM_ERR_TIMEOUT = 7      /* reserved for bounded device-side waits; unused by the
+                                   current kernels, which never wait on one another */
+} adasum_status_t;
+
+/*
+ * flags: how the tree is evaluated (the RESULT is the same binary tree in every case).
+ *
+ * A group of R = 2^j adjacent operands is a complete sub-tree of the binary tree, and every
+ * node of that sub-tree is a linear combination of its R leaves.  One "level" of this library
+ * therefore reads the operands once to form each group's R x R Gram matrix per tensor, derives
+ * on the device the R leaf weights that the sub-tree's recursion produces, and reads the
+ * operands a second time to write the group's weighted sum.  R = 2 is the literal
+ * level-by-level tree (three scalars a.b, a.a, b.b per pair, as in Algorithm 1).
+ *
+ *   bits 0..7    radix of the first level: 0 = choose automatically, else 2, 4, 8 or 16
+ *   bits 8..15   radix of the later levels: 0 = same rule as the first level
+ */
+#define ADASUM_RADIX_AUTO 0u
+#define ADASUM_FLAGS_RADIX(first, later) (((uint32_t)(first) & 0xffu) | (((uint32_t)(later) & 0xffu) << 8))
+
+#define ADASUM_MAX_WORKERS 4096
+#define ADASUM_MAX_LEVELS 12
+
+/*
+ * Bytes of device workspace that adasum_reduce / adasum_pair need for these sizes (an upper
+ * bound that depends only on the arguments given here, not on the offset values).
+ * Returns 0 on invalid arguments.  Host-only; touches no CUDA state.
+ */
+size_t adasum_workspace_bytes(int64_t total_elems, int32_t num_tensors, int32_t n_workers,
+                              adasum_dtype_t dtype, uint32_t flags);
+
+/*
+ * How a reduce with these sizes will run: writes the radix of each level into radices[]
+ * (room for ADASUM_MAX_LEVELS entries), the number of levels into *num_levels and the number
+ * of kernel launches into *num_launches (each may be NULL).  Host-only.
+ */
+adasum_status_t adasum_plan_info(int64_t total_elems, int32_t num_tensors, int32_t n_workers,
+                                 adasum_dtype_t dtype, uint32_t flags, int32_t* radices,
+                                 int32_t* num_levels, int32_t* num_launches);
+
+/*
+ * N-way Adasum combine (Section 3.4 tree of the Section 3 operator, per tensor).
+ *
+ *   grads           host array of n_workers device pointers; grads[w] is worker w's fused
+ *                   gradient buffer of tensor_offsets[num_tensors] elements of `dtype`,
+ *                   aligned to its element size (16-byte alignment of every buffer selects
+ *                   the vectorised kernels; anything else falls back to scalar loads)
+ *   tensor_offsets  host array of num_tensors + 1 element offsets into each buffer:
+ *                   tensor_offsets[0] = 0, non-decreasing; empty tensors are allowed
+ *   n_workers       1 .. ADASUM_MAX_WORKERS; n_workers = 1 converts grads[0] to fp32
+ *   out             device, tensor_offsets[num_tensors] floats, 4-byte aligned
+ *   workspace       device, at least adasum_workspace_bytes(...) bytes, 256-byte aligned;
+ *                   contents on entry are ignored and on exit unspecified
+ *   flags           see above; 0 is the recommended default
+ *   stream          cudaStream_t
+ *
+ * A zero-element reduce (tensor_offsets[num_tensors] == 0) returns ADASUM_OK without a launch.
+ */
+adasum_status_t adasum_reduce(const void* const* grads, const int64_t* tensor_offsets,
+                              int32_t num_tensors, int32_t n_workers, adasum_dtype_t dtype,
+                              float* out, void* workspace, size_t workspace_bytes,
+                              uint32_t flags, void* stream);
+
+/*
+ * One application of the operator per tensor, out = Adasum(a, b) (Section 3; the "partial dot
+ * products" and "apply Adasum" steps of Algorithm 1).  Same conventions as adasum_reduce with
+ * n_workers = 2; `a` and `b` are device pointers.
+ */
+adasum_status_t adasum_pair(const void* a, const void* b, const int64_t* tensor_offsets,
+                            int32_t num_tensors, adasum_dtype_t dtype, float* out,
+                            void* workspace, size_t workspace_bytes, uint32_t flags,
+                            void* stream);
+
+/* Static, human-readable name of a status code. */
+const char* adasum_status_string(adasum_status_t status);
+
+/* Detail of the most recent failure on the calling thread ("" if none); valid until the next
+ * call into the library from the same thread. */
+const char* adasum_last_error(void);
+
+/*
+ * Per-launch device timing, for benchmarks (the paper has no counterpart; it reports wall-clock
+ * times only).  Between adasum_profile_enable() and adasum_profile_collect(), every reduce/pair
+ * call records a CUDA event on its stream before its first kernel and after each kernel.
+ * adasum_profile_collect() stops recording, waits for the last event and writes one record per
+ * kernel launch in launch order (at most `capacity`; *count receives the number available).
+ * `kernel` is one of the ADASUM_KERNEL_* values, `level` the tree level (0 = first), `radix`
+ * the level's group size, `ms` the time from the previous event to the one after the launch.
+ * Use from one thread, with all profiled calls on one stream.
+ * Errors: ADASUM_ERR_ARG (max_launches < 1, or more launches happened than were reserved:
+ * the records that were taken are still returned), ADASUM_ERR_NULL, ADASUM_ERR_CUDA.
+ */
+#define ADASUM_KERNEL_GRAM_PARTIAL 0
+#define ADASUM_KERNEL_TREE_WEIGHTS 1
+#define ADASUM_KERNEL_WEIGHTED_SUM 2
+#define ADASUM_KERNEL_CONVERT 3
+
+typedef struct {
+    int32_t kernel;
+    int32_t level;
+    int32_t radix;
+    float ms;
+} adasum_launch_record_t;
+
+adasum_status_t adasum_profile_enable(int32_t max_launches);
+adasum_status_t adasum_profile_collect(adasum_launch_record_t* records, int32_t capacity, int32_t* count);
+
+/* Frees every cached segment table on every device and the profiling events.  Outstanding work that uses them must
+ * have completed.  Returns ADASUM_OK or ADASUM_ERR_CUDA. */
+adasum_status_t adasum_shutdown(void);
+
+#ifdef __cplusplus
+}
+#endif
+
+#endif /* ADASUM_H_ */

@@ -1,0 +1,681 @@
+// Host side of the C ABI declared in include/adasum.h: argument checks, the level plan, the cached
+// segment tables and the kernel launches.  Nothing here synchronises the stream.
+#include "adasum.h"
+
+#include <cuda_runtime.h>
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <memory>
+#include <mutex>
+#include <vector>
+
+#include "adasum_kernels.cuh"
+
+namespace adasum {
+namespace {
+
+thread_local char g_error[512] = "";
+
+adasum_status_t fail(adasum_status_t status, const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_error, sizeof g_error, fmt, ap);
+    va_end(ap);
+    return status;
+}
+
+#define ADASUM_CUDA_CHECK(expr)                                                                  \
+    do {                                                                                         \
+        cudaError_t err__ = (expr);                                                              \
+        if (err__ != cudaSuccess)                                                                \
+            return fail(ADASUM_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(err__));            \
+    } while (0)
+
+// ---- optional per-launch timing ---------------------------------------------------------------
+// When enabled, an event is recorded on the caller's stream before the first launch of a reduce
+// and after every launch; launch i lasted from event i to event i + 1.  Meant for benchmarking
+// from one thread.
+
+struct ProfileMark {
+    int32_t kernel, level, radix;
+    bool starts_call;     // the event opens a reduce call: no launch ends here
+};
+
+struct Profiler {
+    bool enabled = false;
+    std::vector<cudaEvent_t> events;
+    std::vector<ProfileMark> marks;
+    size_t used = 0;
+    bool overflow = false;
+};
+
+Profiler g_profiler;
+std::mutex g_profiler_mutex;
+
+void profile_mark(cudaStream_t stream, int kernel, int level, int radix, bool starts_call)
+{
+    if (!g_profiler.enabled)
+        return;
+    std::lock_guard<std::mutex> lock(g_profiler_mutex);
+    if (!g_profiler.enabled)
+        return;
+    if (g_profiler.used >= g_profiler.events.size()) {
+        g_profiler.overflow = true;
+        return;
+    }
+    if (cudaEventRecord(g_profiler.events[g_profiler.used], stream) != cudaSuccess)
+        return;
+    g_profiler.marks[g_profiler.used] = ProfileMark{kernel, level, radix, starts_call};
+    ++g_profiler.used;
+}
+
+constexpr size_t kAlign = 256;
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+int dtype_bytes(adasum_dtype_t dtype) { return dtype == ADASUM_F32 ? 4 : 2; }
+
+bool valid_radix(int r) { return r == 2 || r == 4 || r == 8 || r == 16; }
+
+int pow2_ceil(int x)
+{
+    int p = 1;
+    while (p < x)
+        p *= 2;
+    return p;
+}
+
+// Elements per segment for a level of radix R.  Per-block fp32 accumulation never spans more
+// than this many elements; longer tensors are finished in fp64.
+int segment_length(int radix) { return radix >= 16 ? 16384 : 8192; }
+
+struct Level {
+    int radix;
+    int operands;   // operands entering the level
+    int groups;     // operands leaving it
+    int seg_len;
+};
+
+struct LevelPlan {
+    int num_levels = 0;
+    Level level[ADASUM_MAX_LEVELS];
+};
+
+bool plan_levels(int n_workers, adasum_dtype_t dtype, uint32_t flags, LevelPlan* plan)
+{
+    (void)dtype;
+    const int first = (int)(flags & 0xffu), later_flag = (int)((flags >> 8) & 0xffu);
+    if ((flags >> 16) != 0)
+        return false;
+    if (first != 0 && !valid_radix(first))
+        return false;
+    if (later_flag != 0 && !valid_radix(later_flag))
+        return false;
+    const int later = later_flag != 0 ? later_flag : first;
+    int m = n_workers;
+    plan->num_levels = 0;
+    while (m > 1) {
+        if (plan->num_levels == ADASUM_MAX_LEVELS)
+            return false;
+        const int want = plan->num_levels == 0 ? first : later;
+        int radix = want != 0 ? want : kMaxRadix;
+        if (radix > pow2_ceil(m))
+            radix = pow2_ceil(m);
+        Level& lv = plan->level[plan->num_levels++];
+        lv.radix = radix;
+        lv.operands = m;
+        lv.groups = (m + radix - 1) / radix;
+        lv.seg_len = segment_length(radix);
+        m = lv.groups;
+    }
+    return true;
+}
+
+int64_t segment_bound(int64_t total, int32_t num_tensors, int seg_len)
+{
+    return total / seg_len + 2 * (int64_t)num_tensors + 1;
+}
+
+struct Layout {
+    size_t partials = 0, weights = 0, buffer[2] = {0, 0};
+    size_t partials_bytes = 0, weights_bytes = 0, buffer_bytes[2] = {0, 0};
+    int64_t padded_elems = 0;
+    size_t total = 0;
+};
+
+Layout make_layout(const LevelPlan& plan, int64_t total_elems, int32_t num_tensors)
+{
+    Layout lay;
+    lay.padded_elems = (total_elems + 63) / 64 * 64;
+    for (int l = 0; l < plan.num_levels; ++l) {
+        const Level& lv = plan.level[l];
+        const size_t p = (size_t)segment_bound(total_elems, num_tensors, lv.seg_len) * lv.groups *
+                         gram_entries(lv.radix) * sizeof(float);
+        const size_t w = (size_t)(num_tensors > 0 ? num_tensors : 1) * lv.groups * lv.radix * sizeof(float);
+        if (p > lay.partials_bytes)
+            lay.partials_bytes = p;
+        if (w > lay.weights_bytes)
+            lay.weights_bytes = w;
+        if (l + 1 < plan.num_levels) {      // this level's output is an intermediate
+            const size_t b = (size_t)lv.groups * lay.padded_elems * sizeof(float);
+            if (b > lay.buffer_bytes[l & 1])
+                lay.buffer_bytes[l & 1] = b;
+        }
+    }
+    size_t off = 0;
+    lay.partials = off;
+    off += align_up(lay.partials_bytes);
+    lay.weights = off;
+    off += align_up(lay.weights_bytes);
+    lay.buffer[0] = off;
+    off += align_up(lay.buffer_bytes[0]);
+    lay.buffer[1] = off;
+    off += align_up(lay.buffer_bytes[1]);
+    lay.total = off > 0 ? off : kAlign;
+    return lay;
+}
+
+// ---- cached segment tables ---------------------------------------------------------------------
+
+struct SegmentTable {
+    int device = -1;
+    int seg_len = 0;
+    std::vector<int64_t> offsets;
+    Segment* d_segments = nullptr;
+    int32_t* d_seg_first = nullptr;
+    int32_t num_segments = 0;
+    std::vector<Segment> h_segments;
+    std::vector<int32_t> h_seg_first;
+};
+
+std::mutex g_tables_mutex;
+std::vector<std::unique_ptr<SegmentTable>> g_tables;
+constexpr size_t kMaxCachedTables = 64;
+
+void build_segments(const int64_t* offsets, int32_t num_tensors, int seg_len, SegmentTable* tab)
+{
+    tab->h_segments.clear();
+    tab->h_seg_first.assign((size_t)num_tensors + 1, 0);
+    for (int32_t t = 0; t < num_tensors; ++t) {
+        tab->h_seg_first[t] = (int32_t)tab->h_segments.size();
+        int64_t b = offsets[t];
+        const int64_t e = offsets[t + 1];
+        while (b < e) {
+            // cut on a 64-element grid of the fused buffer so that interior cuts keep 16-byte
+            // alignment whatever the tensor's own start
+            int64_t next = b / 64 * 64 + seg_len;
+            if (next > e)
+                next = e;
+            tab->h_segments.push_back(Segment{b, (int32_t)(next - b), t});
+            b = next;
+        }
+    }
+    tab->h_seg_first[num_tensors] = (int32_t)tab->h_segments.size();
+    tab->num_segments = (int32_t)tab->h_segments.size();
+}
+
+adasum_status_t get_segment_table(const int64_t* offsets, int32_t num_tensors, int seg_len,
+                                  const SegmentTable** out)
+{
+    int device = 0;
+    ADASUM_CUDA_CHECK(cudaGetDevice(&device));
+    std::lock_guard<std::mutex> lock(g_tables_mutex);
+    for (const auto& tab : g_tables) {
+        if (tab->device == device && tab->seg_len == seg_len &&
+            tab->offsets.size() == (size_t)num_tensors + 1 &&
+            std::memcmp(tab->offsets.data(), offsets, sizeof(int64_t) * tab->offsets.size()) == 0) {
+            *out = tab.get();
+            return ADASUM_OK;
+        }
+    }
+    if (g_tables.size() >= kMaxCachedTables) {
+        // Drop the oldest table.  cudaFree waits for work already submitted to the device, so
+        // kernels still reading the table finish first.
+        SegmentTable* oldest = g_tables.front().get();
+        int current = device;
+        if (oldest->device != current)
+            ADASUM_CUDA_CHECK(cudaSetDevice(oldest->device));
+        cudaError_t e1 = cudaFree(oldest->d_segments), e2 = cudaFree(oldest->d_seg_first);
+        if (oldest->device != current)
+            ADASUM_CUDA_CHECK(cudaSetDevice(current));
+        g_tables.erase(g_tables.begin());
+        if (e1 != cudaSuccess || e2 != cudaSuccess)
+            return fail(ADASUM_ERR_CUDA, "freeing an evicted segment table failed");
+    }
+    auto tab = std::make_unique<SegmentTable>();
+    tab->device = device;
+    tab->seg_len = seg_len;
+    tab->offsets.assign(offsets, offsets + num_tensors + 1);
+    build_segments(offsets, num_tensors, seg_len, tab.get());
+    const size_t seg_bytes = sizeof(Segment) * (tab->h_segments.size() + 1);
+    const size_t first_bytes = sizeof(int32_t) * tab->h_seg_first.size();
+    ADASUM_CUDA_CHECK(cudaMalloc(&tab->d_segments, seg_bytes));
+    cudaError_t err = cudaMalloc(&tab->d_seg_first, first_bytes);
+    // Blocking copies: the table may be used from any stream afterwards.
+    if (err == cudaSuccess && !tab->h_segments.empty())
+        err = cudaMemcpy(tab->d_segments, tab->h_segments.data(),
+                         sizeof(Segment) * tab->h_segments.size(), cudaMemcpyHostToDevice);
+    if (err == cudaSuccess)
+        err = cudaMemcpy(tab->d_seg_first, tab->h_seg_first.data(), first_bytes, cudaMemcpyHostToDevice);
+    if (err != cudaSuccess) {
+        cudaFree(tab->d_segments);
+        cudaFree(tab->d_seg_first);
+        return fail(ADASUM_ERR_CUDA, "segment table upload: %s", cudaGetErrorString(err));
+    }
+    *out = tab.get();
+    g_tables.push_back(std::move(tab));
+    return ADASUM_OK;
+}
+
+// ---- launches ----------------------------------------------------------------------------------
+
+template <typename T, int R, bool VEC>
+void launch_gram(const OperandTable& ops, int operands, int groups_here, const SegmentTable& tab,
+                 float* partials, int groups_total, int group_base, cudaStream_t stream)
+{
+    dim3 grid((unsigned)tab.num_segments, (unsigned)groups_here);
+    gram_partial_kernel<T, R, VEC><<<grid, kThreads, 0, stream>>>(ops, operands, tab.d_segments, partials,
+                                                                  groups_total, group_base);
+}
+
+template <typename T, int R, bool VEC>
+void launch_wsum(const OperandTable& ops, int operands, int groups_here, const SegmentTable& tab,
+                 const float* weights, int groups_total, int group_base, float* dst, int64_t dst_stride,
+                 cudaStream_t stream)
+{
+    dim3 grid((unsigned)tab.num_segments, (unsigned)groups_here);
+    weighted_sum_kernel<T, R, VEC><<<grid, kThreads, 0, stream>>>(ops, operands, tab.d_segments, weights,
+                                                                  groups_total, group_base, dst, dst_stride);
+}
+
+template <int R>
+void launch_weights(const float* partials, const SegmentTable& tab, int32_t num_tensors, int operands,
+                    int groups, float* weights, cudaStream_t stream)
+{
+    dim3 grid((unsigned)num_tensors, (unsigned)groups);
+    tree_weights_kernel<R><<<grid, kThreads, 0, stream>>>(partials, tab.d_seg_first, operands, weights);
+}
+
+struct LevelArgs {
+    const void* const* operand_ptrs;   // host array, `operands` entries
+    int operands;
+    int groups;
+    const SegmentTable* tab;
+    int32_t num_tensors;
+    float* partials;
+    float* weights;
+    float* dst;
+    int64_t dst_stride;
+    bool vec;
+    cudaStream_t stream;
+    int level;
+};
+
+template <typename T, int R>
+adasum_status_t run_level_typed(const LevelArgs& a)
+{
+    constexpr int kGroupsPerLaunch = kMaxOperandsPerLaunch / R;
+    // pass 1
+    for (int g0 = 0; g0 < a.groups; g0 += kGroupsPerLaunch) {
+        const int groups_here = a.groups - g0 < kGroupsPerLaunch ? a.groups - g0 : kGroupsPerLaunch;
+        const int op0 = g0 * R;
+        const int ops_here = a.operands - op0 < kMaxOperandsPerLaunch ? a.operands - op0 : kMaxOperandsPerLaunch;
+        OperandTable table;
+        for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
+            table.ptr[i] = a.operand_ptrs[op0 + (i < ops_here ? i : 0)];
+        if (a.vec)
+            launch_gram<T, R, true>(table, ops_here, groups_here, *a.tab, a.partials, a.groups, g0, a.stream);
+        else
+            launch_gram<T, R, false>(table, ops_here, groups_here, *a.tab, a.partials, a.groups, g0, a.stream);
+        profile_mark(a.stream, ADASUM_KERNEL_GRAM_PARTIAL, a.level, R, false);
+    }
+    launch_weights<R>(a.partials, *a.tab, a.num_tensors, a.operands, a.groups, a.weights, a.stream);
+    profile_mark(a.stream, ADASUM_KERNEL_TREE_WEIGHTS, a.level, R, false);
+    // pass 2
+    for (int g0 = 0; g0 < a.groups; g0 += kGroupsPerLaunch) {
+        const int groups_here = a.groups - g0 < kGroupsPerLaunch ? a.groups - g0 : kGroupsPerLaunch;
+        const int op0 = g0 * R;
+        const int ops_here = a.operands - op0 < kMaxOperandsPerLaunch ? a.operands - op0 : kMaxOperandsPerLaunch;
+        OperandTable table;
+        for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
+            table.ptr[i] = a.operand_ptrs[op0 + (i < ops_here ? i : 0)];
+        if (a.vec)
+            launch_wsum<T, R, true>(table, ops_here, groups_here, *a.tab, a.weights, a.groups, g0, a.dst,
+                                    a.dst_stride, a.stream);
+        else
+            launch_wsum<T, R, false>(table, ops_here, groups_here, *a.tab, a.weights, a.groups, g0, a.dst,
+                                     a.dst_stride, a.stream);
+        profile_mark(a.stream, ADASUM_KERNEL_WEIGHTED_SUM, a.level, R, false);
+    }
+    ADASUM_CUDA_CHECK(cudaGetLastError());
+    return ADASUM_OK;
+}
+
+template <typename T>
+adasum_status_t run_level(int radix, const LevelArgs& a)
+{
+    switch (radix) {
+    case 2: return run_level_typed<T, 2>(a);
+    case 4: return run_level_typed<T, 4>(a);
+    case 8: return run_level_typed<T, 8>(a);
+    case 16: return run_level_typed<T, 16>(a);
+    default: return fail(ADASUM_ERR_ARG, "unsupported radix %d", radix);
+    }
+}
+
+int launches_of(const LevelPlan& plan, int n_workers)
+{
+    if (n_workers == 1)
+        return 1;
+    int n = 0;
+    for (int l = 0; l < plan.num_levels; ++l) {
+        const int per_launch = kMaxOperandsPerLaunch / plan.level[l].radix;
+        const int batches = (plan.level[l].groups + per_launch - 1) / per_launch;
+        n += 2 * batches + 1;
+    }
+    return n;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool ranges_overlap(const void* a, size_t a_bytes, const void* b, size_t b_bytes)
+{
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+    return a0 < b0 + b_bytes && b0 < a0 + a_bytes;
+}
+
+adasum_status_t check_common(const int64_t* offsets, int32_t num_tensors, int32_t n_workers,
+                             adasum_dtype_t dtype)
+{
+    if (!offsets)
+        return fail(ADASUM_ERR_NULL, "tensor_offsets is NULL");
+    if (dtype != ADASUM_F32 && dtype != ADASUM_F16 && dtype != ADASUM_BF16)
+        return fail(ADASUM_ERR_DTYPE, "unknown dtype %d", (int)dtype);
+    if (n_workers < 1 || n_workers > ADASUM_MAX_WORKERS)
+        return fail(ADASUM_ERR_ARG, "n_workers = %d outside 1..%d", n_workers, ADASUM_MAX_WORKERS);
+    if (num_tensors < 0)
+        return fail(ADASUM_ERR_ARG, "num_tensors = %d is negative", num_tensors);
+    if (offsets[0] != 0)
+        return fail(ADASUM_ERR_OFFSETS, "tensor_offsets[0] = %lld, expected 0", (long long)offsets[0]);
+    for (int32_t t = 0; t < num_tensors; ++t)
+        if (offsets[t + 1] < offsets[t])
+            return fail(ADASUM_ERR_OFFSETS, "tensor_offsets decreases at tensor %d", t);
+    return ADASUM_OK;
+}
+
+adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, int32_t num_tensors,
+                            int32_t n_workers, adasum_dtype_t dtype, float* out, void* workspace,
+                            size_t workspace_bytes, uint32_t flags, cudaStream_t stream)
+{
+    g_error[0] = '\0';
+    if (!grads)
+        return fail(ADASUM_ERR_NULL, "grads is NULL");
+    adasum_status_t st = check_common(offsets, num_tensors, n_workers, dtype);
+    if (st != ADASUM_OK)
+        return st;
+    LevelPlan plan;
+    if (!plan_levels(n_workers, dtype, flags, &plan))
+        return fail(ADASUM_ERR_ARG, "invalid flags 0x%x", flags);
+    const int64_t total = offsets[num_tensors];
+    if (total == 0)
+        return ADASUM_OK;
+    if (!out)
+        return fail(ADASUM_ERR_NULL, "out is NULL");
+    if (reinterpret_cast<uintptr_t>(out) & 3u)
+        return fail(ADASUM_ERR_ARG, "out is not 4-byte aligned");
+    const int eb = dtype_bytes(dtype);
+    const size_t in_bytes = (size_t)total * eb, out_bytes = (size_t)total * sizeof(float);
+    bool vec = aligned16(out);
+    for (int w = 0; w < n_workers; ++w) {
+        if (!grads[w])
+            return fail(ADASUM_ERR_NULL, "grads[%d] is NULL", w);
+        if (reinterpret_cast<uintptr_t>(grads[w]) & (uintptr_t)(eb - 1))
+            return fail(ADASUM_ERR_ARG, "grads[%d] is not aligned to its element size", w);
+        if (ranges_overlap(grads[w], in_bytes, out, out_bytes))
+            return fail(ADASUM_ERR_ARG, "out overlaps grads[%d]", w);
+        vec = vec && aligned16(grads[w]);
+    }
+    const Layout lay = make_layout(plan, total, num_tensors);
+    if (n_workers > 1) {
+        if (!workspace)
+            return fail(ADASUM_ERR_WORKSPACE, "workspace is NULL");
+        if (workspace_bytes < lay.total)
+            return fail(ADASUM_ERR_WORKSPACE, "workspace has %zu bytes, need %zu", workspace_bytes, lay.total);
+        if (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1))
+            return fail(ADASUM_ERR_ARG, "workspace is not %zu-byte aligned", kAlign);
+        if (ranges_overlap(workspace, lay.total, out, out_bytes))
+            return fail(ADASUM_ERR_ARG, "workspace overlaps out");
+        for (int w = 0; w < n_workers; ++w)
+            if (ranges_overlap(workspace, lay.total, grads[w], in_bytes))
+                return fail(ADASUM_ERR_ARG, "workspace overlaps grads[%d]", w);
+    }
+
+    profile_mark(stream, -1, 0, 0, true);
+    if (n_workers == 1) {
+        const int64_t blocks = (total + kThreads - 1) / kThreads;
+        const unsigned grid = (unsigned)(blocks < 148 * 16 ? blocks : 148 * 16);
+        if (dtype == ADASUM_F32)
+            convert_kernel<float><<<grid, kThreads, 0, stream>>>((const float*)grads[0], out, total);
+        else if (dtype == ADASUM_F16)
+            convert_kernel<__half><<<grid, kThreads, 0, stream>>>((const __half*)grads[0], out, total);
+        else
+            convert_kernel<__nv_bfloat16><<<grid, kThreads, 0, stream>>>((const __nv_bfloat16*)grads[0], out, total);
+        ADASUM_CUDA_CHECK(cudaGetLastError());
+        profile_mark(stream, ADASUM_KERNEL_CONVERT, 0, 1, false);
+        return ADASUM_OK;
+    }
+
+    char* ws = static_cast<char*>(workspace);
+    std::vector<const void*> operand_ptrs(grads, grads + n_workers);
+    for (int l = 0; l < plan.num_levels; ++l) {
+        const Level& lv = plan.level[l];
+        const SegmentTable* tab = nullptr;
+        st = get_segment_table(offsets, num_tensors, lv.seg_len, &tab);
+        if (st != ADASUM_OK)
+            return st;
+        const bool last = l + 1 == plan.num_levels;
+        LevelArgs a;
+        a.operand_ptrs = operand_ptrs.data();
+        a.operands = lv.operands;
+        a.groups = lv.groups;
+        a.tab = tab;
+        a.num_tensors = num_tensors;
+        a.partials = reinterpret_cast<float*>(ws + lay.partials);
+        a.weights = reinterpret_cast<float*>(ws + lay.weights);
+        a.dst = last ? out : reinterpret_cast<float*>(ws + lay.buffer[l & 1]);
+        a.dst_stride = last ? 0 : lay.padded_elems;
+        a.vec = vec;
+        a.stream = stream;
+        a.level = l;
+        if (l == 0) {
+            if (dtype == ADASUM_F32)
+                st = run_level<float>(lv.radix, a);
+            else if (dtype == ADASUM_F16)
+                st = run_level<__half>(lv.radix, a);
+            else
+                st = run_level<__nv_bfloat16>(lv.radix, a);
+        } else {
+            st = run_level<float>(lv.radix, a);
+        }
+        if (st != ADASUM_OK)
+            return st;
+        if (!last) {
+            operand_ptrs.resize((size_t)lv.groups);
+            for (int g = 0; g < lv.groups; ++g)
+                operand_ptrs[g] = a.dst + (int64_t)g * lay.padded_elems;
+        }
+    }
+    return ADASUM_OK;
+}
+
+}  // namespace
+}  // namespace adasum
+
+extern "C" {
+
+size_t adasum_workspace_bytes(int64_t total_elems, int32_t num_tensors, int32_t n_workers,
+                              adasum_dtype_t dtype, uint32_t flags)
+{
+    using namespace adasum;
+    if (total_elems < 0 || num_tensors < 0 || n_workers < 1 || n_workers > ADASUM_MAX_WORKERS)
+        return 0;
+    if (dtype != ADASUM_F32 && dtype != ADASUM_F16 && dtype != ADASUM_BF16)
+        return 0;
+    LevelPlan plan;
+    if (!plan_levels(n_workers, dtype, flags, &plan))
+        return 0;
+    return make_layout(plan, total_elems, num_tensors).total;
+}
+
+adasum_status_t adasum_plan_info(int64_t total_elems, int32_t num_tensors, int32_t n_workers,
+                                 adasum_dtype_t dtype, uint32_t flags, int32_t* radices,
+                                 int32_t* num_levels, int32_t* num_launches)
+{
+    using namespace adasum;
+    g_error[0] = '\0';
+    if (total_elems < 0 || num_tensors < 0 || n_workers < 1 || n_workers > ADASUM_MAX_WORKERS)
+        return fail(ADASUM_ERR_ARG, "invalid sizes");
+    if (dtype != ADASUM_F32 && dtype != ADASUM_F16 && dtype != ADASUM_BF16)
+        return fail(ADASUM_ERR_DTYPE, "unknown dtype %d", (int)dtype);
+    LevelPlan plan;
+    if (!plan_levels(n_workers, dtype, flags, &plan))
+        return fail(ADASUM_ERR_ARG, "invalid flags 0x%x", flags);
+    if (radices)
+        for (int l = 0; l < plan.num_levels; ++l)
+            radices[l] = plan.level[l].radix;
+    if (num_levels)
+        *num_levels = plan.num_levels;
+    if (num_launches)
+        *num_launches = total_elems == 0 ? 0 : launches_of(plan, n_workers);
+    return ADASUM_OK;
+}
+
+adasum_status_t adasum_reduce(const void* const* grads, const int64_t* tensor_offsets,
+                              int32_t num_tensors, int32_t n_workers, adasum_dtype_t dtype,
+                              float* out, void* workspace, size_t workspace_bytes, uint32_t flags,
+                              void* stream)
+{
+    return adasum::reduce_impl(grads, tensor_offsets, num_tensors, n_workers, dtype, out, workspace,
+                               workspace_bytes, flags, static_cast<cudaStream_t>(stream));
+}
+
+adasum_status_t adasum_pair(const void* a, const void* b, const int64_t* tensor_offsets,
+                            int32_t num_tensors, adasum_dtype_t dtype, float* out, void* workspace,
+                            size_t workspace_bytes, uint32_t flags, void* stream)
+{
+    const void* grads[2] = {a, b};
+    return adasum::reduce_impl(grads, tensor_offsets, num_tensors, 2, dtype, out, workspace,
+                               workspace_bytes, flags, static_cast<cudaStream_t>(stream));
+}
+
+const char* adasum_status_string(adasum_status_t status)
+{
+    switch (status) {
+    case ADASUM_OK: return "ADASUM_OK";
+    case ADASUM_ERR_NULL: return "ADASUM_ERR_NULL";
+    case ADASUM_ERR_ARG: return "ADASUM_ERR_ARG";
+    case ADASUM_ERR_OFFSETS: return "ADASUM_ERR_OFFSETS";
+    case ADASUM_ERR_DTYPE: return "ADASUM_ERR_DTYPE";
+    case ADASUM_ERR_WORKSPACE: return "ADASUM_ERR_WORKSPACE";
+    case ADASUM_ERR_CUDA: return "ADASUM_ERR_CUDA";
+    case ADASUM_ERR_TIMEOUT: return "ADASUM_ERR_TIMEOUT";
+    }
+    return "ADASUM_ERR_UNKNOWN";
+}
+
+const char* adasum_last_error(void) { return adasum::g_error; }
+
+adasum_status_t adasum_profile_enable(int32_t max_launches)
+{
+    using namespace adasum;
+    g_error[0] = '\0';
+    if (max_launches < 1)
+        return fail(ADASUM_ERR_ARG, "max_launches must be positive");
+    std::lock_guard<std::mutex> lock(g_profiler_mutex);
+    g_profiler.enabled = false;
+    const size_t want = (size_t)max_launches * 2;    // room for the call-opening events too
+    while (g_profiler.events.size() < want) {
+        cudaEvent_t ev;
+        cudaError_t err = cudaEventCreate(&ev);
+        if (err != cudaSuccess)
+            return fail(ADASUM_ERR_CUDA, "cudaEventCreate: %s", cudaGetErrorString(err));
+        g_profiler.events.push_back(ev);
+    }
+    g_profiler.marks.resize(g_profiler.events.size());
+    g_profiler.used = 0;
+    g_profiler.overflow = false;
+    g_profiler.enabled = true;
+    return ADASUM_OK;
+}
+
+adasum_status_t adasum_profile_collect(adasum_launch_record_t* records, int32_t capacity, int32_t* count)
+{
+    using namespace adasum;
+    g_error[0] = '\0';
+    if (!count || (capacity > 0 && !records))
+        return fail(ADASUM_ERR_NULL, "records / count is NULL");
+    std::lock_guard<std::mutex> lock(g_profiler_mutex);
+    g_profiler.enabled = false;
+    int32_t n = 0;
+    if (g_profiler.used > 0) {
+        cudaError_t err = cudaEventSynchronize(g_profiler.events[g_profiler.used - 1]);
+        if (err != cudaSuccess)
+            return fail(ADASUM_ERR_CUDA, "cudaEventSynchronize: %s", cudaGetErrorString(err));
+    }
+    for (size_t i = 1; i < g_profiler.used; ++i) {
+        const ProfileMark& m = g_profiler.marks[i];
+        if (m.starts_call)
+            continue;
+        float ms = 0.0f;
+        cudaError_t err = cudaEventElapsedTime(&ms, g_profiler.events[i - 1], g_profiler.events[i]);
+        if (err != cudaSuccess)
+            return fail(ADASUM_ERR_CUDA, "cudaEventElapsedTime: %s", cudaGetErrorString(err));
+        if (n < capacity)
+            records[n] = adasum_launch_record_t{m.kernel, m.level, m.radix, ms};
+        ++n;
+    }
+    *count = n;
+    const bool overflow = g_profiler.overflow;
+    g_profiler.used = 0;
+    g_profiler.overflow = false;
+    if (overflow)
+        return fail(ADASUM_ERR_ARG, "more launches than adasum_profile_enable() reserved; records are incomplete");
+    return ADASUM_OK;
+}
+
+adasum_status_t adasum_shutdown(void)
+{
+    using namespace adasum;
+    g_error[0] = '\0';
+    {
+        std::lock_guard<std::mutex> plock(g_profiler_mutex);
+        g_profiler.enabled = false;
+        for (cudaEvent_t ev : g_profiler.events)
+            cudaEventDestroy(ev);
+        g_profiler.events.clear();
+        g_profiler.marks.clear();
+        g_profiler.used = 0;
+    }
+    std::lock_guard<std::mutex> lock(g_tables_mutex);
+    if (g_tables.empty())
+        return ADASUM_OK;
+    int current = 0;
+    cudaError_t err = cudaGetDevice(&current);
+    bool ok = err == cudaSuccess;
+    for (auto& tab : g_tables) {
+        if (ok && cudaSetDevice(tab->device) == cudaSuccess) {
+            if (cudaFree(tab->d_segments) != cudaSuccess || cudaFree(tab->d_seg_first) != cudaSuccess)
+                ok = false;
+        } else {
+            ok = false;
+        }
+    }
+    g_tables.clear();
+    if (err == cudaSuccess)
+        cudaSetDevice(current);
+    return ok ? ADASUM_OK : fail(ADASUM_ERR_CUDA, "adasum_shutdown: a CUDA call failed");
+}
+
+}  // extern "C"

@@ -135,9 +135,11 @@ def per_tensor_parameters(spec: WorkloadSpec, num_tensors: int):
     return rho, sigma, zeroed
 
 
-def generate(spec: WorkloadSpec | str, device="cpu", tensor_sizes=None, n_workers=None) -> Workload:
+def generate(spec: WorkloadSpec | str, device="cpu", tensor_sizes=None, n_workers=None,
+             replica: int = 0) -> Workload:
     """Materialise a workload on ``device``.  ``tensor_sizes`` / ``n_workers`` override the
-    spec's (used for reduced-size test cases that keep the same structure)."""
+    spec's (used for reduced-size test cases that keep the same structure); ``replica`` selects
+    an independent draw of the element noise (one per GPU in a multi-GPU run)."""
     if isinstance(spec, str):
         spec = SPECS[spec]
     if n_workers is not None:
@@ -147,7 +149,7 @@ def generate(spec: WorkloadSpec | str, device="cpu", tensor_sizes=None, n_worker
     total = int(offsets[-1])
     rho, sigma, zeroed = per_tensor_parameters(spec, len(sizes))
     device = torch.device(device)
-    seed = BASE_SEED + 1000 * spec.seed_index
+    seed = BASE_SEED + 1000 * spec.seed_index + 100_000 * int(replica)
 
     lengths = torch.as_tensor(np.asarray(sizes, dtype=np.int64), device=device)
     shared_scale = torch.repeat_interleave(
