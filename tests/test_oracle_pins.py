@@ -7,6 +7,7 @@ import numpy as np
 import pytest
 
 from oracle import adasum_oracle as oracle
+from tree_algebra import leaf_weights_from_gram
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -224,31 +225,11 @@ def test_norm_identity_and_bounds():
 
 
 # -- every tree node is a linear combination of the leaves: weights from the Gram matrix ------
-def _leaf_weights_from_gram(gram):
-    n = gram.shape[0]
-    c = np.ones(n)
-    blocks = [([i], gram[i, i]) for i in range(n)]
-    while len(blocks) > 1:
-        nxt = []
-        for i in range(0, len(blocks) - 1, 2):
-            (left, na), (right, nb) = blocks[i], blocks[i + 1]
-            d = sum(c[p] * c[q] * gram[p, q] for p in left for q in right)
-            ca = 1.0 if na == 0 else 1.0 - d / (2 * na)
-            cb = 1.0 if nb == 0 else 1.0 - d / (2 * nb)
-            c[left] *= ca
-            c[right] *= cb
-            nxt.append((left + right, ca * ca * na + cb * cb * nb + 2 * ca * cb * d))
-        if len(blocks) % 2:
-            nxt.append(blocks[-1])
-        blocks = nxt
-    return c
-
-
 @pytest.mark.parametrize("n", [2, 3, 5, 8, 16])
 def test_gram_derived_leaf_weights_reproduce_the_tree(n):
     rng = _rng(200 + n)
     gs = np.stack([rng.standard_normal(48) + 0.4 for _ in range(n)])
-    c = _leaf_weights_from_gram(gs @ gs.T)
+    c = leaf_weights_from_gram(gs @ gs.T)
     np.testing.assert_allclose(oracle.adasum_reduce(list(gs)), c @ gs, rtol=1e-12, atol=1e-14)
 
 
