@@ -355,6 +355,20 @@ def reference_arm(args):
 
 # ---- main ---------------------------------------------------------------------------------------------
 
+def aggregate_over_ranks(ms_local: float, bytes_local: float, world: int, device="cpu"):
+    """Whole-job figures of a run with one independent workload per rank: the step time is the
+    slowest rank's, the work is the sum over ranks.  Returns (ms, total bytes)."""
+    if world <= 1:
+        return ms_local, bytes_local
+    import torch.distributed as dist
+
+    t = torch.tensor([ms_local], device=device, dtype=torch.float64)
+    b = torch.tensor([bytes_local], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(b, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(b.item())
+
+
 def measure_workload(lib, name, steps, warmup, flags, replica, world, sampler=None):
     wl = workloads.generate(name, device="cuda", replica=replica)
     ms, out, ws = time_reduce(lib, wl, steps, warmup, flags, world=world, sampler=sampler)
@@ -392,12 +406,8 @@ def cuda_arm(args):
     steps, warmup = max(args.steps, 1), max(args.warmup, 3)
 
     wl, ms_local, out, ws = measure_workload(lib, args.workload, steps, warmup, flags, rank, world, sampler)
-    ms = ms_local
-    if world > 1:
-        t = torch.tensor([ms_local], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * wl.input_bytes / (ms * 1e-3) / 1e9
+    ms, job_bytes = aggregate_over_ranks(ms_local, float(wl.input_bytes), world, "cuda")
+    value = job_bytes / (ms * 1e-3) / 1e9
 
     rows, ms_instrumented, info, levels = kernel_breakdown(lib, wl, steps, flags, out, ws)
     top = rows[0]
@@ -417,12 +427,8 @@ def cuda_arm(args):
 
     e2e_steps = min(steps, 20)
     e2e_ms_local, h2d, d2h, _ = time_e2e(lib, wl, e2e_steps, flags, out, ws)
-    e2e_ms = e2e_ms_local
-    if world > 1:
-        t = torch.tensor([e2e_ms_local], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e = {"value": world * wl.input_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+    e2e_ms, _ = aggregate_over_ranks(e2e_ms_local, float(wl.input_bytes), world, "cuda")
+    e2e = {"value": job_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps}
 
     cpu_baseline = None

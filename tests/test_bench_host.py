@@ -1,0 +1,70 @@
+"""Host-side logic of bench.py that runs without a GPU: the multi-rank aggregation (gloo, two
+ranks), the oracle sampling, the roofline byte counts and the reference arm's rank handling."""
+import json
+import os
+import subprocess
+import sys
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+
+import bench  # noqa: E402
+from paper_2006_02924_b200 import workloads  # noqa: E402
+
+
+def _rank_main(rank, world, port, results):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    ms, total = bench.aggregate_over_ranks(10.0 + 5.0 * rank, 1000.0 * (rank + 1), world, "cpu")
+    results[rank] = (ms, total)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_aggregation_takes_slowest_rank_and_sums_work():
+    world = 2
+    with mp.Manager() as manager:
+        results = manager.dict()
+        mp.spawn(_rank_main, args=(world, 29653, results), nprocs=world, join=True)
+        assert results[0] == results[1] == (15.0, 3000.0)
+    assert bench.aggregate_over_ranks(7.0, 11.0, 1) == (7.0, 11.0)
+
+
+def test_algorithmic_bytes_per_launch():
+    levels = [{"radix": 16, "operands": 256, "groups": 16}, {"radix": 16, "operands": 16, "groups": 1}]
+    p = 1000
+    assert bench.algorithmic_bytes({"kernel": "gram_partial", "level": 0}, levels, p, 2) == 256 * p * 2
+    assert bench.algorithmic_bytes({"kernel": "weighted_sum", "level": 0}, levels, p, 2) == 256 * p * 2 + 16 * p * 4
+    assert bench.algorithmic_bytes({"kernel": "gram_partial", "level": 1}, levels, p, 2) == 16 * p * 4
+    assert bench.algorithmic_bytes({"kernel": "weighted_sum", "level": 1}, levels, p, 2) == 16 * p * 4 + p * 4
+    assert bench.algorithmic_bytes({"kernel": "tree_weights", "level": 0}, levels, p, 2) == 0
+
+
+def test_oracle_sample_is_bounded_and_whole_tensors():
+    wl = workloads.generate("c2", tensor_sizes=workloads.reduced_sizes(workloads.resnet50_tensor_sizes(), 64))
+    budget = 2.0 * 7 * 50_000
+    chosen = bench.oracle_sample(wl, budget)
+    sizes = np.diff(wl.offsets)
+    assert chosen == sorted(set(chosen)) and len(chosen) >= 1
+    assert 2.0 * 7 * sizes[chosen].sum() <= budget + 2.0 * 7 * sizes.max()
+    dt, nbytes, threads = bench.run_oracle(wl, chosen, threads=1)
+    assert nbytes == 8 * int(sizes[chosen].sum()) * 4 and dt > 0 and threads == 1
+
+
+def test_reference_arm_prints_one_line_on_rank0_only():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "c1",
+                          "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0 and out.stdout.strip() == ""
+    env["RANK"] = "0"
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "c1",
+                          "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["unit"] == "GB/s" and line["value"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
