@@ -132,6 +132,39 @@ adasum_status_t adasum_pair(const void* a, const void* b, const int64_t* tensor_
                             void* workspace, size_t workspace_bytes, uint32_t flags,
                             void* stream);
 
+/*
+ * adasum_pair for callers that must not allocate device memory (the paper has no counterpart).
+ *
+ * Some hosts of this library cannot call cudaMalloc where they run the reduction: code inside a
+ * framework's memory-pool callback, a process whose whole GPU budget was handed to another
+ * allocator at start-up, a real-time loop that forbids driver allocations after initialisation.
+ * adasum_pair needs a workspace from its caller and builds a cached segment table with cudaMalloc
+ * on first use; this entry point needs neither.  Its scratch (segment table, per-segment partial
+ * sums, per-tensor coefficients; about 0.5 MB) is a fixed array inside the library's device
+ * image, so every GPU that loads the library carries it until the process exits.
+ *
+ *   a, b, tensor_offsets, num_tensors, dtype, out, stream   as for adasum_pair
+ *
+ * Limits: at most ADASUM_NOALLOC_MAX_ELEMS elements per input and ADASUM_NOALLOC_MAX_TENSORS
+ * tensors; larger arguments return ADASUM_ERR_ARG with a message and launch nothing.  The result
+ * equals adasum_pair's with default flags.
+ *
+ * The call performs no cudaMalloc / cudaFree and uses no allocating library routine; it enqueues
+ * two small host-to-device copies (the segment table of this call) and three kernels on `stream`.
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ * that device current); make that first call before any stream capture begins.
+ *
+ * All calls on a device share the one scratch array, which keeps the previous call's contents.
+ * Every entry that a call reads is first rewritten by the same call, so nothing has to be
+ * cleared; but two calls whose work overlaps on the GPU (different streams, no ordering between
+ * them) race on it.  Serialise them with events or use adasum_pair with separate workspaces.
+ */
+#define ADASUM_NOALLOC_MAX_ELEMS 67108864    /* 2^26 elements per input */
+#define ADASUM_NOALLOC_MAX_TENSORS 4096
+
+adasum_status_t adasum_pair_noalloc(const void* a, const void* b, const int64_t* tensor_offsets,
+                                    int32_t num_tensors, adasum_dtype_t dtype, float* out, void* stream);
+
 /* Static, human-readable name of a status code. */
 const char* adasum_status_string(adasum_status_t status);
 

@@ -193,3 +193,28 @@ def adasum_profile_collect(capacity: int = 4096) -> list[dict]:
         raise AdasumError(status)
     return [{"kernel": KERNEL_NAMES.get(r.kernel, str(r.kernel)), "level": r.level, "radix": r.radix,
              "ms": float(r.ms)} for r in records[:min(count.value, capacity)]]
+
+
+ADASUM_NOALLOC_MAX_ELEMS = 1 << 26
+ADASUM_NOALLOC_MAX_TENSORS = 4096
+
+_lib.adasum_pair_noalloc.restype = ctypes.c_int
+_lib.adasum_pair_noalloc.argtypes = [ctypes.c_void_p, ctypes.c_void_p, _i64p, ctypes.c_int32, ctypes.c_int,
+                                     ctypes.c_void_p, ctypes.c_void_p]
+
+
+def adasum_pair_noalloc(a, b, tensor_offsets=None, out=None, stream=None):
+    """``adasum_pair_noalloc`` of the C ABI: the pair operator for callers that cannot allocate
+    device memory.  The library uses a fixed scratch array of its own instead of a workspace, so
+    pass ``out`` to keep this wrapper from allocating either (it allocates ``out`` with torch only
+    when none is given)."""
+    total = a.numel()
+    offs = _offsets_array(tensor_offsets, total)
+    if out is None:
+        out = torch.empty(total, dtype=torch.float32, device=a.device)
+    with torch.cuda.device(a.device):
+        status = _lib.adasum_pair_noalloc(a.data_ptr(), b.data_ptr(), offs.ctypes.data_as(_i64p), offs.size - 1,
+                                          _dtype_code(a.dtype), out.data_ptr(), _stream_handle(stream))
+    if status != ADASUM_OK:
+        raise AdasumError(status)
+    return out

@@ -510,6 +510,127 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     return ADASUM_OK;
 }
 
+// ---- pair operator without any device allocation -------------------------------------------------
+//
+// Scratch for adasum_pair_noalloc: the segment table, the per-segment partial sums and the
+// per-tensor coefficients live in one file-scope device array that every GPU loading this library
+// holds until the process exits.  In host code `g_noalloc_scratch` is only a handle for
+// cudaGetSymbolAddress; the kernels receive the device address obtained from it.
+
+constexpr int64_t kNoallocMaxElems = ADASUM_NOALLOC_MAX_ELEMS;
+constexpr int32_t kNoallocMaxTensors = ADASUM_NOALLOC_MAX_TENSORS;
+constexpr int kNoallocSegLen = 8192;
+constexpr int64_t kNoallocMaxSegments = kNoallocMaxElems / kNoallocSegLen + 2 * (int64_t)kNoallocMaxTensors + 1;
+constexpr size_t kNoallocSegBytes = ((size_t)kNoallocMaxSegments * sizeof(Segment) + 255) / 256 * 256;
+constexpr size_t kNoallocFirstBytes = ((size_t)(kNoallocMaxTensors + 1) * sizeof(int32_t) + 255) / 256 * 256;
+constexpr size_t kNoallocPartialBytes = ((size_t)kNoallocMaxSegments * gram_entries(2) * sizeof(float) + 255) / 256 * 256;
+constexpr size_t kNoallocWeightBytes = ((size_t)kNoallocMaxTensors * 2 * sizeof(float) + 255) / 256 * 256;
+constexpr size_t kNoallocScratchBytes = kNoallocSegBytes + kNoallocFirstBytes + kNoallocPartialBytes + kNoallocWeightBytes;
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoallocScratchBytes];
+
+constexpr int kNoallocMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+unsigned char* g_noalloc_device_ptr[kNoallocMaxDevices] = {};
+
+// Device address of the scratch array on the current device (looked up once per device).
+adasum_status_t noalloc_scratch(unsigned char** ptr)
+{
+    int device = 0;
+    ADASUM_CUDA_CHECK(cudaGetDevice(&device));
+    if (device < 0 || device >= kNoallocMaxDevices)
+        return fail(ADASUM_ERR_ARG, "device index %d is beyond the %d devices this entry point tracks", device,
+                    kNoallocMaxDevices);
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_device_ptr[device]) {
+        void* addr = nullptr;
+        ADASUM_CUDA_CHECK(cudaGetSymbolAddress(&addr, g_noalloc_scratch));
+        g_noalloc_device_ptr[device] = static_cast<unsigned char*>(addr);
+    }
+    *ptr = g_noalloc_device_ptr[device];
+    return ADASUM_OK;
+}
+
+template <typename T>
+void noalloc_launch(bool vec, const OperandTable& ops, const SegmentTable& tab, int32_t num_tensors,
+                    float* partials, float* weights, float* out, cudaStream_t stream)
+{
+    if (vec) {
+        launch_gram<T, 2, true>(ops, 2, 1, tab, partials, 1, 0, stream);
+        launch_weights<2>(partials, tab, num_tensors, 2, 1, weights, stream);
+        launch_wsum<T, 2, true>(ops, 2, 1, tab, weights, 1, 0, out, 0, stream);
+    } else {
+        launch_gram<T, 2, false>(ops, 2, 1, tab, partials, 1, 0, stream);
+        launch_weights<2>(partials, tab, num_tensors, 2, 1, weights, stream);
+        launch_wsum<T, 2, false>(ops, 2, 1, tab, weights, 1, 0, out, 0, stream);
+    }
+}
+
+adasum_status_t pair_noalloc_impl(const void* a, const void* b, const int64_t* offsets, int32_t num_tensors,
+                                  adasum_dtype_t dtype, float* out, cudaStream_t stream)
+{
+    g_error[0] = '\0';
+    if (!a || !b)
+        return fail(ADASUM_ERR_NULL, "an input pointer is NULL");
+    adasum_status_t st = check_common(offsets, num_tensors, 2, dtype);
+    if (st != ADASUM_OK)
+        return st;
+    const int64_t total = offsets[num_tensors];
+    if (num_tensors > kNoallocMaxTensors)
+        return fail(ADASUM_ERR_ARG, "num_tensors = %d exceeds the static scratch limit of %d tensors", num_tensors,
+                    kNoallocMaxTensors);
+    if (total > kNoallocMaxElems)
+        return fail(ADASUM_ERR_ARG, "%lld elements exceed the static scratch limit of %lld elements",
+                    (long long)total, (long long)kNoallocMaxElems);
+    if (total == 0)
+        return ADASUM_OK;
+    if (!out)
+        return fail(ADASUM_ERR_NULL, "out is NULL");
+    if (reinterpret_cast<uintptr_t>(out) & 3u)
+        return fail(ADASUM_ERR_ARG, "out is not 4-byte aligned");
+    const int eb = dtype_bytes(dtype);
+    const size_t in_bytes = (size_t)total * eb, out_bytes = (size_t)total * sizeof(float);
+    const void* in[2] = {a, b};
+    bool vec = aligned16(out);
+    for (int w = 0; w < 2; ++w) {
+        if (reinterpret_cast<uintptr_t>(in[w]) & (uintptr_t)(eb - 1))
+            return fail(ADASUM_ERR_ARG, "input %d is not aligned to its element size", w);
+        if (ranges_overlap(in[w], in_bytes, out, out_bytes))
+            return fail(ADASUM_ERR_ARG, "out overlaps input %d", w);
+        vec = vec && aligned16(in[w]);
+    }
+
+    unsigned char* scratch = nullptr;
+    st = noalloc_scratch(&scratch);
+    if (st != ADASUM_OK)
+        return st;
+    SegmentTable tab;                       // host-side only; its device pointers aim into the scratch
+    build_segments(offsets, num_tensors, kNoallocSegLen, &tab);
+    if ((int64_t)tab.num_segments > kNoallocMaxSegments)
+        return fail(ADASUM_ERR_ARG, "segment table does not fit the static scratch");
+    tab.d_segments = reinterpret_cast<Segment*>(scratch);
+    tab.d_seg_first = reinterpret_cast<int32_t*>(scratch + kNoallocSegBytes);
+    float* partials = reinterpret_cast<float*>(scratch + kNoallocSegBytes + kNoallocFirstBytes);
+    float* weights = reinterpret_cast<float*>(scratch + kNoallocSegBytes + kNoallocFirstBytes + kNoallocPartialBytes);
+    // The host vectors are pageable memory: cudaMemcpyAsync has read them completely when it
+    // returns, and the copies are ordered before the kernels on `stream`.
+    ADASUM_CUDA_CHECK(cudaMemcpyAsync(tab.d_segments, tab.h_segments.data(), sizeof(Segment) * tab.h_segments.size(),
+                                      cudaMemcpyHostToDevice, stream));
+    ADASUM_CUDA_CHECK(cudaMemcpyAsync(tab.d_seg_first, tab.h_seg_first.data(),
+                                      sizeof(int32_t) * tab.h_seg_first.size(), cudaMemcpyHostToDevice, stream));
+    OperandTable ops;
+    for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
+        ops.ptr[i] = in[i < 2 ? i : 0];
+    if (dtype == ADASUM_F32)
+        noalloc_launch<float>(vec, ops, tab, num_tensors, partials, weights, out, stream);
+    else if (dtype == ADASUM_F16)
+        noalloc_launch<__half>(vec, ops, tab, num_tensors, partials, weights, out, stream);
+    else
+        noalloc_launch<__nv_bfloat16>(vec, ops, tab, num_tensors, partials, weights, out, stream);
+    ADASUM_CUDA_CHECK(cudaGetLastError());
+    return ADASUM_OK;
+}
+
 }  // namespace
 }  // namespace adasum
 
@@ -568,6 +689,13 @@ adasum_status_t adasum_pair(const void* a, const void* b, const int64_t* tensor_
     const void* grads[2] = {a, b};
     return adasum::reduce_impl(grads, tensor_offsets, num_tensors, 2, dtype, out, workspace,
                                workspace_bytes, flags, static_cast<cudaStream_t>(stream));
+}
+
+adasum_status_t adasum_pair_noalloc(const void* a, const void* b, const int64_t* tensor_offsets,
+                                    int32_t num_tensors, adasum_dtype_t dtype, float* out, void* stream)
+{
+    return adasum::pair_noalloc_impl(a, b, tensor_offsets, num_tensors, dtype, out,
+                                     static_cast<cudaStream_t>(stream));
 }
 
 const char* adasum_status_string(adasum_status_t status)
