@@ -75,7 +75,11 @@ typedef enum {
  *
  *   bits 0..7    radix of the first level: 0 = choose automatically, else 2, 4, 8 or 16
  *   bits 8..15   radix of the later levels: 0 = same rule as the first level
+ *   bit 16       ADASUM_FLAG_SIMPLE_KERNELS: use the register-only kernels everywhere instead
+ *                of the shared-memory-pipelined ones (same results up to summation order;
+ *                for comparison and debugging)
  */
+#define ADASUM_FLAG_SIMPLE_KERNELS (1u << 16)
 #define ADASUM_RADIX_AUTO 0u
 #define ADASUM_FLAGS_RADIX(first, later) (((uint32_t)(first) & 0xffu) | (((uint32_t)(later) & 0xffu) << 8))
 

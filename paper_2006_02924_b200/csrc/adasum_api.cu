@@ -77,7 +77,9 @@ size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 int dtype_bytes(adasum_dtype_t dtype) { return dtype == ADASUM_F32 ? 4 : 2; }
 
-bool valid_radix(int r) { return r == 2 || r == 4 || r == 8 || r == 16; }
+int max_radix_for(adasum_dtype_t dtype) { return dtype == ADASUM_F32 ? 32 : 64; }
+
+bool valid_radix(int r) { return r == 2 || r == 4 || r == 8 || r == 16 || r == 32 || r == 64; }
 
 int pow2_ceil(int x)
 {
@@ -87,15 +89,46 @@ int pow2_ceil(int x)
     return p;
 }
 
-// Elements per segment for a level of radix R.  Per-block fp32 accumulation never spans more
-// than this many elements; longer tensors are finished in fp64.
-int segment_length(int radix) { return radix >= 16 ? 16384 : 8192; }
+// Which Gram kernel serves a level.
+enum GramKind {
+    GRAM_SIMPLE,      // fp32 pipes, operands in registers (any alignment, radix <= 16)
+    GRAM_PIPELINED,   // fp32 pipes, persistent blocks, cp.async staging (16-byte aligned, radix <= 8)
+    GRAM_MMA          // tensor cores (radix >= 16)
+};
+
+GramKind gram_kind(int radix, bool vec, bool simple_kernels)
+{
+    if (radix >= 32 || (radix == 16 && !simple_kernels))
+        return GRAM_MMA;
+    return vec && !simple_kernels ? GRAM_PIPELINED : GRAM_SIMPLE;
+}
+
+// Elements per segment.  One block accumulates a whole segment in fp32 (per thread: segment /
+// 256 elements; on the tensor cores: per warp segment / 8), longer tensors are finished in fp64.
+int gram_segment_length(GramKind kind, int64_t total)
+{
+    switch (kind) {
+    case GRAM_PIPELINED: return 32768;
+    case GRAM_MMA: return total >= (int64_t(1) << 26) ? 32768 : 8192;
+    default: return total >= (int64_t(1) << 23) ? 8192 : 2048;
+    }
+}
+int min_gram_segment_length(int radix, int64_t total)
+{
+    int best = 1 << 30;
+    for (int vec = 0; vec < 2; ++vec)
+        for (int simple = 0; simple < 2; ++simple) {
+            const int len = gram_segment_length(gram_kind(radix, vec != 0, simple != 0), total);
+            best = len < best ? len : best;
+        }
+    return best;
+}
+int wsum_segment_length(int64_t total) { return total >= (int64_t(1) << 23) ? 8192 : 2048; }
 
 struct Level {
     int radix;
     int operands;   // operands entering the level
     int groups;     // operands leaving it
-    int seg_len;
 };
 
 struct LevelPlan {
@@ -105,29 +138,39 @@ struct LevelPlan {
 
 bool plan_levels(int n_workers, adasum_dtype_t dtype, uint32_t flags, LevelPlan* plan)
 {
-    (void)dtype;
     const int first = (int)(flags & 0xffu), later_flag = (int)((flags >> 8) & 0xffu);
-    if ((flags >> 16) != 0)
+    if ((flags >> 17) != 0)
         return false;
-    if (first != 0 && !valid_radix(first))
+    if (first != 0 && (!valid_radix(first) || first > max_radix_for(dtype)))
         return false;
-    if (later_flag != 0 && !valid_radix(later_flag))
+    if (later_flag != 0 && (!valid_radix(later_flag) || later_flag > max_radix_for(ADASUM_F32)))
         return false;
-    const int later = later_flag != 0 ? later_flag : first;
+    if ((flags & ADASUM_FLAG_SIMPLE_KERNELS) && (first > 16 || later_flag > 16))
+        return false;
+    int later = later_flag != 0 ? later_flag : first;
+    if (later > max_radix_for(ADASUM_F32))
+        later = max_radix_for(ADASUM_F32);      // intermediates are fp32
+    const int cap_auto = (flags & ADASUM_FLAG_SIMPLE_KERNELS) ? 16 : 64;
     int m = n_workers;
     plan->num_levels = 0;
     while (m > 1) {
         if (plan->num_levels == ADASUM_MAX_LEVELS)
             return false;
-        const int want = plan->num_levels == 0 ? first : later;
-        int radix = want != 0 ? want : kMaxRadix;
+        const bool first_level = plan->num_levels == 0;
+        const int want = first_level ? first : later;
+        int radix = want;
+        if (radix == 0) {
+            radix = max_radix_for(first_level ? dtype : ADASUM_F32);
+            if (first_level ? dtype == ADASUM_F32 : true)
+                radix = 16;
+            radix = radix < cap_auto ? radix : cap_auto;
+        }
         if (radix > pow2_ceil(m))
             radix = pow2_ceil(m);
         Level& lv = plan->level[plan->num_levels++];
         lv.radix = radix;
         lv.operands = m;
         lv.groups = (m + radix - 1) / radix;
-        lv.seg_len = segment_length(radix);
         m = lv.groups;
     }
     return true;
@@ -139,8 +182,8 @@ int64_t segment_bound(int64_t total, int32_t num_tensors, int seg_len)
 }
 
 struct Layout {
-    size_t partials = 0, weights = 0, buffer[2] = {0, 0};
-    size_t partials_bytes = 0, weights_bytes = 0, buffer_bytes[2] = {0, 0};
+    size_t partials = 0, weights = 0, gram64 = 0, buffer[2] = {0, 0};
+    size_t partials_bytes = 0, weights_bytes = 0, gram64_bytes = 0, buffer_bytes[2] = {0, 0};
     int64_t padded_elems = 0;
     size_t total = 0;
 };
@@ -151,13 +194,20 @@ Layout make_layout(const LevelPlan& plan, int64_t total_elems, int32_t num_tenso
     lay.padded_elems = (total_elems + 63) / 64 * 64;
     for (int l = 0; l < plan.num_levels; ++l) {
         const Level& lv = plan.level[l];
-        const size_t p = (size_t)segment_bound(total_elems, num_tensors, lv.seg_len) * lv.groups *
-                         gram_entries(lv.radix) * sizeof(float);
+        const size_t p = (size_t)segment_bound(total_elems, num_tensors,
+                                               min_gram_segment_length(lv.radix, total_elems)) *
+                         lv.groups * gram_entries(lv.radix) * sizeof(float);
         const size_t w = (size_t)(num_tensors > 0 ? num_tensors : 1) * lv.groups * lv.radix * sizeof(float);
         if (p > lay.partials_bytes)
             lay.partials_bytes = p;
         if (w > lay.weights_bytes)
             lay.weights_bytes = w;
+        if (lv.radix >= 32) {
+            const size_t g64 = (size_t)(num_tensors > 0 ? num_tensors : 1) * lv.groups * gram_entries(lv.radix) *
+                               sizeof(double);
+            if (g64 > lay.gram64_bytes)
+                lay.gram64_bytes = g64;
+        }
         if (l + 1 < plan.num_levels) {      // this level's output is an intermediate
             const size_t b = (size_t)lv.groups * lay.padded_elems * sizeof(float);
             if (b > lay.buffer_bytes[l & 1])
@@ -169,6 +219,8 @@ Layout make_layout(const LevelPlan& plan, int64_t total_elems, int32_t num_tenso
     off += align_up(lay.partials_bytes);
     lay.weights = off;
     off += align_up(lay.weights_bytes);
+    lay.gram64 = off;
+    off += align_up(lay.gram64_bytes);
     lay.buffer[0] = off;
     off += align_up(lay.buffer_bytes[0]);
     lay.buffer[1] = off;
@@ -271,13 +323,94 @@ adasum_status_t get_segment_table(const int64_t* offsets, int32_t num_tensors, i
 
 // ---- launches ----------------------------------------------------------------------------------
 
-template <typename T, int R, bool VEC>
-void launch_gram(const OperandTable& ops, int operands, int groups_here, const SegmentTable& tab,
-                 float* partials, int groups_total, int group_base, cudaStream_t stream)
+int multiprocessor_count()
 {
-    dim3 grid((unsigned)tab.num_segments, (unsigned)groups_here);
-    gram_partial_kernel<T, R, VEC><<<grid, kThreads, 0, stream>>>(ops, operands, tab.d_segments, partials,
-                                                                  groups_total, group_base);
+    static int cached[64] = {};
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64)
+        return 148;
+    if (cached[device] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || n <= 0)
+            n = 148;
+        cached[device] = n;
+    }
+    return cached[device];
+}
+
+// Opt a kernel in to `bytes` of dynamic shared memory, once per device.
+template <typename Kernel>
+cudaError_t allow_dynamic_smem(Kernel kernel, size_t bytes, bool (&configured)[64])
+{
+    int device = 0;
+    cudaError_t err = cudaGetDevice(&device);
+    if (err != cudaSuccess)
+        return err;
+    if (device < 0 || device >= 64)
+        return cudaErrorInvalidDevice;
+    if (!configured[device]) {
+        err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+        if (err != cudaSuccess)
+            return err;
+        configured[device] = true;
+    }
+    return cudaSuccess;
+}
+
+constexpr int kGramStages = 3;
+
+template <typename T, int R, bool VEC>
+cudaError_t launch_gram(GramKind kind, const OperandTable& ops, int operands, int groups_here,
+                        const SegmentTable& tab, float* partials, int groups_total, int group_base,
+                        cudaStream_t stream)
+{
+    if constexpr (R >= 16) {
+        if (kind == GRAM_MMA) {
+            if constexpr (R <= 32 || sizeof(T) == 2) {
+                constexpr size_t smem = mma_smem_bytes<T, R>();
+                auto kernel = gram_partial_mma_kernel<T, R, VEC>;
+                static bool configured[64] = {};
+                cudaError_t err = allow_dynamic_smem(kernel, smem, configured);
+                if (err != cudaSuccess)
+                    return err;
+                dim3 grid((unsigned)tab.num_segments, (unsigned)groups_here);
+                kernel<<<grid, kThreads, smem, stream>>>(ops, operands, tab.d_segments, partials, groups_total,
+                                                         group_base);
+                return cudaSuccess;
+            } else {
+                return cudaErrorInvalidValue;
+            }
+        }
+    }
+    if constexpr (R <= 8 && VEC) {
+        if (kind == GRAM_PIPELINED) {
+            constexpr size_t smem = (size_t)kGramStages * R * kThreads * 16;
+            auto kernel = gram_partial_pipelined_kernel<T, R, kGramStages>;
+            static bool configured[64] = {};
+            cudaError_t err = allow_dynamic_smem(kernel, smem, configured);
+            if (err != cudaSuccess)
+                return err;
+            // persistent blocks: fill every SM, never more blocks than fit at once
+            int blocks_x = multiprocessor_count() * pipelined_min_blocks<R>() / groups_here;
+            if (blocks_x > tab.num_segments)
+                blocks_x = tab.num_segments;
+            if (blocks_x < 1)
+                blocks_x = 1;
+            dim3 grid((unsigned)blocks_x, (unsigned)groups_here);
+            kernel<<<grid, kThreads, smem, stream>>>(ops, operands, tab.d_segments, tab.num_segments, partials,
+                                                     groups_total, group_base);
+            return cudaSuccess;
+        }
+    }
+    if constexpr (R <= 16) {
+        if (kind == GRAM_SIMPLE) {
+            dim3 grid((unsigned)tab.num_segments, (unsigned)groups_here);
+            gram_partial_kernel<T, R, VEC><<<grid, kThreads, 0, stream>>>(ops, operands, tab.d_segments, partials,
+                                                                          groups_total, group_base);
+            return cudaSuccess;
+        }
+    }
+    return cudaErrorInvalidValue;
 }
 
 template <typename T, int R, bool VEC>
@@ -291,20 +424,30 @@ void launch_wsum(const OperandTable& ops, int operands, int groups_here, const S
 }
 
 template <int R>
-void launch_weights(const float* partials, const SegmentTable& tab, int32_t num_tensors, int operands,
-                    int groups, float* weights, cudaStream_t stream)
+cudaError_t launch_weights(const float* partials, const SegmentTable& tab, int32_t num_tensors, int operands,
+                           int groups, double* gram64, float* weights, cudaStream_t stream, int* launches)
 {
-    dim3 grid((unsigned)num_tensors, (unsigned)groups);
-    tree_weights_kernel<R><<<grid, kThreads, 0, stream>>>(partials, tab.d_seg_first, operands, weights);
+    dim3 grid((unsigned)num_tensors, (unsigned)groups, (unsigned)tree_entry_blocks(R));
+    gram_finish_kernel<R><<<grid, kTreeThreads, 0, stream>>>(partials, tab.d_seg_first, operands, gram64, weights);
+    *launches = 1;
+    if constexpr (tree_entry_blocks(R) > 1) {
+        dim3 grid2((unsigned)num_tensors, (unsigned)groups);
+        tree_weights_kernel<R><<<grid2, kThreads, 0, stream>>>(gram64, operands, weights);
+        *launches = 2;
+    }
+    return cudaSuccess;
 }
 
 struct LevelArgs {
     const void* const* operand_ptrs;   // host array, `operands` entries
     int operands;
     int groups;
-    const SegmentTable* tab;
+    GramKind kind;
+    const SegmentTable* gram_tab;
+    const SegmentTable* wsum_tab;
     int32_t num_tensors;
     float* partials;
+    double* gram64;
     float* weights;
     float* dst;
     int64_t dst_stride;
@@ -326,12 +469,16 @@ adasum_status_t run_level_typed(const LevelArgs& a)
         for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
             table.ptr[i] = a.operand_ptrs[op0 + (i < ops_here ? i : 0)];
         if (a.vec)
-            launch_gram<T, R, true>(table, ops_here, groups_here, *a.tab, a.partials, a.groups, g0, a.stream);
+            ADASUM_CUDA_CHECK((launch_gram<T, R, true>(a.kind, table, ops_here, groups_here, *a.gram_tab,
+                                                       a.partials, a.groups, g0, a.stream)));
         else
-            launch_gram<T, R, false>(table, ops_here, groups_here, *a.tab, a.partials, a.groups, g0, a.stream);
+            ADASUM_CUDA_CHECK((launch_gram<T, R, false>(a.kind, table, ops_here, groups_here, *a.gram_tab,
+                                                        a.partials, a.groups, g0, a.stream)));
         profile_mark(a.stream, ADASUM_KERNEL_GRAM_PARTIAL, a.level, R, false);
     }
-    launch_weights<R>(a.partials, *a.tab, a.num_tensors, a.operands, a.groups, a.weights, a.stream);
+    int weight_launches = 0;
+    ADASUM_CUDA_CHECK(launch_weights<R>(a.partials, *a.gram_tab, a.num_tensors, a.operands, a.groups, a.gram64,
+                                        a.weights, a.stream, &weight_launches));
     profile_mark(a.stream, ADASUM_KERNEL_TREE_WEIGHTS, a.level, R, false);
     // pass 2
     for (int g0 = 0; g0 < a.groups; g0 += kGroupsPerLaunch) {
@@ -342,10 +489,10 @@ adasum_status_t run_level_typed(const LevelArgs& a)
         for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
             table.ptr[i] = a.operand_ptrs[op0 + (i < ops_here ? i : 0)];
         if (a.vec)
-            launch_wsum<T, R, true>(table, ops_here, groups_here, *a.tab, a.weights, a.groups, g0, a.dst,
+            launch_wsum<T, R, true>(table, ops_here, groups_here, *a.wsum_tab, a.weights, a.groups, g0, a.dst,
                                     a.dst_stride, a.stream);
         else
-            launch_wsum<T, R, false>(table, ops_here, groups_here, *a.tab, a.weights, a.groups, g0, a.dst,
+            launch_wsum<T, R, false>(table, ops_here, groups_here, *a.wsum_tab, a.weights, a.groups, g0, a.dst,
                                      a.dst_stride, a.stream);
         profile_mark(a.stream, ADASUM_KERNEL_WEIGHTED_SUM, a.level, R, false);
     }
@@ -361,6 +508,12 @@ adasum_status_t run_level(int radix, const LevelArgs& a)
     case 4: return run_level_typed<T, 4>(a);
     case 8: return run_level_typed<T, 8>(a);
     case 16: return run_level_typed<T, 16>(a);
+    case 32: return run_level_typed<T, 32>(a);
+    case 64:
+        if constexpr (sizeof(T) == 2)
+            return run_level_typed<T, 64>(a);
+        else
+            return fail(ADASUM_ERR_ARG, "radix 64 needs fp16 / bf16 operands");
     default: return fail(ADASUM_ERR_ARG, "unsupported radix %d", radix);
     }
 }
@@ -373,7 +526,7 @@ int launches_of(const LevelPlan& plan, int n_workers)
     for (int l = 0; l < plan.num_levels; ++l) {
         const int per_launch = kMaxOperandsPerLaunch / plan.level[l].radix;
         const int batches = (plan.level[l].groups + per_launch - 1) / per_launch;
-        n += 2 * batches + 1;
+        n += 2 * batches + (plan.level[l].radix >= 32 ? 2 : 1);
     }
     return n;
 }
@@ -471,8 +624,14 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     std::vector<const void*> operand_ptrs(grads, grads + n_workers);
     for (int l = 0; l < plan.num_levels; ++l) {
         const Level& lv = plan.level[l];
-        const SegmentTable* tab = nullptr;
-        st = get_segment_table(offsets, num_tensors, lv.seg_len, &tab);
+        const bool simple_kernels = (flags & ADASUM_FLAG_SIMPLE_KERNELS) != 0;
+        const GramKind kind = gram_kind(lv.radix, vec, simple_kernels);
+        const SegmentTable* gram_tab = nullptr;
+        const SegmentTable* wsum_tab = nullptr;
+        st = get_segment_table(offsets, num_tensors, gram_segment_length(kind, total), &gram_tab);
+        if (st != ADASUM_OK)
+            return st;
+        st = get_segment_table(offsets, num_tensors, wsum_segment_length(total), &wsum_tab);
         if (st != ADASUM_OK)
             return st;
         const bool last = l + 1 == plan.num_levels;
@@ -480,10 +639,13 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         a.operand_ptrs = operand_ptrs.data();
         a.operands = lv.operands;
         a.groups = lv.groups;
-        a.tab = tab;
+        a.kind = kind;
+        a.gram_tab = gram_tab;
+        a.wsum_tab = wsum_tab;
         a.num_tensors = num_tensors;
         a.partials = reinterpret_cast<float*>(ws + lay.partials);
         a.weights = reinterpret_cast<float*>(ws + lay.weights);
+        a.gram64 = reinterpret_cast<double*>(ws + lay.gram64);
         a.dst = last ? out : reinterpret_cast<float*>(ws + lay.buffer[l & 1]);
         a.dst_stride = last ? 0 : lay.padded_elems;
         a.vec = vec;
@@ -552,18 +714,22 @@ adasum_status_t noalloc_scratch(unsigned char** ptr)
 }
 
 template <typename T>
-void noalloc_launch(bool vec, const OperandTable& ops, const SegmentTable& tab, int32_t num_tensors,
-                    float* partials, float* weights, float* out, cudaStream_t stream)
+cudaError_t noalloc_launch(bool vec, const OperandTable& ops, const SegmentTable& tab, int32_t num_tensors,
+                           float* partials, float* weights, float* out, cudaStream_t stream)
 {
-    if (vec) {
-        launch_gram<T, 2, true>(ops, 2, 1, tab, partials, 1, 0, stream);
-        launch_weights<2>(partials, tab, num_tensors, 2, 1, weights, stream);
+    cudaError_t err = vec ? launch_gram<T, 2, true>(GRAM_SIMPLE, ops, 2, 1, tab, partials, 1, 0, stream)
+                          : launch_gram<T, 2, false>(GRAM_SIMPLE, ops, 2, 1, tab, partials, 1, 0, stream);
+    if (err != cudaSuccess)
+        return err;
+    int weight_launches = 0;
+    err = launch_weights<2>(partials, tab, num_tensors, 2, 1, nullptr, weights, stream, &weight_launches);
+    if (err != cudaSuccess)
+        return err;
+    if (vec)
         launch_wsum<T, 2, true>(ops, 2, 1, tab, weights, 1, 0, out, 0, stream);
-    } else {
-        launch_gram<T, 2, false>(ops, 2, 1, tab, partials, 1, 0, stream);
-        launch_weights<2>(partials, tab, num_tensors, 2, 1, weights, stream);
+    else
         launch_wsum<T, 2, false>(ops, 2, 1, tab, weights, 1, 0, out, 0, stream);
-    }
+    return cudaSuccess;
 }
 
 adasum_status_t pair_noalloc_impl(const void* a, const void* b, const int64_t* offsets, int32_t num_tensors,
@@ -622,11 +788,11 @@ adasum_status_t pair_noalloc_impl(const void* a, const void* b, const int64_t* o
     for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
         ops.ptr[i] = in[i < 2 ? i : 0];
     if (dtype == ADASUM_F32)
-        noalloc_launch<float>(vec, ops, tab, num_tensors, partials, weights, out, stream);
+        ADASUM_CUDA_CHECK(noalloc_launch<float>(vec, ops, tab, num_tensors, partials, weights, out, stream));
     else if (dtype == ADASUM_F16)
-        noalloc_launch<__half>(vec, ops, tab, num_tensors, partials, weights, out, stream);
+        ADASUM_CUDA_CHECK(noalloc_launch<__half>(vec, ops, tab, num_tensors, partials, weights, out, stream));
     else
-        noalloc_launch<__nv_bfloat16>(vec, ops, tab, num_tensors, partials, weights, out, stream);
+        ADASUM_CUDA_CHECK(noalloc_launch<__nv_bfloat16>(vec, ops, tab, num_tensors, partials, weights, out, stream));
     ADASUM_CUDA_CHECK(cudaGetLastError());
     return ADASUM_OK;
 }

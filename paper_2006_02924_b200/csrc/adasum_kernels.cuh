@@ -1,6 +1,6 @@
 // Device kernels of the N-way Adasum combine for sm_100a.
 //
-// One "level" of the reduction handles groups of R adjacent operands (R = 2, 4, 8 or 16).  A group
+// One "level" of the reduction handles groups of R adjacent operands (R = 2 ... 64).  A group
 // is a complete sub-tree of the paper's binary tree (Section 3.4; Algorithm 1 pairs neighbours at
 // distance 1, 2, 4, ...), and every node of that sub-tree is a linear combination of the group's
 // leaves.  So a level is three kernels:
@@ -12,6 +12,11 @@
 //                  order, then run the binary tree on the Gram matrix alone to get the R leaf
 //                  weights (the "Apply Adasum" coefficients, composed down the sub-tree).
 //   weighted_sum   stream the operands a second time; out = sum_i weight_i x_i.
+//
+// The Gram matrix of a group is a dense contraction X X^T (R x P times P x R).  For R <= 8 it is
+// cheap enough for the fp32 pipes (gram_partial_kernel, gram_partial_pipelined_kernel); for
+// R >= 16 it runs on the tensor cores (gram_partial_mma_kernel): fp16 / bf16 products are exact in
+// the fp32 accumulator, fp32 inputs are split into two tf32 terms (three products).
 //
 // The kernels never wait on one another and use no floating-point atomics, so results are
 // deterministic and there is nothing that can spin.
@@ -26,7 +31,7 @@ namespace adasum {
 constexpr int kThreads = 256;               // threads per block of the streaming kernels
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxOperandsPerLaunch = 256;  // operand pointers carried in one kernel argument
-constexpr int kMaxRadix = 16;
+constexpr int kMaxRadix = 64;
 
 // A contiguous run of elements of one tensor inside the fused buffers.
 struct Segment {
@@ -230,6 +235,634 @@ gram_partial_kernel(const __grid_constant__ OperandTable ops, int operands,
     }
 }
 
+// ---- pass 1, pipelined: persistent blocks, operands staged through shared memory ---------------
+//
+// The register-only kernel above cannot overlap its loads with its arithmetic at radix 16 (136
+// accumulators leave room for one column set only).  Here every thread copies its own 16 bytes of
+// each operand row into shared memory with cp.async, STAGES tiles deep, and reads back only what it
+// copied itself: no thread ever waits for another one inside the loop, so nothing can dead-lock.
+// A block walks the segments blockIdx.x, blockIdx.x + gridDim.x, ... and keeps the copy pipeline
+// running across segment boundaries; accumulators are flushed (block reduction, one partial per
+// segment) when a segment ends.  Requires 16-byte aligned operands (the VEC case).
+
+__device__ __forceinline__ void cp_async_16B(void* smem_dst, const void* gmem_src)
+{
+    const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait()
+{
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// Elements decoded per round from one thread's 16 bytes of a row, and how.
+template <typename T, int R>
+struct Rounds;
+template <int R>
+struct Rounds<float, R> {
+    static constexpr int kWords = 4, kElems = 4, kRounds = 1;
+    static __device__ __forceinline__ void decode(const uint32_t (&w)[kWords], float (&x)[kElems])
+    {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            x[j] = __uint_as_float(w[j]);
+    }
+};
+template <int R>
+struct Rounds<__half, R> {
+    static constexpr int kWords = R >= 16 ? 1 : 4, kElems = 2 * kWords, kRounds = 4 / kWords;
+    static __device__ __forceinline__ void decode(const uint32_t (&w)[kWords], float (&x)[kElems])
+    {
+#pragma unroll
+        for (int j = 0; j < kWords; ++j) {
+            float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[j]));
+            x[2 * j] = f.x;
+            x[2 * j + 1] = f.y;
+        }
+    }
+};
+template <int R>
+struct Rounds<__nv_bfloat16, R> {
+    static constexpr int kWords = R >= 16 ? 1 : 4, kElems = 2 * kWords, kRounds = 4 / kWords;
+    static __device__ __forceinline__ void decode(const uint32_t (&w)[kWords], float (&x)[kElems])
+    {
+#pragma unroll
+        for (int j = 0; j < kWords; ++j) {
+            x[2 * j] = __uint_as_float(w[j] << 16);
+            x[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+        }
+    }
+};
+
+template <int WORDS>
+__device__ __forceinline__ void load_shared_words(const unsigned char* p, uint32_t (&w)[WORDS])
+{
+    if (WORDS == 4) {
+        uint4 v = *reinterpret_cast<const uint4*>(p);
+        w[0] = v.x; w[1 % WORDS] = v.y; w[2 % WORDS] = v.z; w[3 % WORDS] = v.w;
+    } else if (WORDS == 2) {
+        uint2 v = *reinterpret_cast<const uint2*>(p);
+        w[0] = v.x; w[1 % WORDS] = v.y;
+    } else {
+        w[0] = *reinterpret_cast<const uint32_t*>(p);
+    }
+}
+
+// Where one thread stands in its block's sequence of tiles.  A tile is kThreads consecutive
+// 16-byte vectors of the aligned body of a segment.
+template <int V>
+struct TileCursor {
+    int seg;              // index into the segment table, >= num_segments when exhausted
+    int64_t v;            // element index of this thread's vector in the current tile
+    int64_t tile_begin;   // element index where the current tile starts
+    int64_t body_end;     // end of the aligned body of the current segment
+
+    __device__ __forceinline__ void enter(const Segment* __restrict__ segments, int num_segments)
+    {
+        // position on the first tile of segment `seg`, skipping segments without an aligned body
+        while (seg < num_segments) {
+            const Segment s = segments[seg];
+            int64_t bb, be;
+            split_segment<V, true>(s.begin, s.begin + s.len, bb, be);
+            if (bb < be) {
+                tile_begin = bb;
+                body_end = be;
+                v = bb + (int64_t)threadIdx.x * V;
+                return;
+            }
+            seg += gridDim.x;
+        }
+    }
+    __device__ __forceinline__ void next_tile(const Segment* __restrict__ segments, int num_segments)
+    {
+        tile_begin += (int64_t)kThreads * V;
+        v += (int64_t)kThreads * V;
+        if (tile_begin >= body_end) {
+            seg += gridDim.x;
+            enter(segments, num_segments);
+        }
+    }
+};
+
+template <int R, int E>
+__device__ __forceinline__ void block_reduce_and_store(float (&acc)[E], float (*warp_sums)[E], float* dst)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int k = 0; k < E; ++k) {
+        float s = acc[k];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1)
+            s += __shfl_xor_sync(0xffffffffu, s, d);
+        if (lane == 0)
+            warp_sums[warp][k] = s;
+    }
+    __syncthreads();
+    for (int k = threadIdx.x; k < E; k += kThreads) {
+        float s = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w)
+            s += warp_sums[w][k];
+        dst[k] = s;
+    }
+    __syncthreads();   // warp_sums is reused by the next segment
+}
+
+template <int R>
+__host__ __device__ constexpr int pipelined_min_blocks() { return R >= 16 ? 1 : (R >= 8 ? 2 : 4); }
+
+// grid = (persistent blocks, groups in this launch); block = kThreads;
+// dynamic shared memory = STAGES * R * kThreads * 16 bytes.
+template <typename T, int R, int STAGES>
+__global__ void __launch_bounds__(kThreads, pipelined_min_blocks<R>())
+gram_partial_pipelined_kernel(const __grid_constant__ OperandTable ops, int operands,
+                              const Segment* __restrict__ segments, int num_segments,
+                              float* __restrict__ partials, int groups_total, int group_base)
+{
+    constexpr int E = gram_entries(R);
+    constexpr int V = Element<T>::kVec;
+    using Rd = Rounds<T, R>;
+    extern __shared__ __align__(16) unsigned char stage_mem[];
+    __shared__ float warp_sums[kWarps][E];
+
+    const int first = blockIdx.y * R;
+    const int members = min(R, operands - first);
+    unsigned char* my_smem = stage_mem + (size_t)threadIdx.x * 16;   // + (stage * R + row) * kThreads * 16
+
+    TileCursor<V> prod, cons;
+    prod.seg = blockIdx.x;
+    prod.enter(segments, num_segments);
+    cons = prod;
+
+    auto issue = [&](int stage) {
+        if (prod.seg < num_segments) {
+            if (prod.v < prod.body_end) {
+#pragma unroll
+                for (int i = 0; i < R; ++i)
+                    if (i < members)
+                        cp_async_16B(my_smem + (size_t)(stage * R + i) * kThreads * 16,
+                                     static_cast<const T*>(ops.ptr[first + i]) + prod.v);
+            }
+            prod.next_tile(segments, num_segments);
+        }
+        cp_async_commit();
+    };
+
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s)
+        issue(s);
+
+    int stage = 0;
+    for (int seg = blockIdx.x; seg < num_segments; seg += gridDim.x) {
+        float acc[E];
+#pragma unroll
+        for (int k = 0; k < E; ++k)
+            acc[k] = 0.0f;
+
+        // tiles of this segment's aligned body
+        while (cons.seg == seg) {
+            int refill = stage + STAGES - 1;
+            if (refill >= STAGES)
+                refill -= STAGES;
+            issue(refill);
+            cp_async_wait<STAGES - 1>();
+            if (cons.v < cons.body_end) {
+                const unsigned char* base = my_smem + (size_t)stage * R * kThreads * 16;
+#pragma unroll
+                for (int round = 0; round < Rd::kRounds; ++round) {
+                    float x[R][Rd::kElems];
+#pragma unroll
+                    for (int i = 0; i < R; ++i) {
+                        if (i < members) {
+                            uint32_t w[Rd::kWords];
+                            load_shared_words<Rd::kWords>(base + (size_t)i * kThreads * 16 + round * Rd::kWords * 4, w);
+                            Rd::decode(w, x[i]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < Rd::kElems; ++j)
+                                x[i][j] = 0.0f;
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < Rd::kElems; ++j) {
+                        float col[R];
+#pragma unroll
+                        for (int i = 0; i < R; ++i)
+                            col[i] = x[i][j];
+                        gram_accumulate<R>(col, acc);
+                    }
+                }
+            }
+            cons.next_tile(segments, num_segments);
+            if (++stage == STAGES)
+                stage = 0;
+        }
+
+        // scalar head and tail of the segment, straight from global memory
+        const Segment s = segments[seg];
+        const int64_t begin = s.begin, end = s.begin + s.len;
+        int64_t body_begin, body_end;
+        split_segment<V, true>(begin, end, body_begin, body_end);
+        for (int pass = 0; pass < 2; ++pass) {
+            const int64_t lo = pass == 0 ? begin : body_end;
+            const int64_t hi = pass == 0 ? body_begin : end;
+            for (int64_t e = lo + threadIdx.x; e < hi; e += kThreads) {
+                float col[R];
+#pragma unroll
+                for (int i = 0; i < R; ++i)
+                    col[i] = i < members ? Element<T>::one(static_cast<const T*>(ops.ptr[first + i]) + e) : 0.0f;
+                gram_accumulate<R>(col, acc);
+            }
+        }
+        block_reduce_and_store<R, E>(acc, warp_sums,
+                                     partials + ((int64_t)seg * groups_total + group_base + blockIdx.y) * E);
+    }
+    cp_async_wait<0>();
+}
+
+// ---- pass 1 on the tensor cores ----------------------------------------------------------------
+//
+// G = X X^T with X the R x (segment length) matrix of a group's rows.  A thread block streams the
+// segment in tiles of 32 KB (R rows of 32 KB / R contiguous bytes, fully coalesced 512-byte warp
+// accesses, cp.async, several tiles in flight).  Warp w multiplies chunks w * DEPTH ... of each
+// tile (a chunk is 64 bytes of every row).  Lane (g, t) = (lane / 4, lane % 4) reads, for every
+// block of 8 rows, the 16 bytes of row 8 rb + g at chunk offset 16 t: those four words are exactly
+// the lane's share of the A fragment (rows g and g + 8 of a 16-row block) and of the B fragment
+// (column g of an 8-column block) of mma.sync m16n8k8 (tf32) / m16n8k16 (fp16, bf16), because both
+// operands of X X^T are the same rows and the order of the K index inside a chunk is free as long
+// as A and B agree.
+//
+// fp16 / bf16 products are exact in the fp32 accumulator.  fp32 inputs are split x = hi + lo with
+// hi the nearest tf32: G = H + C + C^T with H = Xhi Xhi^T (upper blocks only) and C = Xhi Xlo^T
+// (all blocks; lo lo^T, about 2^-22 relative, is dropped).  The tensor core's own accumulation is
+// not correctly rounded, so for fp32 inputs its chains are kept to one tile and the tile results
+// are added with ordinary rounded adds.
+
+template <int R>
+__host__ __device__ constexpr int mma_upper_blocks()     // 16 x 8 blocks that touch the upper triangle
+{
+    int n = 0;
+    for (int mb = 0; mb < R / 16; ++mb)
+        n += R / 8 - 2 * mb;
+    return n;
+}
+template <int R>
+__host__ __device__ constexpr int mma_all_blocks() { return (R / 16) * (R / 8); }
+
+// Index of block (mb, nb), nb >= 2 mb, in the upper-block numbering.
+template <int R>
+__host__ __device__ constexpr int mma_upper_index(int mb, int nb)
+{
+    int n = 0;
+    for (int m = 0; m < mb; ++m)
+        n += R / 8 - 2 * m;
+    return n + nb - 2 * mb;
+}
+
+// Where element (r, c) of a 16 x 8 accumulator block lives: register (0..3) * 32 + lane.
+__host__ __device__ constexpr int mma_fragment_slot(int r, int c)
+{
+    return (((r >= 8 ? 2 : 0) + (c & 1)) * 32) + (r % 8) * 4 + c / 2;
+}
+
+#define ADASUM_MMA_ASM(shape, types)                                                                   \
+    asm volatile("mma.sync.aligned." shape ".row.col.f32." types ".f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, " \
+                 "{%8,%9}, {%0,%1,%2,%3};"                                                             \
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])                                      \
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1))
+
+template <typename T>
+__device__ __forceinline__ void mma_step(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1);
+template <>
+__device__ __forceinline__ void mma_step<float>(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                                uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    ADASUM_MMA_ASM("m16n8k8", "tf32.tf32");
+}
+template <>
+__device__ __forceinline__ void mma_step<__half>(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                                 uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    ADASUM_MMA_ASM("m16n8k16", "f16.f16");
+}
+template <>
+__device__ __forceinline__ void mma_step<__nv_bfloat16>(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                                        uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    ADASUM_MMA_ASM("m16n8k16", "bf16.bf16");
+}
+#undef ADASUM_MMA_ASM
+
+// The 16 bytes of `row` that start at element e0, as four words, with every element outside
+// [begin, end) replaced by zero.  Used for the ragged ends of a segment and for unaligned buffers.
+template <typename T>
+__device__ __forceinline__ uint4 load_masked_words(const T* row, int64_t e0, int64_t begin, int64_t end);
+template <>
+__device__ __forceinline__ uint4 load_masked_words<float>(const float* row, int64_t e0, int64_t begin, int64_t end)
+{
+    uint32_t w[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int64_t e = e0 + j;
+        w[j] = (e >= begin && e < end) ? __float_as_uint(__ldg(row + e)) : 0u;
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+template <typename T16>
+__device__ __forceinline__ uint4 load_masked_words16(const T16* row, int64_t e0, int64_t begin, int64_t end)
+{
+    const unsigned short* bits = reinterpret_cast<const unsigned short*>(row);
+    uint32_t w[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int64_t e = e0 + 2 * j;
+        const uint32_t lo = (e >= begin && e < end) ? (uint32_t)__ldg(bits + e) : 0u;
+        const uint32_t hi = (e + 1 >= begin && e + 1 < end) ? (uint32_t)__ldg(bits + e + 1) : 0u;
+        w[j] = lo | (hi << 16);
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+template <>
+__device__ __forceinline__ uint4 load_masked_words<__half>(const __half* row, int64_t e0, int64_t begin, int64_t end)
+{
+    return load_masked_words16(row, e0, begin, end);
+}
+template <>
+__device__ __forceinline__ uint4 load_masked_words<__nv_bfloat16>(const __nv_bfloat16* row, int64_t e0,
+                                                                   int64_t begin, int64_t end)
+{
+    return load_masked_words16(row, e0, begin, end);
+}
+
+__device__ __forceinline__ void cp_async_16B_shared(uint32_t smem_addr, const void* gmem_src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void store_shared_16B(uint32_t smem_addr, uint4 v)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(smem_addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+__device__ __forceinline__ uint4 load_shared_16B(uint32_t smem_addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "r"(smem_addr)
+                 : "memory");
+    return v;
+}
+
+template <typename T, int R>
+__host__ __device__ constexpr int mma_depth() { return 64 / R > 0 ? 64 / R : 1; }   // chunks per warp per tile
+template <typename T, int R>
+__host__ __device__ constexpr int mma_min_blocks()
+{
+    return (R >= 64 || (R >= 32 && sizeof(T) == 4)) ? 1 : 2;
+}
+// Tiles kept in shared memory: 3 where two blocks share an SM, 6 for the register-heavy kernels
+// that run one block per SM.
+template <typename T, int R>
+__host__ __device__ constexpr int mma_stages() { return mma_min_blocks<T, R>() == 1 ? 6 : 3; }
+constexpr int kMmaTileBytes = 32 * 1024;
+template <typename T, int R>
+__host__ __device__ constexpr size_t mma_smem_bytes() { return (size_t)mma_stages<T, R>() * kMmaTileBytes; }
+
+// grid = (segments, groups in this launch); block = kThreads; dynamic shared memory =
+// mma_smem_bytes<T, R>().
+//
+// Shared-memory layout of a tile: row-major, 64-byte chunk index XOR (row & 1), so that the
+// fragment reads of a quarter warp (two rows, four 16-byte pieces each) fall into distinct banks.
+// The pipeline is the usual multi-stage one: wait for the oldest copy group, one __syncthreads
+// per tile, refill the slot that was consumed in the previous iteration.
+template <typename T, int R, bool VEC>
+__global__ void __launch_bounds__(kThreads, mma_min_blocks<T, R>())
+gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
+                        const Segment* __restrict__ segments, float* __restrict__ partials,
+                        int groups_total, int group_base)
+{
+    constexpr int E = gram_entries(R);
+    constexpr int V = Element<T>::kVec;          // elements per 16-byte vector
+    constexpr int RB = R / 8;                    // blocks of 8 rows
+    constexpr int UBLK = mma_upper_blocks<R>();
+    constexpr bool SPLIT = sizeof(T) == 4;
+    constexpr int CBLK = SPLIT ? mma_all_blocks<R>() : 0;
+    constexpr int DEPTH = mma_depth<T, R>();
+    constexpr int STAGES = mma_stages<T, R>();
+    constexpr int ROW_BYTES = kMmaTileBytes / R;
+    constexpr int PIECES_PER_ROW = ROW_BYTES / 16;
+    constexpr int TILE_ELEMS = PIECES_PER_ROW * V;               // elements of one row in a tile
+    constexpr int PIECES = kMmaTileBytes / 16 / kThreads;        // 16-byte pieces a thread copies per tile
+    constexpr int ROWS_PER_PASS = kThreads / PIECES_PER_ROW;     // piece i of a thread is in row row0 + i * this
+    static_assert(DEPTH * kWarps * 64 == ROW_BYTES, "a tile row is split evenly among the warps");
+    static_assert(PIECES_PER_ROW % 32 == 0 && kThreads % PIECES_PER_ROW == 0, "a warp copies within one row");
+    static_assert(ROWS_PER_PASS % 2 == 0, "all pieces of a thread have the same row parity");
+    extern __shared__ __align__(128) unsigned char stage_mem[];
+
+    const Segment seg = segments[blockIdx.x];
+    const int first = blockIdx.y * R;
+    const int members = min(R, operands - first);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, t = lane & 3;
+
+    const int64_t begin = seg.begin, end = seg.begin + seg.len;
+    const int64_t k0 = VEC ? begin / V * V : begin;
+    const int ntiles = (int)((end - k0 + TILE_ELEMS - 1) / TILE_ELEMS);
+
+    // ---- copy side: piece i of this thread is (row0 + i * ROWS_PER_PASS, col0) of the tile
+    const uint32_t smem_base = static_cast<uint32_t>(__cvta_generic_to_shared(stage_mem));
+    const int row0 = threadIdx.x / PIECES_PER_ROW, col0 = threadIdx.x % PIECES_PER_ROW;
+    const uint32_t copy_off = row0 * ROW_BYTES + (((col0 >> 2) ^ (row0 & 1)) << 6) + ((col0 & 3) << 4);
+    const T* copy_src[PIECES];     // row pointer + this thread's column; rows beyond the members alias row 0
+#pragma unroll
+    for (int i = 0; i < PIECES; ++i) {
+        const int row = row0 + i * ROWS_PER_PASS;
+        copy_src[i] = static_cast<const T*>(ops.ptr[first + (row < members ? row : 0)]) + col0 * V;
+    }
+    const bool full_group = members == R;
+
+    auto issue = [&](int tile, int stage) {
+        if (tile < ntiles) {
+            const uint32_t dst = smem_base + stage * kMmaTileBytes + copy_off;
+            const int64_t tile_elem0 = k0 + (int64_t)tile * TILE_ELEMS;
+            if (VEC && full_group && tile_elem0 >= begin && tile_elem0 + TILE_ELEMS <= end) {
+#pragma unroll
+                for (int i = 0; i < PIECES; ++i)
+                    cp_async_16B_shared(dst + i * ROWS_PER_PASS * ROW_BYTES, copy_src[i] + tile_elem0);
+            } else {
+                // ragged tile, partial group or unaligned buffers: test every piece
+                const int64_t e0 = tile_elem0 + (int64_t)col0 * V;
+                const bool whole = VEC && e0 >= begin && e0 + V <= end;
+#pragma unroll
+                for (int i = 0; i < PIECES; ++i) {
+                    const uint32_t slot = dst + i * ROWS_PER_PASS * ROW_BYTES;
+                    if (row0 + i * ROWS_PER_PASS >= members)
+                        store_shared_16B(slot, make_uint4(0u, 0u, 0u, 0u));
+                    else if (whole)
+                        cp_async_16B_shared(slot, copy_src[i] + tile_elem0);
+                    else
+                        store_shared_16B(slot, load_masked_words<T>(copy_src[i] - col0 * V, e0, begin, end));
+                }
+            }
+        }
+        cp_async_commit();
+    };
+
+    // ---- multiply side
+    const uint32_t frag_off = g * ROW_BYTES + (t << 4);
+    uint32_t chunk_off[DEPTH];
+#pragma unroll
+    for (int d = 0; d < DEPTH; ++d)
+        chunk_off[d] = ((warp * DEPTH + d) ^ (g & 1)) << 6;
+
+    float acc[UBLK][4];                            // 16-bit inputs: the accumulators; fp32: rounded sums of H
+    float acc_c[SPLIT ? CBLK : 1][4];              // fp32: rounded sums of C
+#pragma unroll
+    for (int b = 0; b < UBLK; ++b)
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+            acc[b][r] = 0.0f;
+#pragma unroll
+    for (int b = 0; b < (SPLIT ? CBLK : 1); ++b)
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+            acc_c[b][r] = 0.0f;
+
+#pragma unroll
+    for (int st = 0; st < STAGES - 1; ++st)
+        issue(st, st);
+
+    int stage = 0;
+    for (int tile = 0; tile < ntiles; ++tile) {
+        cp_async_wait<STAGES - 2>();     // this thread's copies for `tile` have landed
+        __syncthreads();                 // ... and everybody's; the previous tile's slot is free
+        int refill = stage + STAGES - 1;
+        if (refill >= STAGES)
+            refill -= STAGES;
+        issue(tile + STAGES - 1, refill);
+
+        const uint32_t src_stage = smem_base + stage * kMmaTileBytes + frag_off;
+        if (++stage == STAGES)
+            stage = 0;
+
+        if constexpr (!SPLIT) {
+#pragma unroll
+            for (int d = 0; d < DEPTH; ++d) {
+                uint32_t w[RB][4];
+#pragma unroll
+                for (int rb = 0; rb < RB; ++rb) {
+                    const uint4 v = load_shared_16B(src_stage + chunk_off[d] + rb * 8 * ROW_BYTES);
+                    w[rb][0] = v.x; w[rb][1] = v.y; w[rb][2] = v.z; w[rb][3] = v.w;
+                }
+#pragma unroll
+                for (int step = 0; step < 2; ++step) {
+#pragma unroll
+                    for (int mb = 0; mb < R / 16; ++mb)
+#pragma unroll
+                        for (int nb = 2 * mb; nb < RB; ++nb)
+                            mma_step<T>(acc[mma_upper_index<R>(mb, nb)], w[2 * mb][2 * step], w[2 * mb + 1][2 * step],
+                                        w[2 * mb][2 * step + 1], w[2 * mb + 1][2 * step + 1], w[nb][2 * step],
+                                        w[nb][2 * step + 1]);
+                }
+            }
+        } else {
+            float tile_h[UBLK][4], tile_c[SPLIT ? CBLK : 1][4];
+#pragma unroll
+            for (int b = 0; b < UBLK; ++b)
+#pragma unroll
+                for (int r = 0; r < 4; ++r)
+                    tile_h[b][r] = 0.0f;
+#pragma unroll
+            for (int b = 0; b < CBLK; ++b)
+#pragma unroll
+                for (int r = 0; r < 4; ++r)
+                    tile_c[b][r] = 0.0f;
+#pragma unroll
+            for (int d = 0; d < DEPTH; ++d) {
+                uint32_t hi[RB][4], lo[RB][4];
+#pragma unroll
+                for (int rb = 0; rb < RB; ++rb) {
+                    const uint4 v = load_shared_16B(src_stage + chunk_off[d] + rb * 8 * ROW_BYTES);
+                    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        // nearest tf32 by integer arithmetic (the conversion instruction runs on
+                        // the slow special-function pipe): add half a tf32 ulp, drop 13 bits
+                        hi[rb][j] = (w[j] + 0x1000u) & 0xffffe000u;
+                        lo[rb][j] = __float_as_uint(__uint_as_float(w[j]) - __uint_as_float(hi[rb][j]));
+                    }
+                }
+#pragma unroll
+                for (int step = 0; step < 2; ++step) {
+#pragma unroll
+                    for (int mb = 0; mb < R / 16; ++mb) {
+#pragma unroll
+                        for (int nb = 0; nb < RB; ++nb) {
+                            if (nb >= 2 * mb)
+                                mma_step<T>(tile_h[mma_upper_index<R>(mb, nb)], hi[2 * mb][2 * step],
+                                            hi[2 * mb + 1][2 * step], hi[2 * mb][2 * step + 1],
+                                            hi[2 * mb + 1][2 * step + 1], hi[nb][2 * step], hi[nb][2 * step + 1]);
+                            mma_step<T>(tile_c[mb * RB + nb], hi[2 * mb][2 * step], hi[2 * mb + 1][2 * step],
+                                        hi[2 * mb][2 * step + 1], hi[2 * mb + 1][2 * step + 1], lo[nb][2 * step],
+                                        lo[nb][2 * step + 1]);
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int b = 0; b < UBLK; ++b)
+#pragma unroll
+                for (int r = 0; r < 4; ++r)
+                    acc[b][r] += tile_h[b][r];
+#pragma unroll
+            for (int b = 0; b < CBLK; ++b)
+#pragma unroll
+                for (int r = 0; r < 4; ++r)
+                    acc_c[b][r] += tile_c[b][r];
+        }
+    }
+    cp_async_wait<0>();
+
+    // block reduction: the warps add their fragments into shared memory one after the other
+    __shared__ float total[(UBLK + CBLK) * 128];
+#pragma unroll 1
+    for (int w = 0; w < kWarps; ++w) {
+        if (warp == w) {
+#pragma unroll
+            for (int b = 0; b < UBLK; ++b)
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const int slot = (b * 4 + r) * 32 + lane;
+                    total[slot] = w == 0 ? acc[b][r] : total[slot] + acc[b][r];
+                }
+#pragma unroll
+            for (int b = 0; b < CBLK; ++b)
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const int slot = ((UBLK + b) * 4 + r) * 32 + lane;
+                    total[slot] = w == 0 ? acc_c[b][r] : total[slot] + acc_c[b][r];
+                }
+        }
+        __syncthreads();
+    }
+    // entries (i <= j) of the packed upper triangle from the accumulator fragments
+    float* dst = partials + ((int64_t)blockIdx.x * groups_total + group_base + blockIdx.y) * E;
+    for (int idx = threadIdx.x; idx < R * R; idx += kThreads) {
+        const int i = idx / R, j = idx % R;
+        if (i > j)
+            continue;
+        float v = total[mma_upper_index<R>(i / 16, j / 8) * 128 + mma_fragment_slot(i % 16, j % 8)];
+        if (SPLIT) {
+            v += total[(UBLK + (i / 16) * RB + j / 8) * 128 + mma_fragment_slot(i % 16, j % 8)];   // C_ij
+            v += total[(UBLK + (j / 16) * RB + i / 8) * 128 + mma_fragment_slot(j % 16, i % 8)];   // C_ji
+        }
+        dst[gram_index(R, i, j)] = v;
+    }
+}
+
 // ---- coefficients: the binary tree evaluated on a Gram matrix ---------------------------------
 
 // Algorithm 1, "Apply Adasum": x' = a (1 - v1 / 2 v2) + b (1 - v1 / 2 v3) with
@@ -241,107 +874,205 @@ __device__ __forceinline__ void pair_coefficients(double dot, double norm_a, dou
     coef_b = norm_b == 0.0 ? 1.0 : 1.0 - dot / (2.0 * norm_b);
 }
 
-// Leaf weights of the sub-tree over `members` leaves whose Gram matrix is `gram` (packed upper
-// triangle, row length R).  Bottom-up: blocks of width 1, 2, 4, ...; the block [L, L+w) is
-// paired with [L+w, L+2w); a block without a right sibling is carried unchanged.  The squared
-// norm of a parent follows from its children: |ca a + cb b|^2 = ca^2 |a|^2 + cb^2 |b|^2 + 2 ca cb a.b.
+// The binary tree evaluated on a Gram matrix held in shared memory; called by every thread of a
+// block of at least R threads.  Leaf weights start at 1; bottom-up over block widths 1, 2, 4, ...:
+// the block [L, L+w) is paired with [L+w, L+2w) (a block without a right sibling is carried
+// unchanged); with d = sum_{i in left, k in right} w_i w_k G_ik and the two blocks' squared norms
+// the pair coefficients follow, every leaf weight of the left (right) block is multiplied by ca
+// (cb), and the parent's squared norm is ca^2 |a|^2 + cb^2 |b|^2 + 2 ca cb d.
 template <int R>
-__device__ void tree_weights_from_gram(const double* gram, int members, double* weight,
-                                       double* root_norm)
+__device__ void tree_weights_from_gram(const double* gram, int members, float* __restrict__ dst)
 {
-    double norm[R];
-    for (int i = 0; i < members; ++i) {
-        weight[i] = 1.0;
-        norm[i] = gram[gram_index(R, i, i)];
+    __shared__ double weight[R], norm[R], row_dot[R], coef_a[R / 2], coef_b[R / 2];
+    const int tid = threadIdx.x;
+    if (tid < R) {
+        weight[tid] = 1.0;
+        norm[tid] = tid < members ? gram[gram_index(R, tid, tid)] : 0.0;
     }
+    __syncthreads();
     for (int w = 1; w < members; w *= 2) {
-        for (int left = 0; left + w < members; left += 2 * w) {
+        // leaf i of a left block: weight_i * sum over the sibling block of weight_k G_ik
+        if (tid < members) {
+            const int left = tid / (2 * w) * (2 * w);
             const int mid = left + w;
-            const int right_end = min(left + 2 * w, members);
-            double dot = 0.0;
-            for (int i = left; i < mid; ++i) {
-                double row = 0.0;
+            double acc = 0.0;
+            if (tid < mid && mid < members) {
+                const int right_end = min(left + 2 * w, members);
                 for (int k = mid; k < right_end; ++k)
-                    row += weight[k] * gram[gram_index(R, i, k)];
-                dot += weight[i] * row;
+                    acc += weight[k] * gram[gram_index(R, tid, k)];
+                acc *= weight[tid];
             }
-            double ca, cb;
-            pair_coefficients(dot, norm[left], norm[mid], ca, cb);
-            for (int i = left; i < mid; ++i)
-                weight[i] *= ca;
-            for (int k = mid; k < right_end; ++k)
-                weight[k] *= cb;
-            norm[left] = ca * ca * norm[left] + cb * cb * norm[mid] + 2.0 * ca * cb * dot;
+            row_dot[tid] = acc;
         }
+        __syncthreads();
+        // one thread per pair of sibling blocks
+        const int pairs = (members + 2 * w - 1) / (2 * w);
+        if (tid < pairs) {
+            const int left = tid * 2 * w, mid = left + w;
+            double ca = 1.0, cb = 1.0;
+            if (mid < members) {
+                double dot = 0.0;
+                for (int i = left; i < mid; ++i)
+                    dot += row_dot[i];
+                pair_coefficients(dot, norm[left], norm[mid], ca, cb);
+                norm[left] = ca * ca * norm[left] + cb * cb * norm[mid] + 2.0 * ca * cb * dot;
+            }
+            coef_a[tid] = ca;
+            coef_b[tid] = cb;
+        }
+        __syncthreads();
+        if (tid < members) {
+            const int pair = tid / (2 * w);
+            const int mid = pair * 2 * w + w;
+            if (mid < members)
+                weight[tid] *= tid < mid ? coef_a[pair] : coef_b[pair];
+        }
+        __syncthreads();
     }
-    *root_norm = norm[0];
+    if (tid < R)
+        dst[tid] = tid < members ? (float)weight[tid] : 0.0f;
 }
 
-// grid = (tensors, groups); block = kThreads.
-// Sums the tensor's per-segment partial matrices in fp64 (fixed order), then thread 0 runs the
-// tree.  weights[(tensor * groups + group) * R + i] = weight of leaf i (fp32).
+constexpr int kTreeThreads = 1024;
+// Entries of the packed Gram matrix handled by one block of gram_finish_kernel, and the number of
+// slices its segments are split into (entries * slices <= kTreeThreads).
+__host__ __device__ constexpr int tree_entries_per_block(int radix)
+{
+    return gram_entries(radix) < 256 ? gram_entries(radix) : 256;
+}
+__host__ __device__ constexpr int tree_entry_blocks(int radix)
+{
+    return (gram_entries(radix) + tree_entries_per_block(radix) - 1) / tree_entries_per_block(radix);
+}
+__host__ __device__ constexpr int tree_slices(int radix)
+{
+    return kTreeThreads / tree_entries_per_block(radix) < 64 ? kTreeThreads / tree_entries_per_block(radix) : 64;
+}
+
+// grid = (tensors, groups, tree_entry_blocks(R)); block = kTreeThreads.
+// Adds the tensor's per-segment partial matrices in fp64: slice q takes segments q, q + Q, ... in
+// order, then the slices are added in order (fixed order: deterministic).  When the whole matrix
+// fits one block (R <= 16) the same block goes on to run the tree and writes
+// weights[(tensor * groups + group) * R + i]; otherwise it stores its entries to gram64 and
+// tree_weights_kernel finishes.
 template <int R>
-__global__ void __launch_bounds__(kThreads)
-tree_weights_kernel(const float* __restrict__ partials, const int32_t* __restrict__ seg_first,
-                    int operands, float* __restrict__ weights)
+__global__ void __launch_bounds__(kTreeThreads)
+gram_finish_kernel(const float* __restrict__ partials, const int32_t* __restrict__ seg_first, int operands,
+                   double* __restrict__ gram64, float* __restrict__ weights)
 {
     constexpr int E = gram_entries(R);
-    constexpr int Q = kThreads / E > 0 ? kThreads / E : 1;   // segment slices summed in parallel
-    const int tensor = blockIdx.x, group = blockIdx.y, groups = gridDim.y;
-    const int members = min(R, operands - group * R);
-    const int s0 = seg_first[tensor], s1 = seg_first[tensor + 1];
+    constexpr int EPB = tree_entries_per_block(R);
+    constexpr int Q = tree_slices(R);
+    constexpr bool SINGLE = tree_entry_blocks(R) == 1;
+    __shared__ double slice_sum[Q][EPB];
+    __shared__ double gram[SINGLE ? E : 1];
 
-    __shared__ double slice_sum[Q][E];
+    const int tensor = blockIdx.x, group = blockIdx.y, groups = gridDim.y;
+    const int s0 = seg_first[tensor], s1 = seg_first[tensor + 1];
+    const int q = threadIdx.x / EPB, kk = threadIdx.x - q * EPB;
+    const int k = blockIdx.z * EPB + kk;
+    if (q < Q) {
+        double s = 0.0;
+        if (k < E) {
+            const float* src = partials + (int64_t)group * E + k;
+            const int64_t stride = (int64_t)groups * E;
+#pragma unroll 4
+            for (int seg = s0 + q; seg < s1; seg += Q)
+                s += (double)__ldg(src + seg * stride);
+        }
+        slice_sum[q][kk] = s;
+    }
+    __syncthreads();
+    if (q == 0 && k < E) {
+        double s = slice_sum[0][kk];
+        for (int qq = 1; qq < Q; ++qq)
+            s += slice_sum[qq][kk];
+        if (SINGLE)
+            gram[kk] = s;
+        else
+            gram64[((int64_t)tensor * groups + group) * E + k] = s;
+    }
+    if (SINGLE) {
+        __syncthreads();
+        tree_weights_from_gram<R>(gram, min(R, operands - group * R),
+                                  weights + ((int64_t)tensor * groups + group) * R);
+    }
+}
+
+// grid = (tensors, groups); block = kThreads.  Radix >= 32: the Gram matrix was finished by
+// several blocks of gram_finish_kernel; load it and run the tree.
+template <int R>
+__global__ void __launch_bounds__(kThreads)
+tree_weights_kernel(const double* __restrict__ gram64, int operands, float* __restrict__ weights)
+{
+    constexpr int E = gram_entries(R);
     __shared__ double gram[E];
-    for (int idx = threadIdx.x; idx < Q * E; idx += kThreads) {
-        const int q = idx / E, k = idx - q * E;
-        double s = 0.0;
-        for (int seg = s0 + q; seg < s1; seg += Q)
-            s += (double)partials[((int64_t)seg * groups + group) * E + k];
-        slice_sum[q][k] = s;
-    }
+    const int tensor = blockIdx.x, group = blockIdx.y, groups = gridDim.y;
+    const double* src = gram64 + ((int64_t)tensor * groups + group) * E;
+    for (int k = threadIdx.x; k < E; k += kThreads)
+        gram[k] = src[k];
     __syncthreads();
-    for (int k = threadIdx.x; k < E; k += kThreads) {
-        double s = 0.0;
-        for (int q = 0; q < Q; ++q)
-            s += slice_sum[q][k];
-        gram[k] = s;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        double weight[R], root_norm;
-        tree_weights_from_gram<R>(gram, members, weight, &root_norm);
-        float* dst = weights + ((int64_t)tensor * groups + group) * R;
-        for (int i = 0; i < R; ++i)
-            dst[i] = i < members ? (float)weight[i] : 0.0f;
-    }
+    tree_weights_from_gram<R>(gram, min(R, operands - group * R), weights + ((int64_t)tensor * groups + group) * R);
 }
 
 // ---- pass 2: weighted sum ---------------------------------------------------------------------
 
+template <typename T>
+__device__ __forceinline__ void decode_vector(const uint4& v, float (&x)[Element<T>::kVec]);
+template <>
+__device__ __forceinline__ void decode_vector<float>(const uint4& v, float (&x)[4])
+{
+    x[0] = __uint_as_float(v.x);
+    x[1] = __uint_as_float(v.y);
+    x[2] = __uint_as_float(v.z);
+    x[3] = __uint_as_float(v.w);
+}
+template <>
+__device__ __forceinline__ void decode_vector<__half>(const uint4& v, float (&x)[8])
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+        x[2 * i] = f.x;
+        x[2 * i + 1] = f.y;
+    }
+}
+template <>
+__device__ __forceinline__ void decode_vector<__nv_bfloat16>(const uint4& v, float (&x)[8])
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        x[2 * i] = __uint_as_float(w[i] << 16);
+        x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+}
+
 // grid = (segments, groups in this launch); block = kThreads.
 // dst_base + (group_base + blockIdx.y) * dst_stride is the group's output buffer (fp32).
+// Rows are read eight at a time so that the loads of one batch are in flight together while the
+// register count stays low enough for three blocks per SM.
 template <typename T, int R, bool VEC>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 3)
 weighted_sum_kernel(const __grid_constant__ OperandTable ops, int operands,
                     const Segment* __restrict__ segments, const float* __restrict__ weights,
                     int groups_total, int group_base, float* __restrict__ dst_base,
                     int64_t dst_stride)
 {
     constexpr int V = Element<T>::kVec;
+    constexpr int BATCH = R < 8 ? R : 8;
     const Segment seg = segments[blockIdx.x];
     const int first = blockIdx.y * R;
     const int members = min(R, operands - first);
     const int group = group_base + blockIdx.y;
 
-    const T* src[R];
-    float w[R];
-    const float* wsrc = weights + ((int64_t)seg.tensor * groups_total + group) * R;
-#pragma unroll
-    for (int i = 0; i < R; ++i) {
-        src[i] = static_cast<const T*>(ops.ptr[first + (i < members ? i : 0)]);
-        w[i] = i < members ? __ldg(wsrc + i) : 0.0f;
-    }
+    __shared__ float w[R];
+    if (threadIdx.x < R)
+        w[threadIdx.x] = threadIdx.x < members
+                             ? __ldg(weights + ((int64_t)seg.tensor * groups_total + group) * R + threadIdx.x)
+                             : 0.0f;
+    __syncthreads();
     float* dst = dst_base + (int64_t)group * dst_stride;
 
     const int64_t begin = seg.begin, end = seg.begin + seg.len;
@@ -349,21 +1080,29 @@ weighted_sum_kernel(const __grid_constant__ OperandTable ops, int operands,
     split_segment<V, VEC>(begin, end, body_begin, body_end);
 
     for (int64_t v = body_begin + (int64_t)threadIdx.x * V; v < body_end; v += (int64_t)kThreads * V) {
-        float x[R][V];
-#pragma unroll
-        for (int i = 0; i < R; ++i)
-            if (i < members)
-                Element<T>::vec(src[i] + v, x[i]);
         float y[V];
 #pragma unroll
         for (int j = 0; j < V; ++j)
             y[j] = 0.0f;
+        // Two batches may be unrolled together; beyond that the loop stays rolled so that the
+        // compiler cannot hoist every batch's loads and spill.
+#pragma unroll(R / BATCH <= 2 ? 2 : 1)
+        for (int b = 0; b < R; b += BATCH) {
+            uint4 raw[BATCH];
 #pragma unroll
-        for (int i = 0; i < R; ++i) {
-            if (i < members) {
+            for (int i = 0; i < BATCH; ++i)
+                if (b + i < members)
+                    raw[i] = load_streaming_16B(static_cast<const T*>(ops.ptr[first + b + i]) + v);
 #pragma unroll
-                for (int j = 0; j < V; ++j)
-                    y[j] = fmaf(w[i], x[i][j], y[j]);
+            for (int i = 0; i < BATCH; ++i) {
+                if (b + i < members) {
+                    float x[V];
+                    decode_vector<T>(raw[i], x);
+                    const float wi = w[b + i];
+#pragma unroll
+                    for (int j = 0; j < V; ++j)
+                        y[j] = fmaf(wi, x[j], y[j]);
+                }
             }
         }
 #pragma unroll
@@ -375,10 +1114,8 @@ weighted_sum_kernel(const __grid_constant__ OperandTable ops, int operands,
         const int64_t hi = pass == 0 ? body_begin : end;
         for (int64_t e = lo + threadIdx.x; e < hi; e += kThreads) {
             float y = 0.0f;
-#pragma unroll
-            for (int i = 0; i < R; ++i)
-                if (i < members)
-                    y = fmaf(w[i], Element<T>::one(src[i] + e), y);
+            for (int i = 0; i < members; ++i)
+                y = fmaf(w[i], Element<T>::one(static_cast<const T*>(ops.ptr[first + i]) + e), y);
             dst[e] = y;
         }
     }

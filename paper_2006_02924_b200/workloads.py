@@ -175,12 +175,14 @@ def generate(spec: WorkloadSpec | str, device="cpu", tensor_sizes=None, n_worker
     return Workload(spec, grads, offsets, rho, sigma, zeroed)
 
 
-def reduced_sizes(sizes, divisor: int, keep_ragged: bool = True) -> list[int]:
+def reduced_sizes(sizes, divisor: int, keep_ragged: bool = True, smallest: int = 16) -> list[int]:
     """Shrink a tensor list for quick tests while keeping its shape mix; optionally make some
-    sizes odd so that tensor starts lose their vector alignment."""
+    sizes odd so that tensor starts lose their vector alignment.  Tensors are not shrunk below
+    `smallest` elements: a one-element "tensor" of many weakly correlated workers is a sum of
+    scalars of random sign, which no floating-point evaluation of the method resolves."""
     out = []
     for i, s in enumerate(sizes):
-        r = max(1, s // divisor)
+        r = max(min(smallest, s), s // divisor)
         if keep_ragged and i % 3 == 1:
             r += 1 + (i % 5)
         out.append(r)

@@ -131,16 +131,45 @@ def test_awkward_shapes(lib, dtype, n):
     _run_and_check(lib, grads, offsets, dtype)
 
 
-@pytest.mark.parametrize("first,later", [(2, 2), (4, 4), (8, 8), (16, 16), (4, 2), (2, 16), (16, 2)])
-@pytest.mark.parametrize("dtype", ["f32", "f16"])
-def test_every_radix_gives_the_same_tree(lib, dtype, first, later):
+SIMPLE = 1 << 16    # ADASUM_FLAG_SIMPLE_KERNELS
+
+
+@pytest.mark.parametrize("first,later,extra", [
+    (2, 2, 0), (4, 4, 0), (8, 8, 0), (16, 16, 0), (4, 2, 0), (2, 16, 0), (16, 2, 0), (32, 32, 0), (32, 4, 0),
+    (2, 32, 0), (2, 2, SIMPLE), (8, 4, SIMPLE), (16, 16, SIMPLE)])
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+def test_every_radix_gives_the_same_tree(lib, dtype, first, later, extra):
     offsets = workloads.offsets_from_sizes([50_000, 17, 3, 70_001, 64])
-    results = []
-    for n in (13, 64):
+    for n in (13, 64, 100):
         grads = _correlated(n, int(offsets[-1]), dtype, seed=200 + n)
-        _run_and_check(lib, grads, offsets, dtype, flags=lib.flags_radix(first, later))
-        results.append(n)
-    assert results == [13, 64]
+        _run_and_check(lib, grads, offsets, dtype, flags=lib.flags_radix(first, later) | extra)
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("n", [33, 64, 65, 150])
+def test_radix_64_for_16_bit_inputs(lib, dtype, n):
+    offsets = workloads.offsets_from_sizes([40_000, 9, 30_011, 1, 64, 5000])
+    grads = _correlated(n, int(offsets[-1]), dtype, seed=250 + n)
+    assert lib.adasum_plan_info(int(offsets[-1]), 6, n, dtype, lib.flags_radix(64, 0))["radices"][0] == 64
+    _run_and_check(lib, grads, offsets, dtype, flags=lib.flags_radix(64, 0))
+
+
+def test_radix_64_is_refused_for_fp32(lib):
+    grads = _correlated(64, 1000, "f32", seed=260)
+    with pytest.raises(lib.AdasumError):
+        lib.adasum_reduce(grads, [0, 1000], flags=lib.flags_radix(64, 0))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+def test_unaligned_buffers_on_the_tensor_core_path(lib, dtype):
+    sizes = [3000, 33, 20_000, 7]
+    offsets = workloads.offsets_from_sizes(sizes)
+    total = int(offsets[-1])
+    base = _correlated(40, total + 1, dtype, seed=270)
+    grads = [b[1:] if w % 2 == 0 else b[:-1] for w, b in enumerate(base)]
+    assert any(g.data_ptr() % 16 for g in grads)
+    for first in (16, 32):
+        _run_and_check(lib, grads, offsets, dtype, flags=lib.flags_radix(first, 0))
 
 
 @pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
