@@ -73,11 +73,13 @@ typedef enum {
  * operands a second time to write the group's weighted sum.  R = 2 is the literal
  * level-by-level tree (three scalars a.b, a.a, b.b per pair, as in Algorithm 1).
  *
- *   bits 0..7    radix of the first level: 0 = choose automatically, else 2, 4, 8 or 16
- *   bits 8..15   radix of the later levels: 0 = same rule as the first level
- *   bit 16       ADASUM_FLAG_SIMPLE_KERNELS: use the register-only kernels everywhere instead
- *                of the shared-memory-pipelined ones (same results up to summation order;
- *                for comparison and debugging)
+ *   bits 0..7    radix of the first level: 0 = choose automatically, else 2, 4, 8, 16, 32 or,
+ *                for fp16 / bf16 inputs only, 64
+ *   bits 8..15   radix of the later levels (their operands are fp32): 0 = same rule as the
+ *                first level, else 2 ... 32
+ *   bit 16       ADASUM_FLAG_SIMPLE_KERNELS: form the Gram matrices on the fp32 pipes also at
+ *                radix 16 instead of on the tensor cores (radices above 16 are then refused;
+ *                same results up to rounding; for comparison and debugging)
  */
 #define ADASUM_FLAG_SIMPLE_KERNELS (1u << 16)
 #define ADASUM_RADIX_AUTO 0u

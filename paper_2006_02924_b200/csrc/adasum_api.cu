@@ -91,39 +91,33 @@ int pow2_ceil(int x)
 
 // Which Gram kernel serves a level.
 enum GramKind {
-    GRAM_SIMPLE,      // fp32 pipes, operands in registers (any alignment, radix <= 16)
-    GRAM_PIPELINED,   // fp32 pipes, persistent blocks, cp.async staging (16-byte aligned, radix <= 8)
+    GRAM_SIMPLE,      // fp32 pipes, operands in registers (radix <= 8; radix 16 on request)
     GRAM_MMA          // tensor cores (radix >= 16)
 };
 
-GramKind gram_kind(int radix, bool vec, bool simple_kernels)
+GramKind gram_kind(int radix, bool simple_kernels)
 {
-    if (radix >= 32 || (radix == 16 && !simple_kernels))
-        return GRAM_MMA;
-    return vec && !simple_kernels ? GRAM_PIPELINED : GRAM_SIMPLE;
+    return (radix >= 32 || (radix == 16 && !simple_kernels)) ? GRAM_MMA : GRAM_SIMPLE;
 }
 
 // Elements per segment.  One block accumulates a whole segment in fp32 (per thread: segment /
 // 256 elements; on the tensor cores: per warp segment / 8), longer tensors are finished in fp64.
 int gram_segment_length(GramKind kind, int64_t total)
 {
-    switch (kind) {
-    case GRAM_PIPELINED: return 32768;
-    case GRAM_MMA: return total >= (int64_t(1) << 26) ? 32768 : 8192;
-    default: return total >= (int64_t(1) << 23) ? 8192 : 2048;
-    }
+    if (kind == GRAM_MMA)
+        return total >= (int64_t(1) << 26) ? 32768 : 8192;
+    return total >= (int64_t(1) << 23) ? 8192 : 2048;
 }
 int min_gram_segment_length(int radix, int64_t total)
 {
-    int best = 1 << 30;
-    for (int vec = 0; vec < 2; ++vec)
-        for (int simple = 0; simple < 2; ++simple) {
-            const int len = gram_segment_length(gram_kind(radix, vec != 0, simple != 0), total);
-            best = len < best ? len : best;
-        }
-    return best;
+    const int a = gram_segment_length(gram_kind(radix, false), total);
+    const int b = gram_segment_length(gram_kind(radix, true), total);
+    return a < b ? a : b;
 }
-int wsum_segment_length(int64_t total) { return total >= (int64_t(1) << 23) ? 8192 : 2048; }
+int wsum_segment_length(int64_t total)
+{
+    return total >= (int64_t(1) << 26) ? 8192 : (total >= (int64_t(1) << 23) ? 4096 : 2048);
+}
 
 struct Level {
     int radix;
@@ -160,9 +154,9 @@ bool plan_levels(int n_workers, adasum_dtype_t dtype, uint32_t flags, LevelPlan*
         const int want = first_level ? first : later;
         int radix = want;
         if (radix == 0) {
-            radix = max_radix_for(first_level ? dtype : ADASUM_F32);
-            if (first_level ? dtype == ADASUM_F32 : true)
-                radix = 16;
+            // Measured on B200: the tensor-core Gram pass keeps up with HBM at radix 16 for fp32
+            // operands and at radix 32 for fp16 / bf16; beyond that it is bound by the tensor pipe.
+            radix = (first_level && dtype != ADASUM_F32) ? 32 : 16;
             radix = radix < cap_auto ? radix : cap_auto;
         }
         if (radix > pow2_ceil(m))
@@ -238,6 +232,7 @@ struct SegmentTable {
     Segment* d_segments = nullptr;
     int32_t* d_seg_first = nullptr;
     int32_t num_segments = 0;
+    int32_t max_segments_per_tensor = 0;
     std::vector<Segment> h_segments;
     std::vector<int32_t> h_seg_first;
 };
@@ -266,6 +261,12 @@ void build_segments(const int64_t* offsets, int32_t num_tensors, int seg_len, Se
     }
     tab->h_seg_first[num_tensors] = (int32_t)tab->h_segments.size();
     tab->num_segments = (int32_t)tab->h_segments.size();
+    tab->max_segments_per_tensor = 0;
+    for (int32_t t = 0; t < num_tensors; ++t) {
+        const int32_t n = tab->h_seg_first[t + 1] - tab->h_seg_first[t];
+        if (n > tab->max_segments_per_tensor)
+            tab->max_segments_per_tensor = n;
+    }
 }
 
 adasum_status_t get_segment_table(const int64_t* offsets, int32_t num_tensors, int seg_len,
@@ -357,8 +358,6 @@ cudaError_t allow_dynamic_smem(Kernel kernel, size_t bytes, bool (&configured)[6
     return cudaSuccess;
 }
 
-constexpr int kGramStages = 3;
-
 template <typename T, int R, bool VEC>
 cudaError_t launch_gram(GramKind kind, const OperandTable& ops, int operands, int groups_here,
                         const SegmentTable& tab, float* partials, int groups_total, int group_base,
@@ -380,26 +379,6 @@ cudaError_t launch_gram(GramKind kind, const OperandTable& ops, int operands, in
             } else {
                 return cudaErrorInvalidValue;
             }
-        }
-    }
-    if constexpr (R <= 8 && VEC) {
-        if (kind == GRAM_PIPELINED) {
-            constexpr size_t smem = (size_t)kGramStages * R * kThreads * 16;
-            auto kernel = gram_partial_pipelined_kernel<T, R, kGramStages>;
-            static bool configured[64] = {};
-            cudaError_t err = allow_dynamic_smem(kernel, smem, configured);
-            if (err != cudaSuccess)
-                return err;
-            // persistent blocks: fill every SM, never more blocks than fit at once
-            int blocks_x = multiprocessor_count() * pipelined_min_blocks<R>() / groups_here;
-            if (blocks_x > tab.num_segments)
-                blocks_x = tab.num_segments;
-            if (blocks_x < 1)
-                blocks_x = 1;
-            dim3 grid((unsigned)blocks_x, (unsigned)groups_here);
-            kernel<<<grid, kThreads, smem, stream>>>(ops, operands, tab.d_segments, tab.num_segments, partials,
-                                                     groups_total, group_base);
-            return cudaSuccess;
         }
     }
     if constexpr (R <= 16) {
@@ -428,7 +407,10 @@ cudaError_t launch_weights(const float* partials, const SegmentTable& tab, int32
                            int groups, double* gram64, float* weights, cudaStream_t stream, int* launches)
 {
     dim3 grid((unsigned)num_tensors, (unsigned)groups, (unsigned)tree_entry_blocks(R));
-    gram_finish_kernel<R><<<grid, kTreeThreads, 0, stream>>>(partials, tab.d_seg_first, operands, gram64, weights);
+    // wide blocks only pay off when some tensor has many per-segment partials to add
+    const int threads = tab.max_segments_per_tensor > 64 ? kTreeThreadsMax : 256;
+    gram_finish_kernel<R><<<grid, threads, threads * sizeof(double), stream>>>(partials, tab.d_seg_first, operands,
+                                                                                gram64, weights);
     *launches = 1;
     if constexpr (tree_entry_blocks(R) > 1) {
         dim3 grid2((unsigned)num_tensors, (unsigned)groups);
@@ -625,7 +607,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     for (int l = 0; l < plan.num_levels; ++l) {
         const Level& lv = plan.level[l];
         const bool simple_kernels = (flags & ADASUM_FLAG_SIMPLE_KERNELS) != 0;
-        const GramKind kind = gram_kind(lv.radix, vec, simple_kernels);
+        const GramKind kind = gram_kind(lv.radix, simple_kernels);
         const SegmentTable* gram_tab = nullptr;
         const SegmentTable* wsum_tab = nullptr;
         st = get_segment_table(offsets, num_tensors, gram_segment_length(kind, total), &gram_tab);

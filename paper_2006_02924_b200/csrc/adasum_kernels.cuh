@@ -14,8 +14,7 @@
 //   weighted_sum   stream the operands a second time; out = sum_i weight_i x_i.
 //
 // The Gram matrix of a group is a dense contraction X X^T (R x P times P x R).  For R <= 8 it is
-// cheap enough for the fp32 pipes (gram_partial_kernel, gram_partial_pipelined_kernel); for
-// R >= 16 it runs on the tensor cores (gram_partial_mma_kernel): fp16 / bf16 products are exact in
+// cheap enough for the fp32 pipes (gram_partial_kernel); for R >= 16 it runs on the tensor cores (gram_partial_mma_kernel): fp16 / bf16 products are exact in
 // the fp32 accumulator, fp32 inputs are split into two tf32 terms (three products).
 //
 // The kernels never wait on one another and use no floating-point atomics, so results are
@@ -54,12 +53,22 @@ __host__ __device__ constexpr int gram_index(int radix, int i, int j)
 
 // ---- element access -------------------------------------------------------------------------
 
+// Read-once data (pass 2): bypass L1 and mark the lines evict-first in L2.
 __device__ __forceinline__ uint4 load_streaming_16B(const void* p)
 {
     uint4 v;
     asm("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
         : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
         : "l"(p));
+    return v;
+}
+
+// Data that pass 2 will read again (pass 1): ordinary L2 policy, so that the last part of the
+// operands is still resident when pass 2 starts from the end.
+__device__ __forceinline__ uint4 load_keep_16B(const void* p)
+{
+    uint4 v;
+    asm("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
 }
 
@@ -72,7 +81,7 @@ struct Element<float> {
     static __device__ __forceinline__ float one(const float* p) { return __ldg(p); }
     static __device__ __forceinline__ void vec(const float* p, float (&x)[kVec])
     {
-        uint4 v = load_streaming_16B(p);
+        uint4 v = load_keep_16B(p);
         x[0] = __uint_as_float(v.x);
         x[1] = __uint_as_float(v.y);
         x[2] = __uint_as_float(v.z);
@@ -86,7 +95,7 @@ struct Element<__half> {
     static __device__ __forceinline__ float one(const __half* p) { return __half2float(__ldg(p)); }
     static __device__ __forceinline__ void vec(const __half* p, float (&x)[kVec])
     {
-        uint4 v = load_streaming_16B(p);
+        uint4 v = load_keep_16B(p);
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -107,7 +116,7 @@ struct Element<__nv_bfloat16> {
     }
     static __device__ __forceinline__ void vec(const __nv_bfloat16* p, float (&x)[kVec])
     {
-        uint4 v = load_streaming_16B(p);
+        uint4 v = load_keep_16B(p);
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {            // a bf16 is the upper half of an fp32
@@ -235,251 +244,13 @@ gram_partial_kernel(const __grid_constant__ OperandTable ops, int operands,
     }
 }
 
-// ---- pass 1, pipelined: persistent blocks, operands staged through shared memory ---------------
-//
-// The register-only kernel above cannot overlap its loads with its arithmetic at radix 16 (136
-// accumulators leave room for one column set only).  Here every thread copies its own 16 bytes of
-// each operand row into shared memory with cp.async, STAGES tiles deep, and reads back only what it
-// copied itself: no thread ever waits for another one inside the loop, so nothing can dead-lock.
-// A block walks the segments blockIdx.x, blockIdx.x + gridDim.x, ... and keeps the copy pipeline
-// running across segment boundaries; accumulators are flushed (block reduction, one partial per
-// segment) when a segment ends.  Requires 16-byte aligned operands (the VEC case).
+// ---- asynchronous copies into shared memory ----------------------------------------------------
 
-__device__ __forceinline__ void cp_async_16B(void* smem_dst, const void* gmem_src)
-{
-    const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
-}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait()
 {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-
-// Elements decoded per round from one thread's 16 bytes of a row, and how.
-template <typename T, int R>
-struct Rounds;
-template <int R>
-struct Rounds<float, R> {
-    static constexpr int kWords = 4, kElems = 4, kRounds = 1;
-    static __device__ __forceinline__ void decode(const uint32_t (&w)[kWords], float (&x)[kElems])
-    {
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            x[j] = __uint_as_float(w[j]);
-    }
-};
-template <int R>
-struct Rounds<__half, R> {
-    static constexpr int kWords = R >= 16 ? 1 : 4, kElems = 2 * kWords, kRounds = 4 / kWords;
-    static __device__ __forceinline__ void decode(const uint32_t (&w)[kWords], float (&x)[kElems])
-    {
-#pragma unroll
-        for (int j = 0; j < kWords; ++j) {
-            float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[j]));
-            x[2 * j] = f.x;
-            x[2 * j + 1] = f.y;
-        }
-    }
-};
-template <int R>
-struct Rounds<__nv_bfloat16, R> {
-    static constexpr int kWords = R >= 16 ? 1 : 4, kElems = 2 * kWords, kRounds = 4 / kWords;
-    static __device__ __forceinline__ void decode(const uint32_t (&w)[kWords], float (&x)[kElems])
-    {
-#pragma unroll
-        for (int j = 0; j < kWords; ++j) {
-            x[2 * j] = __uint_as_float(w[j] << 16);
-            x[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
-        }
-    }
-};
-
-template <int WORDS>
-__device__ __forceinline__ void load_shared_words(const unsigned char* p, uint32_t (&w)[WORDS])
-{
-    if (WORDS == 4) {
-        uint4 v = *reinterpret_cast<const uint4*>(p);
-        w[0] = v.x; w[1 % WORDS] = v.y; w[2 % WORDS] = v.z; w[3 % WORDS] = v.w;
-    } else if (WORDS == 2) {
-        uint2 v = *reinterpret_cast<const uint2*>(p);
-        w[0] = v.x; w[1 % WORDS] = v.y;
-    } else {
-        w[0] = *reinterpret_cast<const uint32_t*>(p);
-    }
-}
-
-// Where one thread stands in its block's sequence of tiles.  A tile is kThreads consecutive
-// 16-byte vectors of the aligned body of a segment.
-template <int V>
-struct TileCursor {
-    int seg;              // index into the segment table, >= num_segments when exhausted
-    int64_t v;            // element index of this thread's vector in the current tile
-    int64_t tile_begin;   // element index where the current tile starts
-    int64_t body_end;     // end of the aligned body of the current segment
-
-    __device__ __forceinline__ void enter(const Segment* __restrict__ segments, int num_segments)
-    {
-        // position on the first tile of segment `seg`, skipping segments without an aligned body
-        while (seg < num_segments) {
-            const Segment s = segments[seg];
-            int64_t bb, be;
-            split_segment<V, true>(s.begin, s.begin + s.len, bb, be);
-            if (bb < be) {
-                tile_begin = bb;
-                body_end = be;
-                v = bb + (int64_t)threadIdx.x * V;
-                return;
-            }
-            seg += gridDim.x;
-        }
-    }
-    __device__ __forceinline__ void next_tile(const Segment* __restrict__ segments, int num_segments)
-    {
-        tile_begin += (int64_t)kThreads * V;
-        v += (int64_t)kThreads * V;
-        if (tile_begin >= body_end) {
-            seg += gridDim.x;
-            enter(segments, num_segments);
-        }
-    }
-};
-
-template <int R, int E>
-__device__ __forceinline__ void block_reduce_and_store(float (&acc)[E], float (*warp_sums)[E], float* dst)
-{
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-    for (int k = 0; k < E; ++k) {
-        float s = acc[k];
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1)
-            s += __shfl_xor_sync(0xffffffffu, s, d);
-        if (lane == 0)
-            warp_sums[warp][k] = s;
-    }
-    __syncthreads();
-    for (int k = threadIdx.x; k < E; k += kThreads) {
-        float s = 0.0f;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w)
-            s += warp_sums[w][k];
-        dst[k] = s;
-    }
-    __syncthreads();   // warp_sums is reused by the next segment
-}
-
-template <int R>
-__host__ __device__ constexpr int pipelined_min_blocks() { return R >= 16 ? 1 : (R >= 8 ? 2 : 4); }
-
-// grid = (persistent blocks, groups in this launch); block = kThreads;
-// dynamic shared memory = STAGES * R * kThreads * 16 bytes.
-template <typename T, int R, int STAGES>
-__global__ void __launch_bounds__(kThreads, pipelined_min_blocks<R>())
-gram_partial_pipelined_kernel(const __grid_constant__ OperandTable ops, int operands,
-                              const Segment* __restrict__ segments, int num_segments,
-                              float* __restrict__ partials, int groups_total, int group_base)
-{
-    constexpr int E = gram_entries(R);
-    constexpr int V = Element<T>::kVec;
-    using Rd = Rounds<T, R>;
-    extern __shared__ __align__(16) unsigned char stage_mem[];
-    __shared__ float warp_sums[kWarps][E];
-
-    const int first = blockIdx.y * R;
-    const int members = min(R, operands - first);
-    unsigned char* my_smem = stage_mem + (size_t)threadIdx.x * 16;   // + (stage * R + row) * kThreads * 16
-
-    TileCursor<V> prod, cons;
-    prod.seg = blockIdx.x;
-    prod.enter(segments, num_segments);
-    cons = prod;
-
-    auto issue = [&](int stage) {
-        if (prod.seg < num_segments) {
-            if (prod.v < prod.body_end) {
-#pragma unroll
-                for (int i = 0; i < R; ++i)
-                    if (i < members)
-                        cp_async_16B(my_smem + (size_t)(stage * R + i) * kThreads * 16,
-                                     static_cast<const T*>(ops.ptr[first + i]) + prod.v);
-            }
-            prod.next_tile(segments, num_segments);
-        }
-        cp_async_commit();
-    };
-
-#pragma unroll
-    for (int s = 0; s < STAGES - 1; ++s)
-        issue(s);
-
-    int stage = 0;
-    for (int seg = blockIdx.x; seg < num_segments; seg += gridDim.x) {
-        float acc[E];
-#pragma unroll
-        for (int k = 0; k < E; ++k)
-            acc[k] = 0.0f;
-
-        // tiles of this segment's aligned body
-        while (cons.seg == seg) {
-            int refill = stage + STAGES - 1;
-            if (refill >= STAGES)
-                refill -= STAGES;
-            issue(refill);
-            cp_async_wait<STAGES - 1>();
-            if (cons.v < cons.body_end) {
-                const unsigned char* base = my_smem + (size_t)stage * R * kThreads * 16;
-#pragma unroll
-                for (int round = 0; round < Rd::kRounds; ++round) {
-                    float x[R][Rd::kElems];
-#pragma unroll
-                    for (int i = 0; i < R; ++i) {
-                        if (i < members) {
-                            uint32_t w[Rd::kWords];
-                            load_shared_words<Rd::kWords>(base + (size_t)i * kThreads * 16 + round * Rd::kWords * 4, w);
-                            Rd::decode(w, x[i]);
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < Rd::kElems; ++j)
-                                x[i][j] = 0.0f;
-                        }
-                    }
-#pragma unroll
-                    for (int j = 0; j < Rd::kElems; ++j) {
-                        float col[R];
-#pragma unroll
-                        for (int i = 0; i < R; ++i)
-                            col[i] = x[i][j];
-                        gram_accumulate<R>(col, acc);
-                    }
-                }
-            }
-            cons.next_tile(segments, num_segments);
-            if (++stage == STAGES)
-                stage = 0;
-        }
-
-        // scalar head and tail of the segment, straight from global memory
-        const Segment s = segments[seg];
-        const int64_t begin = s.begin, end = s.begin + s.len;
-        int64_t body_begin, body_end;
-        split_segment<V, true>(begin, end, body_begin, body_end);
-        for (int pass = 0; pass < 2; ++pass) {
-            const int64_t lo = pass == 0 ? begin : body_end;
-            const int64_t hi = pass == 0 ? body_begin : end;
-            for (int64_t e = lo + threadIdx.x; e < hi; e += kThreads) {
-                float col[R];
-#pragma unroll
-                for (int i = 0; i < R; ++i)
-                    col[i] = i < members ? Element<T>::one(static_cast<const T*>(ops.ptr[first + i]) + e) : 0.0f;
-                gram_accumulate<R>(col, acc);
-            }
-        }
-        block_reduce_and_store<R, E>(acc, warp_sums,
-                                     partials + ((int64_t)seg * groups_total + group_base + blockIdx.y) * E);
-    }
-    cp_async_wait<0>();
 }
 
 // ---- pass 1 on the tensor cores ----------------------------------------------------------------
@@ -933,9 +704,8 @@ __device__ void tree_weights_from_gram(const double* gram, int members, float* _
         dst[tid] = tid < members ? (float)weight[tid] : 0.0f;
 }
 
-constexpr int kTreeThreads = 1024;
-// Entries of the packed Gram matrix handled by one block of gram_finish_kernel, and the number of
-// slices its segments are split into (entries * slices <= kTreeThreads).
+constexpr int kTreeThreadsMax = 1024;
+// Entries of the packed Gram matrix handled by one block of gram_finish_kernel.
 __host__ __device__ constexpr int tree_entries_per_block(int radix)
 {
     return gram_entries(radix) < 256 ? gram_entries(radix) : 256;
@@ -944,29 +714,27 @@ __host__ __device__ constexpr int tree_entry_blocks(int radix)
 {
     return (gram_entries(radix) + tree_entries_per_block(radix) - 1) / tree_entries_per_block(radix);
 }
-__host__ __device__ constexpr int tree_slices(int radix)
-{
-    return kTreeThreads / tree_entries_per_block(radix) < 64 ? kTreeThreads / tree_entries_per_block(radix) : 64;
-}
 
-// grid = (tensors, groups, tree_entry_blocks(R)); block = kTreeThreads.
-// Adds the tensor's per-segment partial matrices in fp64: slice q takes segments q, q + Q, ... in
-// order, then the slices are added in order (fixed order: deterministic).  When the whole matrix
-// fits one block (R <= 16) the same block goes on to run the tree and writes
-// weights[(tensor * groups + group) * R + i]; otherwise it stores its entries to gram64 and
-// tree_weights_kernel finishes.
+// grid = (tensors, groups, tree_entry_blocks(R)); block = 256 or 1024 threads (1024 when some
+// tensor has many segments); dynamic shared memory = blockDim.x * 8 bytes.
+// Adds the tensor's per-segment partial matrices in fp64: with Q = blockDim.x / entries slices,
+// slice q takes segments q, q + Q, ... in order, then the slices are added in order (fixed order
+// for a given block size: deterministic).  When the whole matrix fits one block (R <= 16) the
+// same block goes on to run the tree and writes weights[(tensor * groups + group) * R + i];
+// otherwise it stores its entries to gram64 and tree_weights_kernel finishes.
 template <int R>
-__global__ void __launch_bounds__(kTreeThreads)
+__global__ void __launch_bounds__(kTreeThreadsMax)
 gram_finish_kernel(const float* __restrict__ partials, const int32_t* __restrict__ seg_first, int operands,
                    double* __restrict__ gram64, float* __restrict__ weights)
 {
     constexpr int E = gram_entries(R);
     constexpr int EPB = tree_entries_per_block(R);
-    constexpr int Q = tree_slices(R);
     constexpr bool SINGLE = tree_entry_blocks(R) == 1;
-    __shared__ double slice_sum[Q][EPB];
+    extern __shared__ __align__(16) unsigned char finish_smem[];
+    double* slice_sum = reinterpret_cast<double*>(finish_smem);      // [Q][EPB]
     __shared__ double gram[SINGLE ? E : 1];
 
+    const int Q = blockDim.x / EPB;
     const int tensor = blockIdx.x, group = blockIdx.y, groups = gridDim.y;
     const int s0 = seg_first[tensor], s1 = seg_first[tensor + 1];
     const int q = threadIdx.x / EPB, kk = threadIdx.x - q * EPB;
@@ -980,13 +748,13 @@ gram_finish_kernel(const float* __restrict__ partials, const int32_t* __restrict
             for (int seg = s0 + q; seg < s1; seg += Q)
                 s += (double)__ldg(src + seg * stride);
         }
-        slice_sum[q][kk] = s;
+        slice_sum[q * EPB + kk] = s;
     }
     __syncthreads();
     if (q == 0 && k < E) {
-        double s = slice_sum[0][kk];
+        double s = slice_sum[kk];
         for (int qq = 1; qq < Q; ++qq)
-            s += slice_sum[qq][kk];
+            s += slice_sum[qq * EPB + kk];
         if (SINGLE)
             gram[kk] = s;
         else
@@ -1062,17 +830,33 @@ weighted_sum_kernel(const __grid_constant__ OperandTable ops, int operands,
 {
     constexpr int V = Element<T>::kVec;
     constexpr int BATCH = R < 8 ? R : 8;
-    const Segment seg = segments[blockIdx.x];
+    // Segments are taken last to first: pass 1 walked them first to last, so the tail of the
+    // operands is what the L2 still holds when this kernel starts.
+    const Segment seg = segments[gridDim.x - 1 - blockIdx.x];
     const int first = blockIdx.y * R;
     const int members = min(R, operands - first);
     const int group = group_base + blockIdx.y;
 
-    __shared__ float w[R];
-    if (threadIdx.x < R)
-        w[threadIdx.x] = threadIdx.x < members
-                             ? __ldg(weights + ((int64_t)seg.tensor * groups_total + group) * R + threadIdx.x)
-                             : 0.0f;
-    __syncthreads();
+    // leaf weights: registers for small groups, shared memory for the wide ones
+    constexpr bool W_IN_SMEM = R > 16;
+    __shared__ float w_smem[W_IN_SMEM ? R : 1];
+    float w_reg[W_IN_SMEM ? 1 : R];
+    const float* wsrc = weights + ((int64_t)seg.tensor * groups_total + group) * R;
+    if constexpr (W_IN_SMEM) {
+        if (threadIdx.x < R)
+            w_smem[threadIdx.x] = threadIdx.x < members ? __ldg(wsrc + threadIdx.x) : 0.0f;
+        __syncthreads();
+    } else {
+#pragma unroll
+        for (int i = 0; i < R; ++i)
+            w_reg[i] = i < members ? __ldg(wsrc + i) : 0.0f;
+    }
+    auto w = [&](int i) -> float {
+        if constexpr (W_IN_SMEM)
+            return w_smem[i];
+        else
+            return w_reg[i];
+    };
     float* dst = dst_base + (int64_t)group * dst_stride;
 
     const int64_t begin = seg.begin, end = seg.begin + seg.len;
@@ -1098,7 +882,7 @@ weighted_sum_kernel(const __grid_constant__ OperandTable ops, int operands,
                 if (b + i < members) {
                     float x[V];
                     decode_vector<T>(raw[i], x);
-                    const float wi = w[b + i];
+                    const float wi = w(b + i);
 #pragma unroll
                     for (int j = 0; j < V; ++j)
                         y[j] = fmaf(wi, x[j], y[j]);
@@ -1114,8 +898,10 @@ weighted_sum_kernel(const __grid_constant__ OperandTable ops, int operands,
         const int64_t hi = pass == 0 ? body_begin : end;
         for (int64_t e = lo + threadIdx.x; e < hi; e += kThreads) {
             float y = 0.0f;
-            for (int i = 0; i < members; ++i)
-                y = fmaf(w[i], Element<T>::one(static_cast<const T*>(ops.ptr[first + i]) + e), y);
+#pragma unroll
+            for (int i = 0; i < R; ++i)
+                if (i < members)
+                    y = fmaf(w(i), Element<T>::one(static_cast<const T*>(ops.ptr[first + i]) + e), y);
             dst[e] = y;
         }
     }
