@@ -80,8 +80,12 @@ typedef enum {
  *   bit 16       ADASUM_FLAG_SIMPLE_KERNELS: form the Gram matrices on the fp32 pipes also at
  *                radix 16 instead of on the tensor cores (radices above 16 are then refused;
  *                same results up to rounding; for comparison and debugging)
+ *   bit 17       ADASUM_FLAG_SEPARATE_FINISH: add up the per-segment Gram matrices and derive
+ *                the leaf weights in a kernel of their own at every level, instead of inside
+ *                the first pass (radix <= 16); for comparison and debugging
  */
 #define ADASUM_FLAG_SIMPLE_KERNELS (1u << 16)
+#define ADASUM_FLAG_SEPARATE_FINISH (1u << 17)
 #define ADASUM_RADIX_AUTO 0u
 #define ADASUM_FLAGS_RADIX(first, later) (((uint32_t)(first) & 0xffu) | (((uint32_t)(later) & 0xffu) << 8))
 

@@ -105,7 +105,7 @@ GramKind gram_kind(int radix, bool simple_kernels)
 int gram_segment_length(GramKind kind, int64_t total)
 {
     if (kind == GRAM_MMA)
-        return total >= (int64_t(1) << 26) ? 32768 : 8192;
+        return total >= (int64_t(1) << 26) ? 32768 : (total >= (int64_t(1) << 23) ? 16384 : 8192);
     return total >= (int64_t(1) << 23) ? 8192 : 2048;
 }
 int min_gram_segment_length(int radix, int64_t total)
@@ -133,7 +133,7 @@ struct LevelPlan {
 bool plan_levels(int n_workers, adasum_dtype_t dtype, uint32_t flags, LevelPlan* plan)
 {
     const int first = (int)(flags & 0xffu), later_flag = (int)((flags >> 8) & 0xffu);
-    if ((flags >> 17) != 0)
+    if ((flags >> 18) != 0)
         return false;
     if (first != 0 && (!valid_radix(first) || first > max_radix_for(dtype)))
         return false;
@@ -176,8 +176,8 @@ int64_t segment_bound(int64_t total, int32_t num_tensors, int seg_len)
 }
 
 struct Layout {
-    size_t partials = 0, weights = 0, gram64 = 0, buffer[2] = {0, 0};
-    size_t partials_bytes = 0, weights_bytes = 0, gram64_bytes = 0, buffer_bytes[2] = {0, 0};
+    size_t partials = 0, weights = 0, gram64 = 0, counters = 0, buffer[2] = {0, 0};
+    size_t partials_bytes = 0, weights_bytes = 0, gram64_bytes = 0, counters_bytes = 0, buffer_bytes[2] = {0, 0};
     int64_t padded_elems = 0;
     size_t total = 0;
 };
@@ -196,6 +196,11 @@ Layout make_layout(const LevelPlan& plan, int64_t total_elems, int32_t num_tenso
             lay.partials_bytes = p;
         if (w > lay.weights_bytes)
             lay.weights_bytes = w;
+        if (lv.radix <= 16) {
+            const size_t c = (size_t)(num_tensors > 0 ? num_tensors : 1) * lv.groups * sizeof(int);
+            if (c > lay.counters_bytes)
+                lay.counters_bytes = c;
+        }
         if (lv.radix >= 32) {
             const size_t g64 = (size_t)(num_tensors > 0 ? num_tensors : 1) * lv.groups * gram_entries(lv.radix) *
                                sizeof(double);
@@ -215,6 +220,8 @@ Layout make_layout(const LevelPlan& plan, int64_t total_elems, int32_t num_tenso
     off += align_up(lay.weights_bytes);
     lay.gram64 = off;
     off += align_up(lay.gram64_bytes);
+    lay.counters = off;
+    off += align_up(lay.counters_bytes);
     lay.buffer[0] = off;
     off += align_up(lay.buffer_bytes[0]);
     lay.buffer[1] = off;
@@ -361,7 +368,7 @@ cudaError_t allow_dynamic_smem(Kernel kernel, size_t bytes, bool (&configured)[6
 template <typename T, int R, bool VEC>
 cudaError_t launch_gram(GramKind kind, const OperandTable& ops, int operands, int groups_here,
                         const SegmentTable& tab, float* partials, int groups_total, int group_base,
-                        cudaStream_t stream)
+                        const FinishArgs& fin, cudaStream_t stream)
 {
     if constexpr (R >= 16) {
         if (kind == GRAM_MMA) {
@@ -374,7 +381,7 @@ cudaError_t launch_gram(GramKind kind, const OperandTable& ops, int operands, in
                     return err;
                 dim3 grid((unsigned)tab.num_segments, (unsigned)groups_here);
                 kernel<<<grid, kThreads, smem, stream>>>(ops, operands, tab.d_segments, partials, groups_total,
-                                                         group_base);
+                                                         group_base, fin);
                 return cudaSuccess;
             } else {
                 return cudaErrorInvalidValue;
@@ -385,7 +392,7 @@ cudaError_t launch_gram(GramKind kind, const OperandTable& ops, int operands, in
         if (kind == GRAM_SIMPLE) {
             dim3 grid((unsigned)tab.num_segments, (unsigned)groups_here);
             gram_partial_kernel<T, R, VEC><<<grid, kThreads, 0, stream>>>(ops, operands, tab.d_segments, partials,
-                                                                          groups_total, group_base);
+                                                                          groups_total, group_base, fin);
             return cudaSuccess;
         }
     }
@@ -429,6 +436,7 @@ struct LevelArgs {
     const SegmentTable* wsum_tab;
     int32_t num_tensors;
     float* partials;
+    int* counters;      // ticket counters for finishing inside pass 1, or nullptr
     double* gram64;
     float* weights;
     float* dst;
@@ -442,6 +450,9 @@ template <typename T, int R>
 adasum_status_t run_level_typed(const LevelArgs& a)
 {
     constexpr int kGroupsPerLaunch = kMaxOperandsPerLaunch / R;
+    // radix <= 16: the last block of every (tensor, group) in pass 1 also derives the weights
+    const bool fused_finish = R <= 16 && a.counters != nullptr;
+    const FinishArgs fin{a.gram_tab->d_seg_first, fused_finish ? a.counters : nullptr, a.weights};
     // pass 1
     for (int g0 = 0; g0 < a.groups; g0 += kGroupsPerLaunch) {
         const int groups_here = a.groups - g0 < kGroupsPerLaunch ? a.groups - g0 : kGroupsPerLaunch;
@@ -452,16 +463,18 @@ adasum_status_t run_level_typed(const LevelArgs& a)
             table.ptr[i] = a.operand_ptrs[op0 + (i < ops_here ? i : 0)];
         if (a.vec)
             ADASUM_CUDA_CHECK((launch_gram<T, R, true>(a.kind, table, ops_here, groups_here, *a.gram_tab,
-                                                       a.partials, a.groups, g0, a.stream)));
+                                                       a.partials, a.groups, g0, fin, a.stream)));
         else
             ADASUM_CUDA_CHECK((launch_gram<T, R, false>(a.kind, table, ops_here, groups_here, *a.gram_tab,
-                                                        a.partials, a.groups, g0, a.stream)));
+                                                        a.partials, a.groups, g0, fin, a.stream)));
         profile_mark(a.stream, ADASUM_KERNEL_GRAM_PARTIAL, a.level, R, false);
     }
-    int weight_launches = 0;
-    ADASUM_CUDA_CHECK(launch_weights<R>(a.partials, *a.gram_tab, a.num_tensors, a.operands, a.groups, a.gram64,
-                                        a.weights, a.stream, &weight_launches));
-    profile_mark(a.stream, ADASUM_KERNEL_TREE_WEIGHTS, a.level, R, false);
+    if (!fused_finish) {
+        int weight_launches = 0;
+        ADASUM_CUDA_CHECK(launch_weights<R>(a.partials, *a.gram_tab, a.num_tensors, a.operands, a.groups,
+                                            a.gram64, a.weights, a.stream, &weight_launches));
+        profile_mark(a.stream, ADASUM_KERNEL_TREE_WEIGHTS, a.level, R, false);
+    }
     // pass 2
     for (int g0 = 0; g0 < a.groups; g0 += kGroupsPerLaunch) {
         const int groups_here = a.groups - g0 < kGroupsPerLaunch ? a.groups - g0 : kGroupsPerLaunch;
@@ -500,7 +513,7 @@ adasum_status_t run_level(int radix, const LevelArgs& a)
     }
 }
 
-int launches_of(const LevelPlan& plan, int n_workers)
+int launches_of(const LevelPlan& plan, int n_workers, uint32_t flags)
 {
     if (n_workers == 1)
         return 1;
@@ -508,7 +521,11 @@ int launches_of(const LevelPlan& plan, int n_workers)
     for (int l = 0; l < plan.num_levels; ++l) {
         const int per_launch = kMaxOperandsPerLaunch / plan.level[l].radix;
         const int batches = (plan.level[l].groups + per_launch - 1) / per_launch;
-        n += 2 * batches + (plan.level[l].radix >= 32 ? 2 : 1);
+        n += 2 * batches;
+        if (plan.level[l].radix >= 32)
+            n += 2;                                     // gram_finish + tree_weights
+        else if (flags & ADASUM_FLAG_SEPARATE_FINISH)
+            n += 1;                                     // gram_finish (otherwise done inside pass 1)
     }
     return n;
 }
@@ -603,6 +620,9 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     }
 
     char* ws = static_cast<char*>(workspace);
+    const bool separate_finish = (flags & ADASUM_FLAG_SEPARATE_FINISH) != 0;
+    if (!separate_finish && lay.counters_bytes > 0)     // the workspace arrives with unknown contents
+        ADASUM_CUDA_CHECK(cudaMemsetAsync(ws + lay.counters, 0, lay.counters_bytes, stream));
     std::vector<const void*> operand_ptrs(grads, grads + n_workers);
     for (int l = 0; l < plan.num_levels; ++l) {
         const Level& lv = plan.level[l];
@@ -628,6 +648,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         a.partials = reinterpret_cast<float*>(ws + lay.partials);
         a.weights = reinterpret_cast<float*>(ws + lay.weights);
         a.gram64 = reinterpret_cast<double*>(ws + lay.gram64);
+        a.counters = separate_finish ? nullptr : reinterpret_cast<int*>(ws + lay.counters);
         a.dst = last ? out : reinterpret_cast<float*>(ws + lay.buffer[l & 1]);
         a.dst_stride = last ? 0 : lay.padded_elems;
         a.vec = vec;
@@ -699,8 +720,9 @@ template <typename T>
 cudaError_t noalloc_launch(bool vec, const OperandTable& ops, const SegmentTable& tab, int32_t num_tensors,
                            float* partials, float* weights, float* out, cudaStream_t stream)
 {
-    cudaError_t err = vec ? launch_gram<T, 2, true>(GRAM_SIMPLE, ops, 2, 1, tab, partials, 1, 0, stream)
-                          : launch_gram<T, 2, false>(GRAM_SIMPLE, ops, 2, 1, tab, partials, 1, 0, stream);
+    const FinishArgs no_fusion{nullptr, nullptr, nullptr};
+    cudaError_t err = vec ? launch_gram<T, 2, true>(GRAM_SIMPLE, ops, 2, 1, tab, partials, 1, 0, no_fusion, stream)
+                          : launch_gram<T, 2, false>(GRAM_SIMPLE, ops, 2, 1, tab, partials, 1, 0, no_fusion, stream);
     if (err != cudaSuccess)
         return err;
     int weight_launches = 0;
@@ -817,7 +839,7 @@ adasum_status_t adasum_plan_info(int64_t total_elems, int32_t num_tensors, int32
     if (num_levels)
         *num_levels = plan.num_levels;
     if (num_launches)
-        *num_launches = total_elems == 0 ? 0 : launches_of(plan, n_workers);
+        *num_launches = total_elems == 0 ? 0 : launches_of(plan, n_workers, flags);
     return ADASUM_OK;
 }
 

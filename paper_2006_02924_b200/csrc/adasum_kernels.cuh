@@ -143,6 +143,51 @@ __device__ __forceinline__ void split_segment(int64_t begin, int64_t end, int64_
     }
 }
 
+// ---- finishing a group inside pass 1 -----------------------------------------------------------
+//
+// For radix <= 16 the block that writes the LAST per-segment partial matrix of a (tensor, group)
+// also adds up all of that tensor's partials and derives the leaf weights, so no separate launch
+// (and no idle GPU while a small kernel runs) separates pass 1 from pass 2.  "Last" is decided by
+// an integer ticket counter per (tensor, group); the sums themselves are taken in segment order,
+// so the result does not depend on which block happens to be last.  The counter is returned to
+// zero by that block.  counters == nullptr switches the mechanism off (the caller then launches
+// gram_finish_kernel).
+struct FinishArgs {
+    const int32_t* seg_first;   // num_tensors + 1: first segment of every tensor
+    int* counters;              // [tensor][group], zero on entry
+    float* weights;             // [tensor][group][R]
+};
+
+template <int R>
+__device__ void finish_group_in_block(const float* partials, int seg_begin, int seg_end, int group,
+                                      int groups_total, int members, float* weights_dst);
+
+// Called by every thread of the block after its partial matrix has been written.
+template <int R>
+__device__ __forceinline__ void finish_if_last(const FinishArgs& fin, const float* partials, int tensor, int group,
+                                               int groups_total, int members)
+{
+    if (fin.counters == nullptr)
+        return;
+    __shared__ int is_last;
+    __threadfence();                       // this block's partial is visible device-wide ...
+    __syncthreads();
+    const int s0 = fin.seg_first[tensor], s1 = fin.seg_first[tensor + 1];
+    if (threadIdx.x == 0) {
+        int* counter = fin.counters + (int64_t)tensor * groups_total + group;
+        const int ticket = atomicAdd(counter, 1);      // ... before its ticket is drawn
+        is_last = ticket == s1 - s0 - 1;
+        if (is_last)
+            *counter = 0;                  // ready for the next level / the next call
+    }
+    __syncthreads();
+    if (is_last) {
+        __threadfence();
+        finish_group_in_block<R>(partials, s0, s1, group, groups_total, members,
+                                 fin.weights + ((int64_t)tensor * groups_total + group) * R);
+    }
+}
+
 // ---- pass 1: partial Gram matrices -------------------------------------------------------------
 
 template <int R>
@@ -165,7 +210,7 @@ template <typename T, int R, bool VEC>
 __global__ void __launch_bounds__(kThreads)
 gram_partial_kernel(const __grid_constant__ OperandTable ops, int operands,
                     const Segment* __restrict__ segments, float* __restrict__ partials,
-                    int groups_total, int group_base)
+                    int groups_total, int group_base, FinishArgs fin)
 {
     constexpr int E = gram_entries(R);
     constexpr int V = Element<T>::kVec;
@@ -242,6 +287,8 @@ gram_partial_kernel(const __grid_constant__ OperandTable ops, int operands,
             s += warp_sums[w][k];
         dst[k] = s;
     }
+    if constexpr (R <= 16)
+        finish_if_last<R>(fin, partials, seg.tensor, group_base + blockIdx.y, groups_total, members);
 }
 
 // ---- asynchronous copies into shared memory ----------------------------------------------------
@@ -413,7 +460,7 @@ template <typename T, int R, bool VEC>
 __global__ void __launch_bounds__(kThreads, mma_min_blocks<T, R>())
 gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
                         const Segment* __restrict__ segments, float* __restrict__ partials,
-                        int groups_total, int group_base)
+                        int groups_total, int group_base, FinishArgs fin)
 {
     constexpr int E = gram_entries(R);
     constexpr int V = Element<T>::kVec;          // elements per 16-byte vector
@@ -632,6 +679,8 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
         }
         dst[gram_index(R, i, j)] = v;
     }
+    if constexpr (R <= 16)
+        finish_if_last<R>(fin, partials, seg.tensor, group_base + blockIdx.y, groups_total, members);
 }
 
 // ---- coefficients: the binary tree evaluated on a Gram matrix ---------------------------------
@@ -702,6 +751,40 @@ __device__ void tree_weights_from_gram(const double* gram, int members, float* _
     }
     if (tid < R)
         dst[tid] = tid < members ? (float)weight[tid] : 0.0f;
+}
+
+// The tensor's partial matrices (segments seg_begin .. seg_end) added in fp64 by one block of
+// kThreads threads, then the tree.  With Q = kThreads / E slices, slice q takes segments
+// q, q + Q, ... in order and the slices are added in order.  Partials were written by other
+// blocks of the running kernel, hence the L2 loads.
+template <int R>
+__device__ void finish_group_in_block(const float* partials, int seg_begin, int seg_end, int group,
+                                      int groups_total, int members, float* weights_dst)
+{
+    constexpr int E = gram_entries(R);
+    static_assert(E <= kThreads, "one thread per entry");
+    constexpr int Q = kThreads / E;
+    __shared__ double slice_sum[kThreads];
+    __shared__ double gram[E];
+    const int q = threadIdx.x / E, kk = threadIdx.x - q * E;
+    if (q < Q) {
+        const float* src = partials + (int64_t)group * E + kk;
+        const int64_t stride = (int64_t)groups_total * E;
+        double s = 0.0;
+#pragma unroll 8
+        for (int seg = seg_begin + q; seg < seg_end; seg += Q)
+            s += (double)__ldcg(src + seg * stride);
+        slice_sum[q * E + kk] = s;
+    }
+    __syncthreads();
+    if (threadIdx.x < E) {
+        double s = slice_sum[threadIdx.x];
+        for (int qq = 1; qq < Q; ++qq)
+            s += slice_sum[qq * E + threadIdx.x];
+        gram[threadIdx.x] = s;
+    }
+    __syncthreads();
+    tree_weights_from_gram<R>(gram, members, weights_dst);
 }
 
 constexpr int kTreeThreadsMax = 1024;

@@ -69,7 +69,11 @@ def test_plan_info(binding):
     assert info(100, 1, 256, "f32", binding.flags_radix(16, 16))["radices"] == [16, 16]
     assert info(100, 1, 5, "f32", binding.flags_radix(4, 4))["radices"] == [4, 2]
     assert info(0, 0, 4, "f32")["launches"] == 0
-    assert info(100, 1, 8, "f32", binding.flags_radix(2, 2))["launches"] == 9
+    assert info(100, 1, 8, "f32", binding.flags_radix(2, 2))["launches"] == 6
+    assert info(100, 1, 8, "f32", binding.flags_radix(2, 2) | (1 << 17))["launches"] == 9
+    assert info(100, 1, 64, "f16")["radices"] == [32, 2]
+    assert info(100, 1, 64, "f16")["launches"] == 4 + 2
+    assert info(100, 1, 256, "f32")["radices"] == [16, 16]
 
 
 def _call_reduce(binding, ptrs, offsets, n, dtype=0, out=0x10000000, ws=0x20000000, ws_bytes=1 << 40, flags=0,
@@ -94,6 +98,7 @@ def test_argument_errors_are_caught_on_the_host(binding):
     assert s(_call_reduce(binding, good, [0, 8, 4], 2)) == "ADASUM_ERR_OFFSETS"
     assert s(_call_reduce(binding, good, [0, 8], 2, flags=3)) == "ADASUM_ERR_ARG"
     assert s(_call_reduce(binding, good, [0, 8], 2, flags=1 << 20)) == "ADASUM_ERR_ARG"
+    assert s(_call_reduce(binding, good, [0, 8], 2, flags=64)) == "ADASUM_ERR_ARG"        # radix 64 needs 16-bit inputs
     assert s(_call_reduce(binding, [0x30000000, 0], [0, 8], 2)) == "ADASUM_ERR_NULL"
     assert s(_call_reduce(binding, good, [0, 8], 2, out=0)) == "ADASUM_ERR_NULL"
     assert s(_call_reduce(binding, good, [0, 8], 2, out=0x10000002)) == "ADASUM_ERR_ARG"

@@ -131,12 +131,14 @@ def test_awkward_shapes(lib, dtype, n):
     _run_and_check(lib, grads, offsets, dtype)
 
 
-SIMPLE = 1 << 16    # ADASUM_FLAG_SIMPLE_KERNELS
+SIMPLE = 1 << 16      # ADASUM_FLAG_SIMPLE_KERNELS
+SEPARATE = 1 << 17    # ADASUM_FLAG_SEPARATE_FINISH
 
 
 @pytest.mark.parametrize("first,later,extra", [
     (2, 2, 0), (4, 4, 0), (8, 8, 0), (16, 16, 0), (4, 2, 0), (2, 16, 0), (16, 2, 0), (32, 32, 0), (32, 4, 0),
-    (2, 32, 0), (2, 2, SIMPLE), (8, 4, SIMPLE), (16, 16, SIMPLE)])
+    (2, 32, 0), (2, 2, SIMPLE), (8, 4, SIMPLE), (16, 16, SIMPLE), (2, 2, SEPARATE), (16, 8, SEPARATE),
+    (16, 16, SIMPLE | SEPARATE)])
 @pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
 def test_every_radix_gives_the_same_tree(lib, dtype, first, later, extra):
     offsets = workloads.offsets_from_sizes([50_000, 17, 3, 70_001, 64])
