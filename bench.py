@@ -35,7 +35,13 @@ NOMINAL_HBM_GBS = 8000.0
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures of the
 # kernels as built from the source whose fingerprint is recorded with them; see profiles/.
 # {(workload, kernel, level): bytes}.  Reported only while the kernel source is unchanged.
-NCU_TRAFFIC = {"fingerprint": None, "bytes": {}}
+NCU_TRAFFIC = {
+    "fingerprint": "072e5b354eb33ba7",
+    "bytes": {
+        "c2/gram_partial/0": 822188032,      # profiles/gram_partial_f32_r8_c2.txt
+        "c2/weighted_sum/0": 874497024,      # profiles/weighted_sum_f32_r8_c2.txt
+    },
+}
 
 
 def kernel_source_fingerprint() -> str:
@@ -383,6 +389,19 @@ def aggregate_over_ranks(ms_local: float, bytes_local: float, world: int, device
     return float(t.item()), float(b.item())
 
 
+def resolve_spec(name, n_workers=None, tensor_list=None):
+    """The named configuration, optionally with another worker count / tensor list (smaller cases
+    of the same kernels, e.g. for profiler captures)."""
+    import dataclasses
+
+    spec = workloads.SPECS[name]
+    if n_workers:
+        spec = dataclasses.replace(spec, n_workers=int(n_workers))
+    if tensor_list:
+        spec = dataclasses.replace(spec, tensor_list=tensor_list)
+    return spec
+
+
 def measure_workload(lib, name, steps, warmup, flags, replica, world, sampler=None):
     wl = workloads.generate(name, device="cuda", replica=replica)
     ms, out, ws = time_reduce(lib, wl, steps, warmup, flags, world=world, sampler=sampler)
@@ -419,7 +438,8 @@ def cuda_arm(args):
     sampler = ClockSampler(local_rank)
     steps, warmup = max(args.steps, 1), max(args.warmup, 3)
 
-    wl, ms_local, out, ws = measure_workload(lib, args.workload, steps, warmup, flags, rank, world, sampler)
+    main_spec = resolve_spec(args.workload, args.n_workers, args.tensor_list)
+    wl, ms_local, out, ws = measure_workload(lib, main_spec, steps, warmup, flags, rank, world, sampler)
     ms, job_bytes = aggregate_over_ranks(ms_local, float(wl.input_bytes), world, "cuda")
     value = job_bytes / (ms * 1e-3) / 1e9
 
@@ -469,7 +489,7 @@ def cuda_arm(args):
     others = []
     if rank == 0 and world == 1 and not args.no_other_workloads:
         for name in ("c1", "c2", "c3", "c4", "c5"):
-            if name == args.workload:
+            if name == args.workload and not (args.n_workers or args.tensor_list):
                 continue
             k = max(3, min(steps, 10 if name in ("c3", "c4", "c5") else 200))
             owl, oms, oout, ows = measure_workload(lib, name, k, 3, flags, 0, 1)
@@ -510,6 +530,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--workload", default="c2", choices=sorted(workloads.SPECS))
+    ap.add_argument("--n-workers", type=int, default=0, help="override the configuration's worker count")
+    ap.add_argument("--tensor-list", default="", choices=["", "single", "resnet50", "bert_large"],
+                    help="override the configuration's tensor list")
     ap.add_argument("--radix-first", type=int, default=0)
     ap.add_argument("--radix-later", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
