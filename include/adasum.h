@@ -78,11 +78,11 @@ typedef enum {
  *   bits 8..15   radix of the later levels (their operands are fp32): 0 = same rule as the
  *                first level, else 2 ... 32
  *   bit 16       ADASUM_FLAG_SIMPLE_KERNELS: form the Gram matrices on the fp32 pipes also at
- *                radix 16 instead of on the tensor cores (radices above 16 are then refused;
+ *                radix 8 and 16 instead of on the tensor cores (radices above 16 are then refused;
  *                same results up to rounding; for comparison and debugging)
  *   bit 17       ADASUM_FLAG_SEPARATE_FINISH: add up the per-segment Gram matrices and derive
  *                the leaf weights in a kernel of their own at every level, instead of inside
- *                the first pass (radix <= 16); for comparison and debugging
+ *                the first pass; for comparison and debugging
  */
 #define ADASUM_FLAG_SIMPLE_KERNELS (1u << 16)
 #define ADASUM_FLAG_SEPARATE_FINISH (1u << 17)

@@ -4,6 +4,7 @@
 
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
@@ -91,13 +92,13 @@ int pow2_ceil(int x)
 
 // Which Gram kernel serves a level.
 enum GramKind {
-    GRAM_SIMPLE,      // fp32 pipes, operands in registers (radix <= 8; radix 16 on request)
-    GRAM_MMA          // tensor cores (radix >= 16)
+    GRAM_SIMPLE,      // fp32 pipes, operands in registers (radix <= 4; radix 8 and 16 on request)
+    GRAM_MMA          // tensor cores (radix >= 8)
 };
 
 GramKind gram_kind(int radix, bool simple_kernels)
 {
-    return (radix >= 32 || (radix == 16 && !simple_kernels)) ? GRAM_MMA : GRAM_SIMPLE;
+    return (radix >= 32 || (radix >= 8 && !simple_kernels)) ? GRAM_MMA : GRAM_SIMPLE;
 }
 
 // Elements per segment.  One block accumulates a whole segment in fp32 (per thread: segment /
@@ -196,11 +197,9 @@ Layout make_layout(const LevelPlan& plan, int64_t total_elems, int32_t num_tenso
             lay.partials_bytes = p;
         if (w > lay.weights_bytes)
             lay.weights_bytes = w;
-        if (lv.radix <= 16) {
-            const size_t c = (size_t)(num_tensors > 0 ? num_tensors : 1) * lv.groups * sizeof(int);
-            if (c > lay.counters_bytes)
-                lay.counters_bytes = c;
-        }
+        const size_t c = (size_t)(num_tensors > 0 ? num_tensors : 1) * lv.groups * sizeof(int);
+        if (c > lay.counters_bytes)
+            lay.counters_bytes = c;
         if (lv.radix >= 32) {
             const size_t g64 = (size_t)(num_tensors > 0 ? num_tensors : 1) * lv.groups * gram_entries(lv.radix) *
                                sizeof(double);
@@ -248,12 +247,24 @@ std::mutex g_tables_mutex;
 std::vector<std::unique_ptr<SegmentTable>> g_tables;
 constexpr size_t kMaxCachedTables = 64;
 
+// Segments are listed tensor by tensor, LARGEST tensor first (ties in index order): the blocks of
+// pass 1 that run last then belong to small tensors, whose per-tensor finish (adding the partial
+// matrices, tree weights) is short, instead of leaving one SM busy with a long tensor's finish
+// while the rest of the GPU idles.  Each tensor's segments stay contiguous, in element order.
 void build_segments(const int64_t* offsets, int32_t num_tensors, int seg_len, SegmentTable* tab)
 {
+    std::vector<int32_t> order((size_t)num_tensors);
+    for (int32_t t = 0; t < num_tensors; ++t)
+        order[t] = t;
+    std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) {
+        return offsets[x + 1] - offsets[x] > offsets[y + 1] - offsets[y];
+    });
     tab->h_segments.clear();
-    tab->h_seg_first.assign((size_t)num_tensors + 1, 0);
-    for (int32_t t = 0; t < num_tensors; ++t) {
-        tab->h_seg_first[t] = (int32_t)tab->h_segments.size();
+    // h_seg_first[2 t], h_seg_first[2 t + 1]: first and one-past-last segment of tensor t
+    tab->h_seg_first.assign(2 * (size_t)num_tensors + 2, 0);
+    tab->max_segments_per_tensor = 0;
+    for (int32_t t : order) {
+        tab->h_seg_first[2 * (size_t)t] = (int32_t)tab->h_segments.size();
         int64_t b = offsets[t];
         const int64_t e = offsets[t + 1];
         while (b < e) {
@@ -265,15 +276,12 @@ void build_segments(const int64_t* offsets, int32_t num_tensors, int seg_len, Se
             tab->h_segments.push_back(Segment{b, (int32_t)(next - b), t});
             b = next;
         }
-    }
-    tab->h_seg_first[num_tensors] = (int32_t)tab->h_segments.size();
-    tab->num_segments = (int32_t)tab->h_segments.size();
-    tab->max_segments_per_tensor = 0;
-    for (int32_t t = 0; t < num_tensors; ++t) {
-        const int32_t n = tab->h_seg_first[t + 1] - tab->h_seg_first[t];
+        tab->h_seg_first[2 * (size_t)t + 1] = (int32_t)tab->h_segments.size();
+        const int32_t n = tab->h_seg_first[2 * (size_t)t + 1] - tab->h_seg_first[2 * (size_t)t];
         if (n > tab->max_segments_per_tensor)
             tab->max_segments_per_tensor = n;
     }
+    tab->num_segments = (int32_t)tab->h_segments.size();
 }
 
 adasum_status_t get_segment_table(const int64_t* offsets, int32_t num_tensors, int seg_len,
@@ -331,21 +339,6 @@ adasum_status_t get_segment_table(const int64_t* offsets, int32_t num_tensors, i
 
 // ---- launches ----------------------------------------------------------------------------------
 
-int multiprocessor_count()
-{
-    static int cached[64] = {};
-    int device = 0;
-    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64)
-        return 148;
-    if (cached[device] == 0) {
-        int n = 0;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || n <= 0)
-            n = 148;
-        cached[device] = n;
-    }
-    return cached[device];
-}
-
 // Opt a kernel in to `bytes` of dynamic shared memory, once per device.
 template <typename Kernel>
 cudaError_t allow_dynamic_smem(Kernel kernel, size_t bytes, bool (&configured)[64])
@@ -370,7 +363,7 @@ cudaError_t launch_gram(GramKind kind, const OperandTable& ops, int operands, in
                         const SegmentTable& tab, float* partials, int groups_total, int group_base,
                         const FinishArgs& fin, cudaStream_t stream)
 {
-    if constexpr (R >= 16) {
+    if constexpr (R >= 8) {
         if (kind == GRAM_MMA) {
             if constexpr (R <= 32 || sizeof(T) == 2) {
                 constexpr size_t smem = mma_smem_bytes<T, R>();
@@ -450,8 +443,8 @@ template <typename T, int R>
 adasum_status_t run_level_typed(const LevelArgs& a)
 {
     constexpr int kGroupsPerLaunch = kMaxOperandsPerLaunch / R;
-    // radix <= 16: the last block of every (tensor, group) in pass 1 also derives the weights
-    const bool fused_finish = R <= 16 && a.counters != nullptr;
+    // the last block of every (tensor, group) in pass 1 also derives the weights
+    const bool fused_finish = a.counters != nullptr;
     const FinishArgs fin{a.gram_tab->d_seg_first, fused_finish ? a.counters : nullptr, a.weights};
     // pass 1
     for (int g0 = 0; g0 < a.groups; g0 += kGroupsPerLaunch) {
@@ -522,10 +515,8 @@ int launches_of(const LevelPlan& plan, int n_workers, uint32_t flags)
         const int per_launch = kMaxOperandsPerLaunch / plan.level[l].radix;
         const int batches = (plan.level[l].groups + per_launch - 1) / per_launch;
         n += 2 * batches;
-        if (plan.level[l].radix >= 32)
-            n += 2;                                     // gram_finish + tree_weights
-        else if (flags & ADASUM_FLAG_SEPARATE_FINISH)
-            n += 1;                                     // gram_finish (otherwise done inside pass 1)
+        if (flags & ADASUM_FLAG_SEPARATE_FINISH)        // otherwise done inside pass 1
+            n += plan.level[l].radix >= 32 ? 2 : 1;     // gram_finish (+ tree_weights)
     }
     return n;
 }
@@ -687,7 +678,7 @@ constexpr int32_t kNoallocMaxTensors = ADASUM_NOALLOC_MAX_TENSORS;
 constexpr int kNoallocSegLen = 8192;
 constexpr int64_t kNoallocMaxSegments = kNoallocMaxElems / kNoallocSegLen + 2 * (int64_t)kNoallocMaxTensors + 1;
 constexpr size_t kNoallocSegBytes = ((size_t)kNoallocMaxSegments * sizeof(Segment) + 255) / 256 * 256;
-constexpr size_t kNoallocFirstBytes = ((size_t)(kNoallocMaxTensors + 1) * sizeof(int32_t) + 255) / 256 * 256;
+constexpr size_t kNoallocFirstBytes = ((size_t)(2 * kNoallocMaxTensors + 2) * sizeof(int32_t) + 255) / 256 * 256;
 constexpr size_t kNoallocPartialBytes = ((size_t)kNoallocMaxSegments * gram_entries(2) * sizeof(float) + 255) / 256 * 256;
 constexpr size_t kNoallocWeightBytes = ((size_t)kNoallocMaxTensors * 2 * sizeof(float) + 255) / 256 * 256;
 constexpr size_t kNoallocScratchBytes = kNoallocSegBytes + kNoallocFirstBytes + kNoallocPartialBytes + kNoallocWeightBytes;

@@ -14,7 +14,7 @@
 //   weighted_sum   stream the operands a second time; out = sum_i weight_i x_i.
 //
 // The Gram matrix of a group is a dense contraction X X^T (R x P times P x R).  For R <= 8 it is
-// cheap enough for the fp32 pipes (gram_partial_kernel); for R >= 16 it runs on the tensor cores (gram_partial_mma_kernel): fp16 / bf16 products are exact in
+// cheap enough for the fp32 pipes (gram_partial_kernel); for R >= 8 it runs on the tensor cores (gram_partial_mma_kernel): fp16 / bf16 products are exact in
 // the fp32 accumulator, fp32 inputs are split into two tf32 terms (three products).
 //
 // The kernels never wait on one another and use no floating-point atomics, so results are
@@ -145,15 +145,15 @@ __device__ __forceinline__ void split_segment(int64_t begin, int64_t end, int64_
 
 // ---- finishing a group inside pass 1 -----------------------------------------------------------
 //
-// For radix <= 16 the block that writes the LAST per-segment partial matrix of a (tensor, group)
-// also adds up all of that tensor's partials and derives the leaf weights, so no separate launch
+// The block that writes the LAST per-segment partial matrix of a (tensor, group) also adds up all
+// of that tensor's partials and derives the leaf weights, so no separate launch
 // (and no idle GPU while a small kernel runs) separates pass 1 from pass 2.  "Last" is decided by
 // an integer ticket counter per (tensor, group); the sums themselves are taken in segment order,
 // so the result does not depend on which block happens to be last.  The counter is returned to
 // zero by that block.  counters == nullptr switches the mechanism off (the caller then launches
 // gram_finish_kernel).
 struct FinishArgs {
-    const int32_t* seg_first;   // num_tensors + 1: first segment of every tensor
+    const int32_t* seg_first;   // [2 t], [2 t + 1]: first and one-past-last segment of tensor t
     int* counters;              // [tensor][group], zero on entry
     float* weights;             // [tensor][group][R]
 };
@@ -172,7 +172,7 @@ __device__ __forceinline__ void finish_if_last(const FinishArgs& fin, const floa
     __shared__ int is_last;
     __threadfence();                       // this block's partial is visible device-wide ...
     __syncthreads();
-    const int s0 = fin.seg_first[tensor], s1 = fin.seg_first[tensor + 1];
+    const int s0 = fin.seg_first[2 * tensor], s1 = fin.seg_first[2 * tensor + 1];
     if (threadIdx.x == 0) {
         int* counter = fin.counters + (int64_t)tensor * groups_total + group;
         const int ticket = atomicAdd(counter, 1);      // ... before its ticket is drawn
@@ -287,8 +287,7 @@ gram_partial_kernel(const __grid_constant__ OperandTable ops, int operands,
             s += warp_sums[w][k];
         dst[k] = s;
     }
-    if constexpr (R <= 16)
-        finish_if_last<R>(fin, partials, seg.tensor, group_base + blockIdx.y, groups_total, members);
+    finish_if_last<R>(fin, partials, seg.tensor, group_base + blockIdx.y, groups_total, members);
 }
 
 // ---- asynchronous copies into shared memory ----------------------------------------------------
@@ -322,12 +321,12 @@ template <int R>
 __host__ __device__ constexpr int mma_upper_blocks()     // 16 x 8 blocks that touch the upper triangle
 {
     int n = 0;
-    for (int mb = 0; mb < R / 16; ++mb)
+    for (int mb = 0; mb < (R + 15) / 16; ++mb)     // R = 8: half a row block, rows 8..15 are zero
         n += R / 8 - 2 * mb;
     return n;
 }
 template <int R>
-__host__ __device__ constexpr int mma_all_blocks() { return (R / 16) * (R / 8); }
+__host__ __device__ constexpr int mma_all_blocks() { return ((R + 15) / 16) * (R / 8); }
 
 // Index of block (mb, nb), nb >= 2 mb, in the upper-block numbering.
 template <int R>
@@ -465,6 +464,8 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
     constexpr int E = gram_entries(R);
     constexpr int V = Element<T>::kVec;          // elements per 16-byte vector
     constexpr int RB = R / 8;                    // blocks of 8 rows
+    constexpr int MB = (R + 15) / 16;            // blocks of 16 rows (R = 8: the upper half is zero)
+    constexpr int RBP = 2 * MB;                  // row blocks the fragments are indexed with
     constexpr int UBLK = mma_upper_blocks<R>();
     constexpr bool SPLIT = sizeof(T) == 4;
     constexpr int CBLK = SPLIT ? mma_all_blocks<R>() : 0;
@@ -477,7 +478,6 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
     constexpr int ROWS_PER_PASS = kThreads / PIECES_PER_ROW;     // piece i of a thread is in row row0 + i * this
     static_assert(DEPTH * kWarps * 64 == ROW_BYTES, "a tile row is split evenly among the warps");
     static_assert(PIECES_PER_ROW % 32 == 0 && kThreads % PIECES_PER_ROW == 0, "a warp copies within one row");
-    static_assert(ROWS_PER_PASS % 2 == 0, "all pieces of a thread have the same row parity");
     extern __shared__ __align__(128) unsigned char stage_mem[];
 
     const Segment seg = segments[blockIdx.x];
@@ -493,7 +493,11 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
     // ---- copy side: piece i of this thread is (row0 + i * ROWS_PER_PASS, col0) of the tile
     const uint32_t smem_base = static_cast<uint32_t>(__cvta_generic_to_shared(stage_mem));
     const int row0 = threadIdx.x / PIECES_PER_ROW, col0 = threadIdx.x % PIECES_PER_ROW;
-    const uint32_t copy_off = row0 * ROW_BYTES + (((col0 >> 2) ^ (row0 & 1)) << 6) + ((col0 & 3) << 4);
+    // byte offset of piece i inside a tile (the swizzle depends on the row's parity)
+    auto copy_off = [&](int i) -> uint32_t {
+        const int row = row0 + i * ROWS_PER_PASS;
+        return row * ROW_BYTES + (((col0 >> 2) ^ (row & 1)) << 6) + ((col0 & 3) << 4);
+    };
     const T* copy_src[PIECES];     // row pointer + this thread's column; rows beyond the members alias row 0
 #pragma unroll
     for (int i = 0; i < PIECES; ++i) {
@@ -504,19 +508,19 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
 
     auto issue = [&](int tile, int stage) {
         if (tile < ntiles) {
-            const uint32_t dst = smem_base + stage * kMmaTileBytes + copy_off;
+            const uint32_t dst = smem_base + stage * kMmaTileBytes;
             const int64_t tile_elem0 = k0 + (int64_t)tile * TILE_ELEMS;
             if (VEC && full_group && tile_elem0 >= begin && tile_elem0 + TILE_ELEMS <= end) {
 #pragma unroll
                 for (int i = 0; i < PIECES; ++i)
-                    cp_async_16B_shared(dst + i * ROWS_PER_PASS * ROW_BYTES, copy_src[i] + tile_elem0);
+                    cp_async_16B_shared(dst + copy_off(i), copy_src[i] + tile_elem0);
             } else {
                 // ragged tile, partial group or unaligned buffers: test every piece
                 const int64_t e0 = tile_elem0 + (int64_t)col0 * V;
                 const bool whole = VEC && e0 >= begin && e0 + V <= end;
 #pragma unroll
                 for (int i = 0; i < PIECES; ++i) {
-                    const uint32_t slot = dst + i * ROWS_PER_PASS * ROW_BYTES;
+                    const uint32_t slot = dst + copy_off(i);
                     if (row0 + i * ROWS_PER_PASS >= members)
                         store_shared_16B(slot, make_uint4(0u, 0u, 0u, 0u));
                     else if (whole)
@@ -569,16 +573,17 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
         if constexpr (!SPLIT) {
 #pragma unroll
             for (int d = 0; d < DEPTH; ++d) {
-                uint32_t w[RB][4];
+                uint32_t w[RBP][4];
 #pragma unroll
-                for (int rb = 0; rb < RB; ++rb) {
-                    const uint4 v = load_shared_16B(src_stage + chunk_off[d] + rb * 8 * ROW_BYTES);
+                for (int rb = 0; rb < RBP; ++rb) {
+                    const uint4 v = rb < RB ? load_shared_16B(src_stage + chunk_off[d] + rb * 8 * ROW_BYTES)
+                                            : make_uint4(0u, 0u, 0u, 0u);
                     w[rb][0] = v.x; w[rb][1] = v.y; w[rb][2] = v.z; w[rb][3] = v.w;
                 }
 #pragma unroll
                 for (int step = 0; step < 2; ++step) {
 #pragma unroll
-                    for (int mb = 0; mb < R / 16; ++mb)
+                    for (int mb = 0; mb < MB; ++mb)
 #pragma unroll
                         for (int nb = 2 * mb; nb < RB; ++nb)
                             mma_step<T>(acc[mma_upper_index<R>(mb, nb)], w[2 * mb][2 * step], w[2 * mb + 1][2 * step],
@@ -600,10 +605,11 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
                     tile_c[b][r] = 0.0f;
 #pragma unroll
             for (int d = 0; d < DEPTH; ++d) {
-                uint32_t hi[RB][4], lo[RB][4];
+                uint32_t hi[RBP][4], lo[RBP][4];
 #pragma unroll
-                for (int rb = 0; rb < RB; ++rb) {
-                    const uint4 v = load_shared_16B(src_stage + chunk_off[d] + rb * 8 * ROW_BYTES);
+                for (int rb = 0; rb < RBP; ++rb) {
+                    const uint4 v = rb < RB ? load_shared_16B(src_stage + chunk_off[d] + rb * 8 * ROW_BYTES)
+                                            : make_uint4(0u, 0u, 0u, 0u);
                     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
@@ -616,7 +622,7 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
 #pragma unroll
                 for (int step = 0; step < 2; ++step) {
 #pragma unroll
-                    for (int mb = 0; mb < R / 16; ++mb) {
+                    for (int mb = 0; mb < MB; ++mb) {
 #pragma unroll
                         for (int nb = 0; nb < RB; ++nb) {
                             if (nb >= 2 * mb)
@@ -679,8 +685,7 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
         }
         dst[gram_index(R, i, j)] = v;
     }
-    if constexpr (R <= 16)
-        finish_if_last<R>(fin, partials, seg.tensor, group_base + blockIdx.y, groups_total, members);
+    finish_if_last<R>(fin, partials, seg.tensor, group_base + blockIdx.y, groups_total, members);
 }
 
 // ---- coefficients: the binary tree evaluated on a Gram matrix ---------------------------------
@@ -754,34 +759,45 @@ __device__ void tree_weights_from_gram(const double* gram, int members, float* _
 }
 
 // The tensor's partial matrices (segments seg_begin .. seg_end) added in fp64 by one block of
-// kThreads threads, then the tree.  With Q = kThreads / E slices, slice q takes segments
-// q, q + Q, ... in order and the slices are added in order.  Partials were written by other
-// blocks of the running kernel, hence the L2 loads.
+// kThreads threads, then the tree.  Small groups: with Q = kThreads / E slices, slice q takes
+// segments q, q + Q, ... in order and the slices are added in order.  Partials were written by
+// other blocks of the running kernel, hence the L2 loads.
 template <int R>
 __device__ void finish_group_in_block(const float* partials, int seg_begin, int seg_end, int group,
                                       int groups_total, int members, float* weights_dst)
 {
     constexpr int E = gram_entries(R);
-    static_assert(E <= kThreads, "one thread per entry");
-    constexpr int Q = kThreads / E;
-    __shared__ double slice_sum[kThreads];
     __shared__ double gram[E];
-    const int q = threadIdx.x / E, kk = threadIdx.x - q * E;
-    if (q < Q) {
-        const float* src = partials + (int64_t)group * E + kk;
-        const int64_t stride = (int64_t)groups_total * E;
-        double s = 0.0;
+    const int64_t stride = (int64_t)groups_total * E;
+    if constexpr (E <= kThreads) {
+        constexpr int Q = kThreads / E;
+        __shared__ double slice_sum[kThreads];
+        const int q = threadIdx.x / E, kk = threadIdx.x - q * E;
+        if (q < Q) {
+            const float* src = partials + (int64_t)group * E + kk;
+            double s = 0.0;
 #pragma unroll 8
-        for (int seg = seg_begin + q; seg < seg_end; seg += Q)
-            s += (double)__ldcg(src + seg * stride);
-        slice_sum[q * E + kk] = s;
-    }
-    __syncthreads();
-    if (threadIdx.x < E) {
-        double s = slice_sum[threadIdx.x];
-        for (int qq = 1; qq < Q; ++qq)
-            s += slice_sum[qq * E + threadIdx.x];
-        gram[threadIdx.x] = s;
+            for (int seg = seg_begin + q; seg < seg_end; seg += Q)
+                s += (double)__ldcg(src + seg * stride);
+            slice_sum[q * E + kk] = s;
+        }
+        __syncthreads();
+        if (threadIdx.x < E) {
+            double s = slice_sum[threadIdx.x];
+            for (int qq = 1; qq < Q; ++qq)
+                s += slice_sum[qq * E + threadIdx.x];
+            gram[threadIdx.x] = s;
+        }
+    } else {
+        // wide groups: every thread owns several entries and adds their partials in segment order
+        for (int k = threadIdx.x; k < E; k += kThreads) {
+            const float* src = partials + (int64_t)group * E + k;
+            double s = 0.0;
+#pragma unroll 8
+            for (int seg = seg_begin; seg < seg_end; ++seg)
+                s += (double)__ldcg(src + seg * stride);
+            gram[k] = s;
+        }
     }
     __syncthreads();
     tree_weights_from_gram<R>(gram, members, weights_dst);
@@ -819,7 +835,7 @@ gram_finish_kernel(const float* __restrict__ partials, const int32_t* __restrict
 
     const int Q = blockDim.x / EPB;
     const int tensor = blockIdx.x, group = blockIdx.y, groups = gridDim.y;
-    const int s0 = seg_first[tensor], s1 = seg_first[tensor + 1];
+    const int s0 = seg_first[2 * tensor], s1 = seg_first[2 * tensor + 1];
     const int q = threadIdx.x / EPB, kk = threadIdx.x - q * EPB;
     const int k = blockIdx.z * EPB + kk;
     if (q < Q) {
