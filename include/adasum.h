@@ -83,9 +83,16 @@ typedef enum {
  *   bit 17       ADASUM_FLAG_SEPARATE_FINISH: add up the per-segment Gram matrices and derive
  *                the leaf weights in a kernel of their own at every level, instead of inside
  *                the first pass; for comparison and debugging
+ *   bit 18       ADASUM_FLAG_LINEAR_ORDER: a DIFFERENT result, the sequential recursion of
+ *                Section 3.4, Adasum(g[0..n+1]) = Adasum(Adasum(g[0..n]), g[n+1]) (the order of
+ *                the paper's ring implementation), instead of the binary tree.  The running
+ *                result depends on all earlier workers, so the whole reduce is one level whose
+ *                Gram matrix covers every worker: n_workers <= 32 for fp32 inputs, <= 64 for
+ *                fp16 / bf16; the radix fields must be 0.  Otherwise ADASUM_ERR_ARG.
  */
 #define ADASUM_FLAG_SIMPLE_KERNELS (1u << 16)
 #define ADASUM_FLAG_SEPARATE_FINISH (1u << 17)
+#define ADASUM_FLAG_LINEAR_ORDER (1u << 18)
 #define ADASUM_RADIX_AUTO 0u
 #define ADASUM_FLAGS_RADIX(first, later) (((uint32_t)(first) & 0xffu) | (((uint32_t)(later) & 0xffu) << 8))
 
@@ -131,6 +138,24 @@ adasum_status_t adasum_reduce(const void* const* grads, const int64_t* tensor_of
                               int32_t num_tensors, int32_t n_workers, adasum_dtype_t dtype,
                               float* out, void* workspace, size_t workspace_bytes,
                               uint32_t flags, void* stream);
+
+/*
+ * adasum_reduce that also returns the per-tensor orthogonality measure of Section 3.6,
+ *
+ *     orthogonality[t] = |Adasum(g_1 .. g_N)|^2 / sum_i |g_i|^2      (tensor t),
+ *
+ * which is 1 for mutually orthogonal gradients and 1/N for identical ones.  It costs nothing
+ * extra: both norms fall out of the Gram matrices the reduce forms anyway.
+ *
+ *   orthogonality   device, num_tensors floats, 4-byte aligned, or NULL (then this is
+ *                   adasum_reduce).  NaN for a tensor that has no elements or whose gradients
+ *                   are all zero.  Needs n_workers >= 2 (ADASUM_ERR_ARG otherwise).
+ * Everything else as for adasum_reduce, including the workspace size.
+ */
+adasum_status_t adasum_reduce_ex(const void* const* grads, const int64_t* tensor_offsets,
+                                 int32_t num_tensors, int32_t n_workers, adasum_dtype_t dtype,
+                                 float* out, float* orthogonality, void* workspace,
+                                 size_t workspace_bytes, uint32_t flags, void* stream);
 
 /*
  * One application of the operator per tensor, out = Adasum(a, b) (Section 3; the "partial dot

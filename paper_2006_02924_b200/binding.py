@@ -23,6 +23,7 @@ if not os.path.exists(LIB_PATH):
 _lib = ctypes.CDLL(LIB_PATH)
 
 ADASUM_F32, ADASUM_F16, ADASUM_BF16 = 0, 1, 2
+ADASUM_FLAG_SIMPLE_KERNELS, ADASUM_FLAG_SEPARATE_FINISH, ADASUM_FLAG_LINEAR_ORDER = 1 << 16, 1 << 17, 1 << 18
 ADASUM_OK = 0
 ADASUM_MAX_WORKERS = 4096
 ADASUM_MAX_LEVELS = 12
@@ -41,6 +42,10 @@ _lib.adasum_reduce.restype = ctypes.c_int
 _lib.adasum_reduce.argtypes = [ctypes.POINTER(ctypes.c_void_p), _i64p, ctypes.c_int32, ctypes.c_int32,
                                ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t,
                                ctypes.c_uint32, ctypes.c_void_p]
+_lib.adasum_reduce_ex.restype = ctypes.c_int
+_lib.adasum_reduce_ex.argtypes = [ctypes.POINTER(ctypes.c_void_p), _i64p, ctypes.c_int32, ctypes.c_int32,
+                                  ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t,
+                                  ctypes.c_uint32, ctypes.c_void_p]
 _lib.adasum_pair.restype = ctypes.c_int
 _lib.adasum_pair.argtypes = [ctypes.c_void_p, ctypes.c_void_p, _i64p, ctypes.c_int32, ctypes.c_int,
                              ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_uint32,
@@ -140,6 +145,31 @@ def adasum_reduce(grads, tensor_offsets=None, out=None, workspace=None, flags: i
     if status != ADASUM_OK:
         raise AdasumError(status)
     return out
+
+
+def adasum_reduce_ex(grads, tensor_offsets=None, out=None, orthogonality=None, workspace=None, flags: int = 0,
+                     stream=None):
+    """``adasum_reduce_ex`` of the C ABI: the reduce plus the per-tensor orthogonality measure.
+    Returns ``(out, orthogonality)`` (both allocated here if not given)."""
+    grads = list(grads)
+    first = grads[0]
+    total = first.numel()
+    offs = _offsets_array(tensor_offsets, total)
+    num_tensors = offs.size - 1
+    if out is None:
+        out = torch.empty(total, dtype=torch.float32, device=first.device)
+    if orthogonality is None:
+        orthogonality = torch.empty(max(num_tensors, 1), dtype=torch.float32, device=first.device)[:num_tensors]
+    need = adasum_workspace_bytes(total, num_tensors, len(grads), first.dtype, flags)
+    workspace, ws_ptr, ws_bytes = _workspace(workspace, need, first.device)
+    ptrs = (ctypes.c_void_p * len(grads))(*[g.data_ptr() for g in grads])
+    with torch.cuda.device(first.device):
+        status = _lib.adasum_reduce_ex(ptrs, offs.ctypes.data_as(_i64p), num_tensors, len(grads),
+                                       _dtype_code(first.dtype), out.data_ptr(), orthogonality.data_ptr(), ws_ptr,
+                                       ws_bytes, int(flags), _stream_handle(stream))
+    if status != ADASUM_OK:
+        raise AdasumError(status)
+    return out, orthogonality
 
 
 def adasum_pair(a, b, tensor_offsets=None, out=None, workspace=None, flags: int = 0, stream=None):

@@ -134,7 +134,7 @@ struct LevelPlan {
 bool plan_levels(int n_workers, adasum_dtype_t dtype, uint32_t flags, LevelPlan* plan)
 {
     const int first = (int)(flags & 0xffu), later_flag = (int)((flags >> 8) & 0xffu);
-    if ((flags >> 18) != 0)
+    if ((flags >> 19) != 0)
         return false;
     if (first != 0 && (!valid_radix(first) || first > max_radix_for(dtype)))
         return false;
@@ -146,6 +146,21 @@ bool plan_levels(int n_workers, adasum_dtype_t dtype, uint32_t flags, LevelPlan*
     if (later > max_radix_for(ADASUM_F32))
         later = max_radix_for(ADASUM_F32);      // intermediates are fp32
     const int cap_auto = (flags & ADASUM_FLAG_SIMPLE_KERNELS) ? 16 : 64;
+    if (flags & ADASUM_FLAG_LINEAR_ORDER) {
+        // the running result of the sequential recursion is a combination of ALL earlier leaves:
+        // one level whose Gram matrix covers every worker
+        if (first != 0 || later_flag != 0)
+            return false;
+        const int radix = pow2_ceil(n_workers < 2 ? 2 : n_workers);
+        if (radix > max_radix_for(dtype) || radix > cap_auto)
+            return false;
+        plan->num_levels = 0;
+        if (n_workers > 1) {
+            plan->num_levels = 1;
+            plan->level[0] = Level{radix, n_workers, 1};
+        }
+        return true;
+    }
     int m = n_workers;
     plan->num_levels = 0;
     while (m > 1) {
@@ -177,8 +192,9 @@ int64_t segment_bound(int64_t total, int32_t num_tensors, int seg_len)
 }
 
 struct Layout {
-    size_t partials = 0, weights = 0, gram64 = 0, counters = 0, buffer[2] = {0, 0};
-    size_t partials_bytes = 0, weights_bytes = 0, gram64_bytes = 0, counters_bytes = 0, buffer_bytes[2] = {0, 0};
+    size_t partials = 0, weights = 0, gram64 = 0, counters = 0, leaf_sums = 0, buffer[2] = {0, 0};
+    size_t partials_bytes = 0, weights_bytes = 0, gram64_bytes = 0, counters_bytes = 0, leaf_sums_bytes = 0,
+           buffer_bytes[2] = {0, 0};
     int64_t padded_elems = 0;
     size_t total = 0;
 };
@@ -221,6 +237,10 @@ Layout make_layout(const LevelPlan& plan, int64_t total_elems, int32_t num_tenso
     off += align_up(lay.gram64_bytes);
     lay.counters = off;
     off += align_up(lay.counters_bytes);
+    if (plan.num_levels > 0)
+        lay.leaf_sums_bytes = (size_t)(num_tensors > 0 ? num_tensors : 1) * plan.level[0].groups * sizeof(double);
+    lay.leaf_sums = off;
+    off += align_up(lay.leaf_sums_bytes);
     lay.buffer[0] = off;
     off += align_up(lay.buffer_bytes[0]);
     lay.buffer[1] = off;
@@ -404,17 +424,18 @@ void launch_wsum(const OperandTable& ops, int operands, int groups_here, const S
 
 template <int R>
 cudaError_t launch_weights(const float* partials, const SegmentTable& tab, int32_t num_tensors, int operands,
-                           int groups, double* gram64, float* weights, cudaStream_t stream, int* launches)
+                           int groups, double* gram64, float* weights, const TreeOptions& opt, cudaStream_t stream,
+                           int* launches)
 {
     dim3 grid((unsigned)num_tensors, (unsigned)groups, (unsigned)tree_entry_blocks(R));
     // wide blocks only pay off when some tensor has many per-segment partials to add
     const int threads = tab.max_segments_per_tensor > 64 ? kTreeThreadsMax : 256;
     gram_finish_kernel<R><<<grid, threads, threads * sizeof(double), stream>>>(partials, tab.d_seg_first, operands,
-                                                                                gram64, weights);
+                                                                                gram64, weights, opt);
     *launches = 1;
     if constexpr (tree_entry_blocks(R) > 1) {
         dim3 grid2((unsigned)num_tensors, (unsigned)groups);
-        tree_weights_kernel<R><<<grid2, kThreads, 0, stream>>>(gram64, operands, weights);
+        tree_weights_kernel<R><<<grid2, kThreads, 0, stream>>>(gram64, operands, weights, opt);
         *launches = 2;
     }
     return cudaSuccess;
@@ -430,6 +451,7 @@ struct LevelArgs {
     int32_t num_tensors;
     float* partials;
     int* counters;      // ticket counters for finishing inside pass 1, or nullptr
+    TreeOptions tree;
     double* gram64;
     float* weights;
     float* dst;
@@ -445,7 +467,7 @@ adasum_status_t run_level_typed(const LevelArgs& a)
     constexpr int kGroupsPerLaunch = kMaxOperandsPerLaunch / R;
     // the last block of every (tensor, group) in pass 1 also derives the weights
     const bool fused_finish = a.counters != nullptr;
-    const FinishArgs fin{a.gram_tab->d_seg_first, fused_finish ? a.counters : nullptr, a.weights};
+    const FinishArgs fin{a.gram_tab->d_seg_first, fused_finish ? a.counters : nullptr, a.weights, a.tree};
     // pass 1
     for (int g0 = 0; g0 < a.groups; g0 += kGroupsPerLaunch) {
         const int groups_here = a.groups - g0 < kGroupsPerLaunch ? a.groups - g0 : kGroupsPerLaunch;
@@ -465,7 +487,7 @@ adasum_status_t run_level_typed(const LevelArgs& a)
     if (!fused_finish) {
         int weight_launches = 0;
         ADASUM_CUDA_CHECK(launch_weights<R>(a.partials, *a.gram_tab, a.num_tensors, a.operands, a.groups,
-                                            a.gram64, a.weights, a.stream, &weight_launches));
+                                            a.gram64, a.weights, a.tree, a.stream, &weight_launches));
         profile_mark(a.stream, ADASUM_KERNEL_TREE_WEIGHTS, a.level, R, false);
     }
     // pass 2
@@ -549,18 +571,22 @@ adasum_status_t check_common(const int64_t* offsets, int32_t num_tensors, int32_
 }
 
 adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, int32_t num_tensors,
-                            int32_t n_workers, adasum_dtype_t dtype, float* out, void* workspace,
-                            size_t workspace_bytes, uint32_t flags, cudaStream_t stream)
+                            int32_t n_workers, adasum_dtype_t dtype, float* out, float* orthogonality,
+                            void* workspace, size_t workspace_bytes, uint32_t flags, cudaStream_t stream)
 {
     g_error[0] = '\0';
     if (!grads)
         return fail(ADASUM_ERR_NULL, "grads is NULL");
+    if (orthogonality && n_workers < 2)
+        return fail(ADASUM_ERR_ARG, "the orthogonality measure needs at least two workers");
+    if (reinterpret_cast<uintptr_t>(orthogonality) & 3u)
+        return fail(ADASUM_ERR_ARG, "orthogonality is not 4-byte aligned");
     adasum_status_t st = check_common(offsets, num_tensors, n_workers, dtype);
     if (st != ADASUM_OK)
         return st;
     LevelPlan plan;
     if (!plan_levels(n_workers, dtype, flags, &plan))
-        return fail(ADASUM_ERR_ARG, "invalid flags 0x%x", flags);
+        return fail(ADASUM_ERR_ARG, "invalid flags 0x%x for %d workers of this dtype", flags, n_workers);
     const int64_t total = offsets[num_tensors];
     if (total == 0)
         return ADASUM_OK;
@@ -614,6 +640,8 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     const bool separate_finish = (flags & ADASUM_FLAG_SEPARATE_FINISH) != 0;
     if (!separate_finish && lay.counters_bytes > 0)     // the workspace arrives with unknown contents
         ADASUM_CUDA_CHECK(cudaMemsetAsync(ws + lay.counters, 0, lay.counters_bytes, stream));
+    if (orthogonality && num_tensors > 0)               // NaN for tensors without elements
+        ADASUM_CUDA_CHECK(cudaMemsetAsync(orthogonality, 0xff, sizeof(float) * (size_t)num_tensors, stream));
     std::vector<const void*> operand_ptrs(grads, grads + n_workers);
     for (int l = 0; l < plan.num_levels; ++l) {
         const Level& lv = plan.level[l];
@@ -640,6 +668,12 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         a.weights = reinterpret_cast<float*>(ws + lay.weights);
         a.gram64 = reinterpret_cast<double*>(ws + lay.gram64);
         a.counters = separate_finish ? nullptr : reinterpret_cast<int*>(ws + lay.counters);
+        a.tree.linear = (flags & ADASUM_FLAG_LINEAR_ORDER) ? 1 : 0;
+        a.tree.level_is_first = l == 0;
+        a.tree.level_is_last = l + 1 == plan.num_levels;
+        a.tree.groups_first = plan.level[0].groups;
+        a.tree.leaf_norm_sums = orthogonality ? reinterpret_cast<double*>(ws + lay.leaf_sums) : nullptr;
+        a.tree.orthogonality = orthogonality;
         a.dst = last ? out : reinterpret_cast<float*>(ws + lay.buffer[l & 1]);
         a.dst_stride = last ? 0 : lay.padded_elems;
         a.vec = vec;
@@ -711,13 +745,14 @@ template <typename T>
 cudaError_t noalloc_launch(bool vec, const OperandTable& ops, const SegmentTable& tab, int32_t num_tensors,
                            float* partials, float* weights, float* out, cudaStream_t stream)
 {
-    const FinishArgs no_fusion{nullptr, nullptr, nullptr};
+    const TreeOptions plain_tree{0, 1, 1, 1, nullptr, nullptr};
+    const FinishArgs no_fusion{nullptr, nullptr, nullptr, plain_tree};
     cudaError_t err = vec ? launch_gram<T, 2, true>(GRAM_SIMPLE, ops, 2, 1, tab, partials, 1, 0, no_fusion, stream)
                           : launch_gram<T, 2, false>(GRAM_SIMPLE, ops, 2, 1, tab, partials, 1, 0, no_fusion, stream);
     if (err != cudaSuccess)
         return err;
     int weight_launches = 0;
-    err = launch_weights<2>(partials, tab, num_tensors, 2, 1, nullptr, weights, stream, &weight_launches);
+    err = launch_weights<2>(partials, tab, num_tensors, 2, 1, nullptr, weights, plain_tree, stream, &weight_launches);
     if (err != cudaSuccess)
         return err;
     if (vec)
@@ -839,7 +874,16 @@ adasum_status_t adasum_reduce(const void* const* grads, const int64_t* tensor_of
                               float* out, void* workspace, size_t workspace_bytes, uint32_t flags,
                               void* stream)
 {
-    return adasum::reduce_impl(grads, tensor_offsets, num_tensors, n_workers, dtype, out, workspace,
+    return adasum::reduce_impl(grads, tensor_offsets, num_tensors, n_workers, dtype, out, nullptr, workspace,
+                               workspace_bytes, flags, static_cast<cudaStream_t>(stream));
+}
+
+adasum_status_t adasum_reduce_ex(const void* const* grads, const int64_t* tensor_offsets,
+                                 int32_t num_tensors, int32_t n_workers, adasum_dtype_t dtype,
+                                 float* out, float* orthogonality, void* workspace, size_t workspace_bytes,
+                                 uint32_t flags, void* stream)
+{
+    return adasum::reduce_impl(grads, tensor_offsets, num_tensors, n_workers, dtype, out, orthogonality, workspace,
                                workspace_bytes, flags, static_cast<cudaStream_t>(stream));
 }
 
@@ -848,7 +892,7 @@ adasum_status_t adasum_pair(const void* a, const void* b, const int64_t* tensor_
                             size_t workspace_bytes, uint32_t flags, void* stream)
 {
     const void* grads[2] = {a, b};
-    return adasum::reduce_impl(grads, tensor_offsets, num_tensors, 2, dtype, out, workspace,
+    return adasum::reduce_impl(grads, tensor_offsets, num_tensors, 2, dtype, out, nullptr, workspace,
                                workspace_bytes, flags, static_cast<cudaStream_t>(stream));
 }
 

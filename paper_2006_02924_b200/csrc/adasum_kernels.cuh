@@ -152,15 +152,27 @@ __device__ __forceinline__ void split_segment(int64_t begin, int64_t end, int64_
 // so the result does not depend on which block happens to be last.  The counter is returned to
 // zero by that block.  counters == nullptr switches the mechanism off (the caller then launches
 // gram_finish_kernel).
+// What the coefficient step produces besides the leaf weights.
+struct TreeOptions {
+    int linear;               // 1: the sequential recursion Adasum(Adasum(g[0..n]), g[n+1]) of Section 3.4
+                              //    instead of the binary tree (single-level plans only)
+    int level_is_first;       // this level's operands are the workers' gradients
+    int level_is_last;        // this level's single group produces the result
+    int groups_first;         // number of groups of the first level
+    double* leaf_norm_sums;   // [tensor][groups_first]: sum of the leaves' squared norms, or nullptr
+    float* orthogonality;     // [tensor]: |result|^2 / sum_i |g_i|^2 (Section 3.6), or nullptr
+};
+
 struct FinishArgs {
     const int32_t* seg_first;   // [2 t], [2 t + 1]: first and one-past-last segment of tensor t
     int* counters;              // [tensor][group], zero on entry
     float* weights;             // [tensor][group][R]
+    TreeOptions tree;
 };
 
 template <int R>
-__device__ void finish_group_in_block(const float* partials, int seg_begin, int seg_end, int group,
-                                      int groups_total, int members, float* weights_dst);
+__device__ void finish_group_in_block(const float* partials, int seg_begin, int seg_end, int tensor, int group,
+                                      int groups_total, int members, float* weights_dst, const TreeOptions& opt);
 
 // Called by every thread of the block after its partial matrix has been written.
 template <int R>
@@ -183,8 +195,8 @@ __device__ __forceinline__ void finish_if_last(const FinishArgs& fin, const floa
     __syncthreads();
     if (is_last) {
         __threadfence();
-        finish_group_in_block<R>(partials, s0, s1, group, groups_total, members,
-                                 fin.weights + ((int64_t)tensor * groups_total + group) * R);
+        finish_group_in_block<R>(partials, s0, s1, tensor, group, groups_total, members,
+                                 fin.weights + ((int64_t)tensor * groups_total + group) * R, fin.tree);
     }
 }
 
@@ -705,57 +717,107 @@ __device__ __forceinline__ void pair_coefficients(double dot, double norm_a, dou
 // unchanged); with d = sum_{i in left, k in right} w_i w_k G_ik and the two blocks' squared norms
 // the pair coefficients follow, every leaf weight of the left (right) block is multiplied by ca
 // (cb), and the parent's squared norm is ca^2 |a|^2 + cb^2 |b|^2 + 2 ca cb d.
+//
+// opt.linear selects the other recursion of Section 3.4 instead: x = g_0, then x = Adasum(x, g_k)
+// for k = 1, 2, ...; the same algebra with the left operand always the running result.
+//
+// Also written, when asked for: the sum of the leaves' squared norms (first level) and the
+// orthogonality measure |result|^2 / sum_i |g_i|^2 of Section 3.6 (last level; NaN when every
+// leaf is zero).
 template <int R>
-__device__ void tree_weights_from_gram(const double* gram, int members, float* __restrict__ dst)
+__device__ void tree_weights_from_gram(const double* gram, int members, float* __restrict__ dst,
+                                       const TreeOptions& opt, int tensor, int group)
 {
-    __shared__ double weight[R], norm[R], row_dot[R], coef_a[R / 2], coef_b[R / 2];
+    __shared__ double weight[R], norm[R], row_dot[R], coef_a[R / 2 > 0 ? R / 2 : 1], coef_b[R / 2 > 0 ? R / 2 : 1];
     const int tid = threadIdx.x;
     if (tid < R) {
         weight[tid] = 1.0;
         norm[tid] = tid < members ? gram[gram_index(R, tid, tid)] : 0.0;
     }
     __syncthreads();
-    for (int w = 1; w < members; w *= 2) {
-        // leaf i of a left block: weight_i * sum over the sibling block of weight_k G_ik
-        if (tid < members) {
-            const int left = tid / (2 * w) * (2 * w);
-            const int mid = left + w;
-            double acc = 0.0;
-            if (tid < mid && mid < members) {
-                const int right_end = min(left + 2 * w, members);
-                for (int k = mid; k < right_end; ++k)
-                    acc += weight[k] * gram[gram_index(R, tid, k)];
-                acc *= weight[tid];
+    double leaf_sum = 0.0;
+    if (tid == 0 && (opt.leaf_norm_sums != nullptr || opt.orthogonality != nullptr))
+        for (int i = 0; i < members; ++i)
+            leaf_sum += norm[i];
+    __syncthreads();
+    if (!opt.linear) {
+        for (int w = 1; w < members; w *= 2) {
+            // leaf i of a left block: weight_i * sum over the sibling block of weight_k G_ik
+            if (tid < members) {
+                const int left = tid / (2 * w) * (2 * w);
+                const int mid = left + w;
+                double acc = 0.0;
+                if (tid < mid && mid < members) {
+                    const int right_end = min(left + 2 * w, members);
+                    for (int k = mid; k < right_end; ++k)
+                        acc += weight[k] * gram[gram_index(R, tid, k)];
+                    acc *= weight[tid];
+                }
+                row_dot[tid] = acc;
             }
-            row_dot[tid] = acc;
+            __syncthreads();
+            // one thread per pair of sibling blocks
+            const int pairs = (members + 2 * w - 1) / (2 * w);
+            if (tid < pairs) {
+                const int left = tid * 2 * w, mid = left + w;
+                double ca = 1.0, cb = 1.0;
+                if (mid < members) {
+                    double dot = 0.0;
+                    for (int i = left; i < mid; ++i)
+                        dot += row_dot[i];
+                    pair_coefficients(dot, norm[left], norm[mid], ca, cb);
+                    norm[left] = ca * ca * norm[left] + cb * cb * norm[mid] + 2.0 * ca * cb * dot;
+                }
+                coef_a[tid] = ca;
+                coef_b[tid] = cb;
+            }
+            __syncthreads();
+            if (tid < members) {
+                const int pair = tid / (2 * w);
+                const int mid = pair * 2 * w + w;
+                if (mid < members)
+                    weight[tid] *= tid < mid ? coef_a[pair] : coef_b[pair];
+            }
+            __syncthreads();
         }
-        __syncthreads();
-        // one thread per pair of sibling blocks
-        const int pairs = (members + 2 * w - 1) / (2 * w);
-        if (tid < pairs) {
-            const int left = tid * 2 * w, mid = left + w;
-            double ca = 1.0, cb = 1.0;
-            if (mid < members) {
+    } else {
+        for (int k = 1; k < members; ++k) {
+            if (tid < k)
+                row_dot[tid] = weight[tid] * gram[gram_index(R, tid, k)];
+            __syncthreads();
+            if (tid == 0) {
                 double dot = 0.0;
-                for (int i = left; i < mid; ++i)
+                for (int i = 0; i < k; ++i)
                     dot += row_dot[i];
-                pair_coefficients(dot, norm[left], norm[mid], ca, cb);
-                norm[left] = ca * ca * norm[left] + cb * cb * norm[mid] + 2.0 * ca * cb * dot;
+                double ca, cb;
+                pair_coefficients(dot, norm[0], norm[k], ca, cb);
+                norm[0] = ca * ca * norm[0] + cb * cb * norm[k] + 2.0 * ca * cb * dot;
+                coef_a[0] = ca;
+                coef_b[0] = cb;
             }
-            coef_a[tid] = ca;
-            coef_b[tid] = cb;
+            __syncthreads();
+            if (tid < k)
+                weight[tid] *= coef_a[0];
+            else if (tid == k)
+                weight[tid] = coef_b[0];
+            __syncthreads();
         }
-        __syncthreads();
-        if (tid < members) {
-            const int pair = tid / (2 * w);
-            const int mid = pair * 2 * w + w;
-            if (mid < members)
-                weight[tid] *= tid < mid ? coef_a[pair] : coef_b[pair];
-        }
-        __syncthreads();
     }
     if (tid < R)
         dst[tid] = tid < members ? (float)weight[tid] : 0.0f;
+    if (tid == 0) {
+        if (opt.leaf_norm_sums != nullptr && opt.level_is_first)
+            opt.leaf_norm_sums[(int64_t)tensor * opt.groups_first + group] = leaf_sum;
+        if (opt.orthogonality != nullptr && opt.level_is_last) {
+            double denom = leaf_sum;
+            if (!opt.level_is_first) {
+                denom = 0.0;
+                for (int gf = 0; gf < opt.groups_first; ++gf)
+                    denom += opt.leaf_norm_sums[(int64_t)tensor * opt.groups_first + gf];
+            }
+            opt.orthogonality[tensor] = denom == 0.0 ? __int_as_float(0x7fc00000) : (float)(norm[0] / denom);
+        }
+    }
 }
 
 // The tensor's partial matrices (segments seg_begin .. seg_end) added in fp64 by one block of
@@ -763,8 +825,8 @@ __device__ void tree_weights_from_gram(const double* gram, int members, float* _
 // segments q, q + Q, ... in order and the slices are added in order.  Partials were written by
 // other blocks of the running kernel, hence the L2 loads.
 template <int R>
-__device__ void finish_group_in_block(const float* partials, int seg_begin, int seg_end, int group,
-                                      int groups_total, int members, float* weights_dst)
+__device__ void finish_group_in_block(const float* partials, int seg_begin, int seg_end, int tensor, int group,
+                                      int groups_total, int members, float* weights_dst, const TreeOptions& opt)
 {
     constexpr int E = gram_entries(R);
     __shared__ double gram[E];
@@ -800,7 +862,7 @@ __device__ void finish_group_in_block(const float* partials, int seg_begin, int 
         }
     }
     __syncthreads();
-    tree_weights_from_gram<R>(gram, members, weights_dst);
+    tree_weights_from_gram<R>(gram, members, weights_dst, opt, tensor, group);
 }
 
 constexpr int kTreeThreadsMax = 1024;
@@ -824,7 +886,7 @@ __host__ __device__ constexpr int tree_entry_blocks(int radix)
 template <int R>
 __global__ void __launch_bounds__(kTreeThreadsMax)
 gram_finish_kernel(const float* __restrict__ partials, const int32_t* __restrict__ seg_first, int operands,
-                   double* __restrict__ gram64, float* __restrict__ weights)
+                   double* __restrict__ gram64, float* __restrict__ weights, TreeOptions opt)
 {
     constexpr int E = gram_entries(R);
     constexpr int EPB = tree_entries_per_block(R);
@@ -862,7 +924,7 @@ gram_finish_kernel(const float* __restrict__ partials, const int32_t* __restrict
     if (SINGLE) {
         __syncthreads();
         tree_weights_from_gram<R>(gram, min(R, operands - group * R),
-                                  weights + ((int64_t)tensor * groups + group) * R);
+                                  weights + ((int64_t)tensor * groups + group) * R, opt, tensor, group);
     }
 }
 
@@ -870,7 +932,7 @@ gram_finish_kernel(const float* __restrict__ partials, const int32_t* __restrict
 // several blocks of gram_finish_kernel; load it and run the tree.
 template <int R>
 __global__ void __launch_bounds__(kThreads)
-tree_weights_kernel(const double* __restrict__ gram64, int operands, float* __restrict__ weights)
+tree_weights_kernel(const double* __restrict__ gram64, int operands, float* __restrict__ weights, TreeOptions opt)
 {
     constexpr int E = gram_entries(R);
     __shared__ double gram[E];
@@ -879,7 +941,8 @@ tree_weights_kernel(const double* __restrict__ gram64, int operands, float* __re
     for (int k = threadIdx.x; k < E; k += kThreads)
         gram[k] = src[k];
     __syncthreads();
-    tree_weights_from_gram<R>(gram, min(R, operands - group * R), weights + ((int64_t)tensor * groups + group) * R);
+    tree_weights_from_gram<R>(gram, min(R, operands - group * R), weights + ((int64_t)tensor * groups + group) * R,
+                              opt, tensor, group);
 }
 
 // ---- pass 2: weighted sum ---------------------------------------------------------------------

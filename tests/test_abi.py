@@ -68,6 +68,13 @@ def test_plan_info(binding):
     assert info(100, 1, 8, "f32", binding.flags_radix(2, 2))["radices"] == [2, 2, 2]
     assert info(100, 1, 256, "f32", binding.flags_radix(16, 16))["radices"] == [16, 16]
     assert info(100, 1, 5, "f32", binding.flags_radix(4, 4))["radices"] == [4, 2]
+    linear = 1 << 18
+    assert info(100, 1, 20, "f32", linear)["radices"] == [32]
+    assert info(100, 1, 64, "bf16", linear)["radices"] == [64]
+    with pytest.raises(binding.AdasumError):
+        info(100, 1, 33, "f32", linear)                      # needs a 64 x 64 Gram matrix of fp32 inputs
+    with pytest.raises(binding.AdasumError):
+        info(100, 1, 8, "f32", linear | binding.flags_radix(8, 0))
     assert info(0, 0, 4, "f32")["launches"] == 0
     assert info(100, 1, 8, "f32", binding.flags_radix(2, 2))["launches"] == 6
     assert info(100, 1, 8, "f32", binding.flags_radix(2, 2) | (1 << 17))["launches"] == 9

@@ -1,0 +1,107 @@
+"""GPU parity of the two by-products of the Gram formulation against the fp64 oracle: the
+per-tensor orthogonality measure (Section 3.6) and the sequential recursion (Section 3.4)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import adasum_oracle as oracle
+from paper_2006_02924_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+TORCH_DT = workloads.TORCH_DTYPES
+LINEAR = 1 << 18
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2006_02924_b200 import binding
+
+    return binding
+
+
+def _np(t, dtype):
+    t = t.detach().cpu().contiguous()
+    return t.view(torch.uint16).numpy() if dtype == "bf16" else t.numpy()
+
+
+def _correlated(n, total, dtype, seed, rho=0.5):
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(seed)
+    shared = torch.randn(total, generator=gen, device="cuda")
+    return [((rho ** 0.5) * shared + ((1 - rho) ** 0.5) * torch.randn(total, generator=gen, device="cuda"))
+            .to(TORCH_DT[dtype]) for _ in range(n)]
+
+
+@pytest.mark.parametrize("dtype,tol", [("f32", 1e-4), ("f16", 5e-3), ("bf16", 2e-2)])
+@pytest.mark.parametrize("n,flags", [(2, 0), (8, 0), (13, 0), (64, 0), (64, (16) | (4 << 8)), (100, (8) | (16 << 8)),
+                                      (16, 1 << 17)])
+def test_orthogonality_measure(lib, dtype, tol, n, flags):
+    offsets = workloads.offsets_from_sizes([30_000, 17, 0, 4099, 64])
+    grads = _correlated(n, int(offsets[-1]), dtype, seed=900 + n)
+    for g in grads:
+        g[30_000:30_017] = 0                       # a tensor that is zero on every worker
+    out, ortho = lib.adasum_reduce_ex(grads, offsets, flags=flags)
+    torch.cuda.synchronize()
+    ref, ref_ortho = oracle.adasum_reduce([_np(g, dtype) for g in grads], offsets=offsets, dtype=dtype,
+                                          return_orthogonality=True, threads=0)
+    got = ortho.cpu().numpy().astype(np.float64)
+    assert np.isnan(got[1]) and np.isnan(ref_ortho[1])       # all-zero leaves
+    assert np.isnan(got[2])                                  # empty tensor
+    for t in (0, 3, 4):
+        assert abs(got[t] - ref_ortho[t]) <= tol * ref_ortho[t], (t, got[t], ref_ortho[t])
+    assert 1.0 / n - 1e-3 <= got[0] <= 1.0 + 1e-3
+    same = lib.adasum_reduce(grads, offsets, flags=flags)
+    assert torch.equal(same, out)                           # asking for the measure does not change the result
+
+
+def test_orthogonality_extremes(lib):
+    """Section 3.6: 1 for mutually orthogonal gradients, 1/n for identical ones (n = 64)."""
+    n, width = 64, 256
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(5)
+    ortho_inputs = []
+    for w in range(n):
+        g = torch.zeros(n * width, device="cuda")
+        g[w * width:(w + 1) * width] = (1 + w) * torch.randn(width, generator=gen, device="cuda")
+        ortho_inputs.append(g)
+    _, measure = lib.adasum_reduce_ex(ortho_inputs)
+    assert abs(float(measure[0]) - 1.0) < 1e-5
+    g = torch.randn(10_000, generator=gen, device="cuda")
+    _, measure = lib.adasum_reduce_ex([g.clone() for _ in range(n)])
+    assert abs(float(measure[0]) - 1.0 / n) < 1e-6
+
+
+def test_orthogonality_needs_two_workers(lib):
+    g = torch.randn(100, device="cuda")
+    with pytest.raises(lib.AdasumError):
+        lib.adasum_reduce_ex([g])
+
+
+@pytest.mark.parametrize("dtype,n,tol", [("f32", 2, 1e-5), ("f32", 3, 1e-5), ("f32", 5, 1e-5), ("f32", 16, 1e-5),
+                                         ("f32", 32, 1e-5), ("f16", 7, 2e-3), ("f16", 64, 2e-3), ("bf16", 33, 2e-3)])
+def test_linear_order(lib, dtype, n, tol):
+    offsets = workloads.offsets_from_sizes([20_000, 33, 4097, 128])
+    grads = _correlated(n, int(offsets[-1]), dtype, seed=950 + n, rho=0.6)
+    out, ortho = lib.adasum_reduce_ex(grads, offsets, flags=LINEAR)
+    torch.cuda.synchronize()
+    hosts = [_np(g, dtype) for g in grads]
+    ref, ref_ortho = oracle.adasum_reduce(hosts, offsets=offsets, dtype=dtype, linear_order=True,
+                                          return_orthogonality=True, threads=0)
+    got = out.cpu().numpy().astype(np.float64)
+    for t in range(4):
+        lo, hi = int(offsets[t]), int(offsets[t + 1])
+        err = np.linalg.norm(got[lo:hi] - ref[lo:hi]) / np.linalg.norm(ref[lo:hi])
+        assert err <= tol, (t, err)
+        assert abs(float(ortho[t]) - ref_ortho[t]) <= max(10 * tol, 1e-4) * ref_ortho[t]
+    if n > 3:      # for three workers the tree with its carried last operand IS the sequential order
+        tree = oracle.adasum_reduce(hosts, offsets=offsets, dtype=dtype, threads=0)
+        assert np.linalg.norm(got - tree) / np.linalg.norm(tree) > 10 * tol      # it really is another order
+
+
+def test_linear_order_limits(lib):
+    grads = [torch.randn(64, device="cuda") for _ in range(33)]
+    with pytest.raises(lib.AdasumError):
+        lib.adasum_reduce(grads, flags=LINEAR)
+    with pytest.raises(lib.AdasumError):
+        lib.adasum_reduce(grads[:8], flags=LINEAR | lib.flags_radix(8, 0))

@@ -156,6 +156,16 @@ def test_radix_64_for_16_bit_inputs(lib, dtype, n):
     _run_and_check(lib, grads, offsets, dtype, flags=lib.flags_radix(64, 0))
 
 
+@pytest.mark.parametrize("dtype,n,first", [("f32", 300, 16), ("f16", 600, 32), ("f32", 520, 2), ("bf16", 257, 8)])
+def test_more_operands_than_one_launch_carries(lib, dtype, n, first):
+    """A launch carries 256 operand pointers; wider levels are split over several launches."""
+    offsets = workloads.offsets_from_sizes([2000, 5, 777, 64])
+    grads = _correlated(n, int(offsets[-1]), dtype, seed=280 + n, rho=0.7)
+    info = lib.adasum_plan_info(int(offsets[-1]), 4, n, dtype, lib.flags_radix(first, 0))
+    assert info["launches"] > 2 * len(info["radices"])
+    _run_and_check(lib, grads, offsets, dtype, flags=lib.flags_radix(first, 0))
+
+
 def test_radix_64_is_refused_for_fp32(lib):
     grads = _correlated(64, 1000, "f32", seed=260)
     with pytest.raises(lib.AdasumError):
