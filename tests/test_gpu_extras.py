@@ -105,3 +105,29 @@ def test_linear_order_limits(lib):
         lib.adasum_reduce(grads, flags=LINEAR)
     with pytest.raises(lib.AdasumError):
         lib.adasum_reduce(grads[:8], flags=LINEAR | lib.flags_radix(8, 0))
+
+
+def test_reduce_can_be_replayed_from_a_cuda_graph(lib):
+    """After one ordinary call (which builds the cached segment tables) the reduce is a fixed
+    sequence of stream operations: capture it once, replay it on new data."""
+    offsets = workloads.offsets_from_sizes([50_000, 300, 9001])
+    total = int(offsets[-1])
+    grads = _correlated(20, total, "f32", seed=990)
+    out = torch.empty(total, device="cuda")
+    ws = torch.empty(lib.adasum_workspace_bytes(total, 3, 20, "f32"), dtype=torch.uint8, device="cuda")
+    expected_first = lib.adasum_reduce(grads, offsets, out=out, workspace=ws).clone()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        lib.adasum_reduce(grads, offsets, out=out, workspace=ws)
+    out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, expected_first)
+    fresh = _correlated(20, total, "f32", seed=991)
+    for dst, src in zip(grads, fresh):
+        dst.copy_(src)                                # same buffers, new contents
+    graph.replay()
+    torch.cuda.synchronize()
+    ref = oracle.adasum_reduce([_np(g, "f32") for g in grads], offsets=offsets, threads=0)
+    got = out.cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-5
