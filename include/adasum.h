@@ -158,6 +158,41 @@ adasum_status_t adasum_reduce_ex(const void* const* grads, const int64_t* tensor
                                  size_t workspace_bytes, uint32_t flags, void* stream);
 
 /*
+ * The same reduce with the ELEMENTS of every tensor spread over several GPUs (one process per GPU).
+ *
+ * Each GPU holds, for all n_workers workers, its own slice of every tensor: grads[w] is worker w's
+ * fused buffer of this GPU's slices and tensor_offsets describes those local slices (the number of
+ * tensors and their order are the same on every GPU; a tensor may be empty on some GPUs).  Dot
+ * products and norms of a tensor are sums over all its elements, so one exchange per level is
+ * needed, exactly the one of Algorithm 1 ("partial dot products", then an all-reduce of the
+ * scalars, then "apply Adasum"): for level = 0 .. num_levels - 1 (adasum_plan_info)
+ *
+ *   1. adasum_sharded_gram(level)   streams this GPU's operands once and leaves this GPU's fp64
+ *                                   Gram sums in the workspace, *sums_count doubles starting
+ *                                   *sums_offset bytes into it (same count and layout on every GPU);
+ *   2. the caller adds those doubles over all GPUs in place (e.g. ncclAllReduce, sum);
+ *   3. adasum_sharded_apply(level)  derives the weights from the summed matrices and streams the
+ *                                   operands a second time; after the last level `out` holds this
+ *                                   GPU's slices of the result (and `orthogonality`, if not NULL,
+ *                                   the per-tensor measure, identical on every GPU).
+ *
+ * Arguments as for adasum_reduce_ex; the workspace (adasum_workspace_bytes of the LOCAL sizes) must
+ * be left untouched between the calls of one reduce, and all calls of one reduce must use the
+ * same flags and be stream-ordered.  n_workers >= 2.  The library itself never communicates.
+ * Errors as for adasum_reduce, plus ADASUM_ERR_ARG for a level outside the plan.
+ */
+adasum_status_t adasum_sharded_gram(const void* const* grads, const int64_t* tensor_offsets,
+                                    int32_t num_tensors, int32_t n_workers, adasum_dtype_t dtype,
+                                    void* workspace, size_t workspace_bytes, uint32_t flags,
+                                    int32_t level, size_t* sums_offset, int64_t* sums_count,
+                                    void* stream);
+adasum_status_t adasum_sharded_apply(const void* const* grads, const int64_t* tensor_offsets,
+                                     int32_t num_tensors, int32_t n_workers, adasum_dtype_t dtype,
+                                     float* out, float* orthogonality, void* workspace,
+                                     size_t workspace_bytes, uint32_t flags, int32_t level,
+                                     void* stream);
+
+/*
  * One application of the operator per tensor, out = Adasum(a, b) (Section 3; the "partial dot
  * products" and "apply Adasum" steps of Algorithm 1).  Same conventions as adasum_reduce with
  * n_workers = 2; `a` and `b` are device pointers.

@@ -172,6 +172,78 @@ def adasum_reduce_ex(grads, tensor_offsets=None, out=None, orthogonality=None, w
     return out, orthogonality
 
 
+_lib.adasum_sharded_gram.restype = ctypes.c_int
+_lib.adasum_sharded_gram.argtypes = [ctypes.POINTER(ctypes.c_void_p), _i64p, ctypes.c_int32, ctypes.c_int32,
+                                     ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_uint32, ctypes.c_int32,
+                                     ctypes.POINTER(ctypes.c_size_t), _i64p, ctypes.c_void_p]
+_lib.adasum_sharded_apply.restype = ctypes.c_int
+_lib.adasum_sharded_apply.argtypes = [ctypes.POINTER(ctypes.c_void_p), _i64p, ctypes.c_int32, ctypes.c_int32,
+                                      ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                      ctypes.c_size_t, ctypes.c_uint32, ctypes.c_int32, ctypes.c_void_p]
+
+
+def adasum_sharded_gram(grads, tensor_offsets, workspace, level: int, flags: int = 0, stream=None):
+    """``adasum_sharded_gram`` of the C ABI.  Returns this GPU's fp64 Gram sums of ``level`` as a
+    float64 view INTO ``workspace`` (add it over the GPUs in place, then call ``adasum_sharded_apply``)."""
+    grads = list(grads)
+    first = grads[0]
+    offs = _offsets_array(tensor_offsets, first.numel())
+    ptrs = (ctypes.c_void_p * len(grads))(*[g.data_ptr() for g in grads])
+    off, count = ctypes.c_size_t(), ctypes.c_int64()
+    with torch.cuda.device(first.device):
+        status = _lib.adasum_sharded_gram(ptrs, offs.ctypes.data_as(_i64p), offs.size - 1, len(grads),
+                                          _dtype_code(first.dtype), workspace.data_ptr(),
+                                          workspace.numel() * workspace.element_size(), int(flags), int(level),
+                                          ctypes.byref(off), ctypes.byref(count), _stream_handle(stream))
+    if status != ADASUM_OK:
+        raise AdasumError(status)
+    return workspace.view(torch.uint8)[off.value:off.value + 8 * count.value].view(torch.float64)
+
+
+def adasum_sharded_apply(grads, tensor_offsets, out, workspace, level: int, orthogonality=None, flags: int = 0,
+                         stream=None):
+    """``adasum_sharded_apply`` of the C ABI."""
+    grads = list(grads)
+    first = grads[0]
+    offs = _offsets_array(tensor_offsets, first.numel())
+    ptrs = (ctypes.c_void_p * len(grads))(*[g.data_ptr() for g in grads])
+    with torch.cuda.device(first.device):
+        status = _lib.adasum_sharded_apply(ptrs, offs.ctypes.data_as(_i64p), offs.size - 1, len(grads),
+                                           _dtype_code(first.dtype), out.data_ptr(),
+                                           None if orthogonality is None else orthogonality.data_ptr(),
+                                           workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                           int(flags), int(level), _stream_handle(stream))
+    if status != ADASUM_OK:
+        raise AdasumError(status)
+    return out
+
+
+def adasum_reduce_sharded(grads, tensor_offsets, group=None, out=None, orthogonality=None, workspace=None,
+                          flags: int = 0, stream=None):
+    """The whole element-sharded reduce on this rank: per level ``adasum_sharded_gram``, a
+    ``torch.distributed.all_reduce`` (sum) of the Gram sums over ``group``, ``adasum_sharded_apply``.
+    ``grads`` are this rank's slices (see ``include/adasum.h``).  Returns this rank's slice of the result."""
+    import torch.distributed as dist
+
+    grads = list(grads)
+    first = grads[0]
+    total = first.numel()
+    offs = _offsets_array(tensor_offsets, total)
+    num_tensors = offs.size - 1
+    if out is None:
+        out = torch.empty(total, dtype=torch.float32, device=first.device)
+    need = adasum_workspace_bytes(total, num_tensors, len(grads), first.dtype, flags)
+    workspace, _, _ = _workspace(workspace, need, first.device)
+    levels = len(adasum_plan_info(total, num_tensors, len(grads), first.dtype, flags)["radices"])
+    for level in range(levels):
+        sums = adasum_sharded_gram(grads, offs, workspace, level, flags=flags, stream=stream)
+        if sums.numel() > 0:
+            dist.all_reduce(sums, op=dist.ReduceOp.SUM, group=group)
+        adasum_sharded_apply(grads, offs, out, workspace, level, orthogonality=orthogonality, flags=flags,
+                             stream=stream)
+    return out
+
+
 def adasum_pair(a, b, tensor_offsets=None, out=None, workspace=None, flags: int = 0, stream=None):
     """``adasum_pair`` of the C ABI: ``out = Adasum(a, b)`` per tensor."""
     total = a.numel()

@@ -216,12 +216,10 @@ Layout make_layout(const LevelPlan& plan, int64_t total_elems, int32_t num_tenso
         const size_t c = (size_t)(num_tensors > 0 ? num_tensors : 1) * lv.groups * sizeof(int);
         if (c > lay.counters_bytes)
             lay.counters_bytes = c;
-        if (lv.radix >= 32) {
-            const size_t g64 = (size_t)(num_tensors > 0 ? num_tensors : 1) * lv.groups * gram_entries(lv.radix) *
-                               sizeof(double);
-            if (g64 > lay.gram64_bytes)
-                lay.gram64_bytes = g64;
-        }
+        const size_t g64 = (size_t)(num_tensors > 0 ? num_tensors : 1) * lv.groups * gram_entries(lv.radix) *
+                           sizeof(double);
+        if (g64 > lay.gram64_bytes)
+            lay.gram64_bytes = g64;
         if (l + 1 < plan.num_levels) {      // this level's output is an intermediate
             const size_t b = (size_t)lv.groups * lay.padded_elems * sizeof(float);
             if (b > lay.buffer_bytes[l & 1])
@@ -425,14 +423,16 @@ void launch_wsum(const OperandTable& ops, int operands, int groups_here, const S
 template <int R>
 cudaError_t launch_weights(const float* partials, const SegmentTable& tab, int32_t num_tensors, int operands,
                            int groups, double* gram64, float* weights, const TreeOptions& opt, cudaStream_t stream,
-                           int* launches)
+                           int* launches, bool sums_only = false)
 {
     dim3 grid((unsigned)num_tensors, (unsigned)groups, (unsigned)tree_entry_blocks(R));
     // wide blocks only pay off when some tensor has many per-segment partials to add
     const int threads = tab.max_segments_per_tensor > 64 ? kTreeThreadsMax : 256;
     gram_finish_kernel<R><<<grid, threads, threads * sizeof(double), stream>>>(partials, tab.d_seg_first, operands,
-                                                                                gram64, weights, opt);
+                                                                                gram64, weights, opt, sums_only ? 1 : 0);
     *launches = 1;
+    if (sums_only)
+        return cudaSuccess;
     if constexpr (tree_entry_blocks(R) > 1) {
         dim3 grid2((unsigned)num_tensors, (unsigned)groups);
         tree_weights_kernel<R><<<grid2, kThreads, 0, stream>>>(gram64, operands, weights, opt);
@@ -440,6 +440,21 @@ cudaError_t launch_weights(const float* partials, const SegmentTable& tab, int32
     }
     return cudaSuccess;
 }
+
+template <int R>
+void launch_tree_from_sums(const double* gram64, int32_t num_tensors, int operands, int groups, float* weights,
+                           const TreeOptions& opt, cudaStream_t stream)
+{
+    dim3 grid((unsigned)num_tensors, (unsigned)groups);
+    tree_weights_kernel<R><<<grid, kThreads, 0, stream>>>(gram64, operands, weights, opt);
+}
+
+// Which part of a level a call runs.
+enum LevelPhase {
+    PHASE_WHOLE = 0,        // pass 1, coefficients, pass 2
+    PHASE_GRAM_SUMS = 1,    // pass 1, then this GPU's fp64 Gram sums to gram64 (to be added across GPUs)
+    PHASE_APPLY = 2         // coefficients from gram64, then pass 2
+};
 
 struct LevelArgs {
     const void* const* operand_ptrs;   // host array, `operands` entries
@@ -452,6 +467,7 @@ struct LevelArgs {
     float* partials;
     int* counters;      // ticket counters for finishing inside pass 1, or nullptr
     TreeOptions tree;
+    LevelPhase phase;
     double* gram64;
     float* weights;
     float* dst;
@@ -466,10 +482,10 @@ adasum_status_t run_level_typed(const LevelArgs& a)
 {
     constexpr int kGroupsPerLaunch = kMaxOperandsPerLaunch / R;
     // the last block of every (tensor, group) in pass 1 also derives the weights
-    const bool fused_finish = a.counters != nullptr;
+    const bool fused_finish = a.counters != nullptr && a.phase == PHASE_WHOLE;
     const FinishArgs fin{a.gram_tab->d_seg_first, fused_finish ? a.counters : nullptr, a.weights, a.tree};
     // pass 1
-    for (int g0 = 0; g0 < a.groups; g0 += kGroupsPerLaunch) {
+    for (int g0 = 0; g0 < a.groups && a.phase != PHASE_APPLY; g0 += kGroupsPerLaunch) {
         const int groups_here = a.groups - g0 < kGroupsPerLaunch ? a.groups - g0 : kGroupsPerLaunch;
         const int op0 = g0 * R;
         const int ops_here = a.operands - op0 < kMaxOperandsPerLaunch ? a.operands - op0 : kMaxOperandsPerLaunch;
@@ -484,14 +500,18 @@ adasum_status_t run_level_typed(const LevelArgs& a)
                                                         a.partials, a.groups, g0, fin, a.stream)));
         profile_mark(a.stream, ADASUM_KERNEL_GRAM_PARTIAL, a.level, R, false);
     }
-    if (!fused_finish) {
+    if (a.phase == PHASE_APPLY) {
+        launch_tree_from_sums<R>(a.gram64, a.num_tensors, a.operands, a.groups, a.weights, a.tree, a.stream);
+        profile_mark(a.stream, ADASUM_KERNEL_TREE_WEIGHTS, a.level, R, false);
+    } else if (!fused_finish) {
         int weight_launches = 0;
         ADASUM_CUDA_CHECK(launch_weights<R>(a.partials, *a.gram_tab, a.num_tensors, a.operands, a.groups,
-                                            a.gram64, a.weights, a.tree, a.stream, &weight_launches));
+                                            a.gram64, a.weights, a.tree, a.stream, &weight_launches,
+                                            a.phase == PHASE_GRAM_SUMS));
         profile_mark(a.stream, ADASUM_KERNEL_TREE_WEIGHTS, a.level, R, false);
     }
     // pass 2
-    for (int g0 = 0; g0 < a.groups; g0 += kGroupsPerLaunch) {
+    for (int g0 = 0; g0 < a.groups && a.phase != PHASE_GRAM_SUMS; g0 += kGroupsPerLaunch) {
         const int groups_here = a.groups - g0 < kGroupsPerLaunch ? a.groups - g0 : kGroupsPerLaunch;
         const int op0 = g0 * R;
         const int ops_here = a.operands - op0 < kMaxOperandsPerLaunch ? a.operands - op0 : kMaxOperandsPerLaunch;
@@ -572,7 +592,9 @@ adasum_status_t check_common(const int64_t* offsets, int32_t num_tensors, int32_
 
 adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, int32_t num_tensors,
                             int32_t n_workers, adasum_dtype_t dtype, float* out, float* orthogonality,
-                            void* workspace, size_t workspace_bytes, uint32_t flags, cudaStream_t stream)
+                            void* workspace, size_t workspace_bytes, uint32_t flags, cudaStream_t stream,
+                            LevelPhase phase = PHASE_WHOLE, int only_level = -1, size_t* sums_offset = nullptr,
+                            int64_t* sums_count = nullptr)
 {
     g_error[0] = '\0';
     if (!grads)
@@ -588,21 +610,31 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     if (!plan_levels(n_workers, dtype, flags, &plan))
         return fail(ADASUM_ERR_ARG, "invalid flags 0x%x for %d workers of this dtype", flags, n_workers);
     const int64_t total = offsets[num_tensors];
-    if (total == 0)
+    const bool sharded = phase != PHASE_WHOLE;
+    if (sharded) {
+        if (n_workers < 2)
+            return fail(ADASUM_ERR_ARG, "the sharded calls need at least two workers");
+        if (only_level < 0 || only_level >= plan.num_levels)
+            return fail(ADASUM_ERR_ARG, "level %d outside 0..%d", only_level, plan.num_levels - 1);
+        if (flags & ADASUM_FLAG_SEPARATE_FINISH)
+            return fail(ADASUM_ERR_ARG, "ADASUM_FLAG_SEPARATE_FINISH has no meaning for the sharded calls");
+    }
+    if (total == 0 && !sharded)
         return ADASUM_OK;
-    if (!out)
+    const bool need_out = phase != PHASE_GRAM_SUMS && total > 0;
+    if (need_out && !out)
         return fail(ADASUM_ERR_NULL, "out is NULL");
     if (reinterpret_cast<uintptr_t>(out) & 3u)
         return fail(ADASUM_ERR_ARG, "out is not 4-byte aligned");
     const int eb = dtype_bytes(dtype);
-    const size_t in_bytes = (size_t)total * eb, out_bytes = (size_t)total * sizeof(float);
-    bool vec = aligned16(out);
-    for (int w = 0; w < n_workers; ++w) {
+    const size_t in_bytes = (size_t)total * eb, out_bytes = out ? (size_t)total * sizeof(float) : 0;
+    bool vec = out ? aligned16(out) : true;
+    for (int w = 0; w < n_workers && total > 0; ++w) {
         if (!grads[w])
             return fail(ADASUM_ERR_NULL, "grads[%d] is NULL", w);
         if (reinterpret_cast<uintptr_t>(grads[w]) & (uintptr_t)(eb - 1))
             return fail(ADASUM_ERR_ARG, "grads[%d] is not aligned to its element size", w);
-        if (ranges_overlap(grads[w], in_bytes, out, out_bytes))
+        if (out && ranges_overlap(grads[w], in_bytes, out, out_bytes))
             return fail(ADASUM_ERR_ARG, "out overlaps grads[%d]", w);
         vec = vec && aligned16(grads[w]);
     }
@@ -614,9 +646,9 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
             return fail(ADASUM_ERR_WORKSPACE, "workspace has %zu bytes, need %zu", workspace_bytes, lay.total);
         if (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1))
             return fail(ADASUM_ERR_ARG, "workspace is not %zu-byte aligned", kAlign);
-        if (ranges_overlap(workspace, lay.total, out, out_bytes))
+        if (out && total > 0 && ranges_overlap(workspace, lay.total, out, out_bytes))
             return fail(ADASUM_ERR_ARG, "workspace overlaps out");
-        for (int w = 0; w < n_workers; ++w)
+        for (int w = 0; w < n_workers && total > 0; ++w)
             if (ranges_overlap(workspace, lay.total, grads[w], in_bytes))
                 return fail(ADASUM_ERR_ARG, "workspace overlaps grads[%d]", w);
     }
@@ -637,14 +669,38 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     }
 
     char* ws = static_cast<char*>(workspace);
-    const bool separate_finish = (flags & ADASUM_FLAG_SEPARATE_FINISH) != 0;
+    const bool separate_finish = (flags & ADASUM_FLAG_SEPARATE_FINISH) != 0 || sharded;
     if (!separate_finish && lay.counters_bytes > 0)     // the workspace arrives with unknown contents
         ADASUM_CUDA_CHECK(cudaMemsetAsync(ws + lay.counters, 0, lay.counters_bytes, stream));
-    if (orthogonality && num_tensors > 0)               // NaN for tensors without elements
+    if (orthogonality && num_tensors > 0 && (!sharded || (phase == PHASE_APPLY && only_level == 0)))
         ADASUM_CUDA_CHECK(cudaMemsetAsync(orthogonality, 0xff, sizeof(float) * (size_t)num_tensors, stream));
+    if (phase == PHASE_GRAM_SUMS) {
+        const Level& lv = plan.level[only_level];
+        const size_t count = (size_t)num_tensors * lv.groups * gram_entries(lv.radix);
+        if (sums_offset)
+            *sums_offset = lay.gram64;
+        if (sums_count)
+            *sums_count = (int64_t)count;
+        if (total == 0 || num_tensors == 0) {           // this GPU holds no element: its sums are zero
+            if (count > 0)
+                ADASUM_CUDA_CHECK(cudaMemsetAsync(ws + lay.gram64, 0, count * sizeof(double), stream));
+            return ADASUM_OK;
+        }
+    }
+    if (total == 0 || num_tensors == 0)
+        return ADASUM_OK;
     std::vector<const void*> operand_ptrs(grads, grads + n_workers);
     for (int l = 0; l < plan.num_levels; ++l) {
         const Level& lv = plan.level[l];
+        if (only_level >= 0 && l != only_level) {       // other levels' operands: the intermediates
+            if (l + 1 < plan.num_levels) {
+                float* buf = reinterpret_cast<float*>(ws + lay.buffer[l & 1]);
+                operand_ptrs.resize((size_t)lv.groups);
+                for (int g = 0; g < lv.groups; ++g)
+                    operand_ptrs[g] = buf + (int64_t)g * lay.padded_elems;
+            }
+            continue;
+        }
         const bool simple_kernels = (flags & ADASUM_FLAG_SIMPLE_KERNELS) != 0;
         const GramKind kind = gram_kind(lv.radix, simple_kernels);
         const SegmentTable* gram_tab = nullptr;
@@ -668,6 +724,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         a.weights = reinterpret_cast<float*>(ws + lay.weights);
         a.gram64 = reinterpret_cast<double*>(ws + lay.gram64);
         a.counters = separate_finish ? nullptr : reinterpret_cast<int*>(ws + lay.counters);
+        a.phase = phase;
         a.tree.linear = (flags & ADASUM_FLAG_LINEAR_ORDER) ? 1 : 0;
         a.tree.level_is_first = l == 0;
         a.tree.level_is_last = l + 1 == plan.num_levels;
@@ -885,6 +942,25 @@ adasum_status_t adasum_reduce_ex(const void* const* grads, const int64_t* tensor
 {
     return adasum::reduce_impl(grads, tensor_offsets, num_tensors, n_workers, dtype, out, orthogonality, workspace,
                                workspace_bytes, flags, static_cast<cudaStream_t>(stream));
+}
+
+adasum_status_t adasum_sharded_gram(const void* const* grads, const int64_t* tensor_offsets,
+                                    int32_t num_tensors, int32_t n_workers, adasum_dtype_t dtype,
+                                    void* workspace, size_t workspace_bytes, uint32_t flags, int32_t level,
+                                    size_t* sums_offset, int64_t* sums_count, void* stream)
+{
+    return adasum::reduce_impl(grads, tensor_offsets, num_tensors, n_workers, dtype, nullptr, nullptr, workspace,
+                               workspace_bytes, flags, static_cast<cudaStream_t>(stream), adasum::PHASE_GRAM_SUMS,
+                               level, sums_offset, sums_count);
+}
+
+adasum_status_t adasum_sharded_apply(const void* const* grads, const int64_t* tensor_offsets,
+                                     int32_t num_tensors, int32_t n_workers, adasum_dtype_t dtype, float* out,
+                                     float* orthogonality, void* workspace, size_t workspace_bytes, uint32_t flags,
+                                     int32_t level, void* stream)
+{
+    return adasum::reduce_impl(grads, tensor_offsets, num_tensors, n_workers, dtype, out, orthogonality, workspace,
+                               workspace_bytes, flags, static_cast<cudaStream_t>(stream), adasum::PHASE_APPLY, level);
 }
 
 adasum_status_t adasum_pair(const void* a, const void* b, const int64_t* tensor_offsets,

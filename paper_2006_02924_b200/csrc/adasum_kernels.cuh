@@ -882,11 +882,12 @@ __host__ __device__ constexpr int tree_entry_blocks(int radix)
 // slice q takes segments q, q + Q, ... in order, then the slices are added in order (fixed order
 // for a given block size: deterministic).  When the whole matrix fits one block (R <= 16) the
 // same block goes on to run the tree and writes weights[(tensor * groups + group) * R + i];
-// otherwise it stores its entries to gram64 and tree_weights_kernel finishes.
+// otherwise, or when sums_only is set (the sums are to be added across GPUs first), it stores
+// its entries to gram64 and tree_weights_kernel finishes.
 template <int R>
 __global__ void __launch_bounds__(kTreeThreadsMax)
 gram_finish_kernel(const float* __restrict__ partials, const int32_t* __restrict__ seg_first, int operands,
-                   double* __restrict__ gram64, float* __restrict__ weights, TreeOptions opt)
+                   double* __restrict__ gram64, float* __restrict__ weights, TreeOptions opt, int sums_only)
 {
     constexpr int E = gram_entries(R);
     constexpr int EPB = tree_entries_per_block(R);
@@ -916,20 +917,21 @@ gram_finish_kernel(const float* __restrict__ partials, const int32_t* __restrict
         double s = slice_sum[kk];
         for (int qq = 1; qq < Q; ++qq)
             s += slice_sum[qq * EPB + kk];
-        if (SINGLE)
+        if (SINGLE && !sums_only)
             gram[kk] = s;
         else
             gram64[((int64_t)tensor * groups + group) * E + k] = s;
     }
-    if (SINGLE) {
+    if (SINGLE && !sums_only) {      // sums_only is uniform over the grid
         __syncthreads();
         tree_weights_from_gram<R>(gram, min(R, operands - group * R),
                                   weights + ((int64_t)tensor * groups + group) * R, opt, tensor, group);
     }
 }
 
-// grid = (tensors, groups); block = kThreads.  Radix >= 32: the Gram matrix was finished by
-// several blocks of gram_finish_kernel; load it and run the tree.
+// grid = (tensors, groups); block = kThreads.  The Gram matrix was finished into gram64 (by
+// several blocks of gram_finish_kernel at radix >= 32, or to be summed across GPUs); load it and
+// run the tree.
 template <int R>
 __global__ void __launch_bounds__(kThreads)
 tree_weights_kernel(const double* __restrict__ gram64, int operands, float* __restrict__ weights, TreeOptions opt)

@@ -187,3 +187,24 @@ def reduced_sizes(sizes, divisor: int, keep_ragged: bool = True, smallest: int =
             r += 1 + (i % 5)
         out.append(r)
     return out
+
+
+def element_shards(offsets, world: int, align: int = 64):
+    """Split every tensor of a fused buffer into `world` contiguous element ranges (the layout the
+    element-sharded reduce expects: rank r holds piece r of every tensor).  Cuts are rounded to
+    `align` elements, so short tensors live on the first ranks only and are empty elsewhere.
+    Returns, per rank, (local_offsets, pieces) with pieces[t] = (lo, hi) in the global buffer."""
+    offsets = np.asarray(offsets, dtype=np.int64)
+    shards = []
+    for rank in range(world):
+        pieces, sizes = [], []
+        for t in range(len(offsets) - 1):
+            lo, hi = int(offsets[t]), int(offsets[t + 1])
+            per = -(-(hi - lo) // world)
+            per = -(-per // align) * align
+            a = min(hi, lo + rank * per)
+            b = min(hi, lo + (rank + 1) * per)
+            pieces.append((a, b))
+            sizes.append(b - a)
+        shards.append((offsets_from_sizes(sizes), pieces))
+    return shards

@@ -68,3 +68,18 @@ def test_reference_arm_prints_one_line_on_rank0_only():
     line = json.loads(out.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["unit"] == "GB/s" and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_element_shards_cover_every_tensor_once():
+    offsets = workloads.offsets_from_sizes([1000, 3, 0, 130, 64])
+    for world in (1, 2, 3, 8):
+        shards = workloads.element_shards(offsets, world)
+        assert len(shards) == world
+        for t in range(len(offsets) - 1):
+            cursor = int(offsets[t])
+            for local_offsets, pieces in shards:
+                lo, hi = pieces[t]
+                assert lo == cursor and hi >= lo
+                assert int(local_offsets[t + 1] - local_offsets[t]) == hi - lo
+                cursor = hi
+            assert cursor == int(offsets[t + 1])
