@@ -110,7 +110,10 @@ size_t adasum_workspace_bytes(int64_t total_elems, int32_t num_tensors, int32_t 
 /*
  * How a reduce with these sizes will run: writes the radix of each level into radices[]
  * (room for ADASUM_MAX_LEVELS entries), the number of levels into *num_levels and the number
- * of kernel launches into *num_launches (each may be NULL).  Host-only.
+ * of kernel launches on a B200 into *num_launches (each may be NULL).  Host-only.  A one-level
+ * reduce of at most 8 workers whose operands total at most 96 MB is a single cooperative launch that
+ * reads the operands from HBM once (the second pass finds them in the L2) unless flag bit 16 or 17
+ * is set.
  */
 adasum_status_t adasum_plan_info(int64_t total_elems, int32_t num_tensors, int32_t n_workers,
                                  adasum_dtype_t dtype, uint32_t flags, int32_t* radices,
@@ -258,6 +261,7 @@ const char* adasum_last_error(void);
 #define ADASUM_KERNEL_TREE_WEIGHTS 1
 #define ADASUM_KERNEL_WEIGHTED_SUM 2
 #define ADASUM_KERNEL_CONVERT 3
+#define ADASUM_KERNEL_FUSED_SMALL 4   /* both passes in one cooperative launch (inputs that fit the L2) */
 
 typedef struct {
     int32_t kernel;

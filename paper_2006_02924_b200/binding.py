@@ -272,7 +272,7 @@ class _LaunchRecord(ctypes.Structure):
                 ("ms", ctypes.c_float)]
 
 
-KERNEL_NAMES = {0: "gram_partial", 1: "tree_weights", 2: "weighted_sum", 3: "convert"}
+KERNEL_NAMES = {0: "gram_partial", 1: "tree_weights", 2: "weighted_sum", 3: "convert", 4: "fused_small"}
 
 _lib.adasum_profile_enable.restype = ctypes.c_int
 _lib.adasum_profile_enable.argtypes = [ctypes.c_int32]

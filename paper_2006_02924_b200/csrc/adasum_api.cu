@@ -456,6 +456,79 @@ enum LevelPhase {
     PHASE_APPLY = 2         // coefficients from gram64, then pass 2
 };
 
+// ---- single-launch path for inputs that fit the L2 ------------------------------------------------
+
+constexpr int64_t kSmallInputBytes = int64_t(96) << 20;    // operands that the 126 MB L2 holds with room to spare
+constexpr int kSmallBlocksPerSm = 2;                       // blocks per SM the grid is sized for (all variants keep >= 2 resident)
+constexpr int kSmallSegmentGrain = 1024;
+
+// Host-only rule (no device query): is this reduce served by fused_small_kernel, and with which
+// segment length?  `blocks` is the number of blocks that can be resident at once.
+bool small_input_plan(const LevelPlan& plan, int64_t total, int32_t num_tensors, int n_workers, int elem_bytes,
+                      uint32_t flags, int blocks, int* seg_len)
+{
+    if (plan.num_levels != 1 || plan.level[0].radix > 8 || plan.level[0].groups != 1)
+        return false;
+    if (flags & (ADASUM_FLAG_SIMPLE_KERNELS | ADASUM_FLAG_SEPARATE_FINISH))
+        return false;
+    if (total <= 0 || (int64_t)n_workers * total * elem_bytes > kSmallInputBytes)
+        return false;
+    // every tensor ends with one ragged segment: budget for those first
+    const int64_t room = (int64_t)blocks - 2 * (int64_t)num_tensors;
+    if (room < 8)
+        return false;
+    int64_t len = (total + room - 1) / room;
+    len = (len + kSmallSegmentGrain - 1) / kSmallSegmentGrain * kSmallSegmentGrain;
+    if (len < 2048)
+        len = 2048;
+    if (len > (int64_t(1) << 20))
+        return false;
+    *seg_len = (int)len;
+    return true;
+}
+
+template <typename T, int R, bool VEC>
+cudaError_t launch_fused_small(const OperandTable& ops, int operands, const SegmentTable& tab, float* partials,
+                               const FinishArgs& fin, float* out, cudaStream_t stream)
+{
+    auto kernel = fused_small_kernel<T, R, VEC>;
+    int operands_arg = operands;
+    const Segment* segments = tab.d_segments;
+    void* args[] = {(void*)&ops, (void*)&operands_arg, (void*)&segments, (void*)&partials, (void*)&fin, (void*)&out};
+    return cudaLaunchCooperativeKernel((const void*)kernel, dim3((unsigned)tab.num_segments), dim3(kThreads), args,
+                                       0, stream);
+}
+
+template <typename T, bool VEC>
+cudaError_t launch_fused_small_radix(int radix, const OperandTable& ops, int operands, const SegmentTable& tab,
+                                     float* partials, const FinishArgs& fin, float* out, cudaStream_t stream)
+{
+    switch (radix) {
+    case 2: return launch_fused_small<T, 2, VEC>(ops, operands, tab, partials, fin, out, stream);
+    case 4: return launch_fused_small<T, 4, VEC>(ops, operands, tab, partials, fin, out, stream);
+    case 8: return launch_fused_small<T, 8, VEC>(ops, operands, tab, partials, fin, out, stream);
+    default: return cudaErrorInvalidValue;
+    }
+}
+
+// Blocks of fused_small_kernel that the current device keeps resident (0: no cooperative launch).
+int resident_small_blocks()
+{
+    static int cached[64] = {};
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64)
+        return 0;
+    if (cached[device] == 0) {
+        int sms = 0, coop = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
+            cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, device) != cudaSuccess || !coop || sms <= 0)
+            cached[device] = -1;
+        else
+            cached[device] = sms * kSmallBlocksPerSm;
+    }
+    return cached[device] > 0 ? cached[device] : 0;
+}
+
 struct LevelArgs {
     const void* const* operand_ptrs;   // host array, `operands` entries
     int operands;
@@ -548,9 +621,13 @@ adasum_status_t run_level(int radix, const LevelArgs& a)
     }
 }
 
-int launches_of(const LevelPlan& plan, int n_workers, uint32_t flags)
+int launches_of(const LevelPlan& plan, int n_workers, uint32_t flags, int64_t total, int32_t num_tensors,
+                int elem_bytes)
 {
     if (n_workers == 1)
+        return 1;
+    int seg_len = 0;        // on a B200: 148 SMs
+    if (small_input_plan(plan, total, num_tensors, n_workers, elem_bytes, flags, 148 * kSmallBlocksPerSm, &seg_len))
         return 1;
     int n = 0;
     for (int l = 0; l < plan.num_levels; ++l) {
@@ -690,6 +767,49 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     if (total == 0 || num_tensors == 0)
         return ADASUM_OK;
     std::vector<const void*> operand_ptrs(grads, grads + n_workers);
+
+    // Inputs that fit the L2: one cooperative launch does both passes and HBM sees the operands once.
+    int small_seg_len = 0;
+    const int small_blocks = sharded ? 0 : resident_small_blocks();
+    if (small_blocks > 0 &&
+        small_input_plan(plan, total, num_tensors, n_workers, eb, flags, small_blocks, &small_seg_len)) {
+        const SegmentTable* tab = nullptr;
+        st = get_segment_table(offsets, num_tensors, small_seg_len, &tab);
+        if (st != ADASUM_OK)
+            return st;
+        if (tab->num_segments <= small_blocks) {
+            OperandTable table;
+            for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
+                table.ptr[i] = grads[i < n_workers ? i : 0];
+            FinishArgs fin;
+            fin.seg_first = tab->d_seg_first;
+            fin.counters = nullptr;
+            fin.weights = nullptr;
+            fin.tree = TreeOptions{(flags & ADASUM_FLAG_LINEAR_ORDER) ? 1 : 0, 1, 1, 1,
+                                   orthogonality ? reinterpret_cast<double*>(ws + lay.leaf_sums) : nullptr,
+                                   orthogonality};
+            float* partials = reinterpret_cast<float*>(ws + lay.partials);
+            const int radix = plan.level[0].radix;
+            cudaError_t err;
+            if (dtype == ADASUM_F32)
+                err = vec ? launch_fused_small_radix<float, true>(radix, table, n_workers, *tab, partials, fin, out, stream)
+                          : launch_fused_small_radix<float, false>(radix, table, n_workers, *tab, partials, fin, out, stream);
+            else if (dtype == ADASUM_F16)
+                err = vec ? launch_fused_small_radix<__half, true>(radix, table, n_workers, *tab, partials, fin, out, stream)
+                          : launch_fused_small_radix<__half, false>(radix, table, n_workers, *tab, partials, fin, out, stream);
+            else
+                err = vec ? launch_fused_small_radix<__nv_bfloat16, true>(radix, table, n_workers, *tab, partials, fin, out, stream)
+                          : launch_fused_small_radix<__nv_bfloat16, false>(radix, table, n_workers, *tab, partials, fin, out, stream);
+            if (err == cudaSuccess) {
+                profile_mark(stream, ADASUM_KERNEL_FUSED_SMALL, 0, radix, false);
+                return ADASUM_OK;
+            }
+            if (err != cudaErrorCooperativeLaunchTooLarge)
+                return fail(ADASUM_ERR_CUDA, "cooperative launch: %s", cudaGetErrorString(err));
+            (void)cudaGetLastError();       // too many blocks for this device after all: the two-pass path serves it
+        }
+    }
+
     for (int l = 0; l < plan.num_levels; ++l) {
         const Level& lv = plan.level[l];
         if (only_level >= 0 && l != only_level) {       // other levels' operands: the intermediates
@@ -922,7 +1042,7 @@ adasum_status_t adasum_plan_info(int64_t total_elems, int32_t num_tensors, int32
     if (num_levels)
         *num_levels = plan.num_levels;
     if (num_launches)
-        *num_launches = total_elems == 0 ? 0 : launches_of(plan, n_workers, flags);
+        *num_launches = total_elems == 0 ? 0 : launches_of(plan, n_workers, flags, total_elems, num_tensors, dtype_bytes(dtype));
     return ADASUM_OK;
 }
 

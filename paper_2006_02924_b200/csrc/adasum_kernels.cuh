@@ -21,6 +21,7 @@
 // deterministic and there is nothing that can spin.
 #pragma once
 
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <stdint.h>
@@ -216,19 +217,14 @@ __device__ __forceinline__ void gram_accumulate(const float (&x)[R], float (&acc
     }
 }
 
-// grid = (segments, groups in this launch); block = kThreads.
-// partials[(segment * groups_total + group_base + blockIdx.y) * E + entry]
+// The Gram matrix of one segment of the group whose first operand is ops.ptr[first], computed by
+// the whole block on the fp32 pipes and written to dst[0 .. E).
 template <typename T, int R, bool VEC>
-__global__ void __launch_bounds__(kThreads)
-gram_partial_kernel(const __grid_constant__ OperandTable ops, int operands,
-                    const Segment* __restrict__ segments, float* __restrict__ partials,
-                    int groups_total, int group_base, FinishArgs fin)
+__device__ __forceinline__ void gram_of_segment(const OperandTable& ops, int first, int members,
+                                                const Segment& seg, float* __restrict__ dst)
 {
     constexpr int E = gram_entries(R);
     constexpr int V = Element<T>::kVec;
-    const Segment seg = segments[blockIdx.x];
-    const int first = blockIdx.y * R;
-    const int members = min(R, operands - first);
 
     const T* src[R];
 #pragma unroll
@@ -291,7 +287,6 @@ gram_partial_kernel(const __grid_constant__ OperandTable ops, int operands,
             warp_sums[warp][k] = s;
     }
     __syncthreads();
-    float* dst = partials + ((int64_t)blockIdx.x * groups_total + group_base + blockIdx.y) * E;
     for (int k = threadIdx.x; k < E; k += kThreads) {
         float s = 0.0f;
 #pragma unroll
@@ -299,6 +294,22 @@ gram_partial_kernel(const __grid_constant__ OperandTable ops, int operands,
             s += warp_sums[w][k];
         dst[k] = s;
     }
+}
+
+// grid = (segments, groups in this launch); block = kThreads.
+// partials[(segment * groups_total + group_base + blockIdx.y) * E + entry]
+template <typename T, int R, bool VEC>
+__global__ void __launch_bounds__(kThreads)
+gram_partial_kernel(const __grid_constant__ OperandTable ops, int operands,
+                    const Segment* __restrict__ segments, float* __restrict__ partials,
+                    int groups_total, int group_base, FinishArgs fin)
+{
+    constexpr int E = gram_entries(R);
+    const Segment seg = segments[blockIdx.x];
+    const int first = blockIdx.y * R;
+    const int members = min(R, operands - first);
+    gram_of_segment<T, R, VEC>(ops, first, members, seg,
+                               partials + ((int64_t)blockIdx.x * groups_total + group_base + blockIdx.y) * E);
     finish_if_last<R>(fin, partials, seg.tensor, group_base + blockIdx.y, groups_total, members);
 }
 
@@ -981,39 +992,29 @@ __device__ __forceinline__ void decode_vector<__nv_bfloat16>(const uint4& v, flo
     }
 }
 
-// grid = (segments, groups in this launch); block = kThreads.
-// dst_base + (group_base + blockIdx.y) * dst_stride is the group's output buffer (fp32).
-// Rows are read eight at a time so that the loads of one batch are in flight together while the
-// register count stays low enough for three blocks per SM.
+// The weighted sum of one segment, dst[e] = sum_i w_i x_i[e], by the whole block.  wsrc[0 .. R)
+// are the leaf weights (global or shared memory).  Rows are read eight at a time so that the
+// loads of one batch are in flight together while the register count stays low enough for three
+// blocks per SM.
 template <typename T, int R, bool VEC>
-__global__ void __launch_bounds__(kThreads, 3)
-weighted_sum_kernel(const __grid_constant__ OperandTable ops, int operands,
-                    const Segment* __restrict__ segments, const float* __restrict__ weights,
-                    int groups_total, int group_base, float* __restrict__ dst_base,
-                    int64_t dst_stride)
+__device__ __forceinline__ void weighted_sum_of_segment(const OperandTable& ops, int first, int members,
+                                                        const Segment& seg, const float* wsrc,
+                                                        float* __restrict__ dst)
 {
     constexpr int V = Element<T>::kVec;
     constexpr int BATCH = R < 8 ? R : 8;
-    // Segments are taken last to first: pass 1 walked them first to last, so the tail of the
-    // operands is what the L2 still holds when this kernel starts.
-    const Segment seg = segments[gridDim.x - 1 - blockIdx.x];
-    const int first = blockIdx.y * R;
-    const int members = min(R, operands - first);
-    const int group = group_base + blockIdx.y;
-
     // leaf weights: registers for small groups, shared memory for the wide ones
     constexpr bool W_IN_SMEM = R > 16;
     __shared__ float w_smem[W_IN_SMEM ? R : 1];
     float w_reg[W_IN_SMEM ? 1 : R];
-    const float* wsrc = weights + ((int64_t)seg.tensor * groups_total + group) * R;
     if constexpr (W_IN_SMEM) {
         if (threadIdx.x < R)
-            w_smem[threadIdx.x] = threadIdx.x < members ? __ldg(wsrc + threadIdx.x) : 0.0f;
+            w_smem[threadIdx.x] = threadIdx.x < members ? wsrc[threadIdx.x] : 0.0f;
         __syncthreads();
     } else {
 #pragma unroll
         for (int i = 0; i < R; ++i)
-            w_reg[i] = i < members ? __ldg(wsrc + i) : 0.0f;
+            w_reg[i] = i < members ? wsrc[i] : 0.0f;
     }
     auto w = [&](int i) -> float {
         if constexpr (W_IN_SMEM)
@@ -1021,7 +1022,6 @@ weighted_sum_kernel(const __grid_constant__ OperandTable ops, int operands,
         else
             return w_reg[i];
     };
-    float* dst = dst_base + (int64_t)group * dst_stride;
 
     const int64_t begin = seg.begin, end = seg.begin + seg.len;
     int64_t body_begin, body_end;
@@ -1069,6 +1069,60 @@ weighted_sum_kernel(const __grid_constant__ OperandTable ops, int operands,
             dst[e] = y;
         }
     }
+}
+
+// grid = (segments, groups in this launch); block = kThreads.
+// dst_base + (group_base + blockIdx.y) * dst_stride is the group's output buffer (fp32).
+template <typename T, int R, bool VEC>
+__global__ void __launch_bounds__(kThreads, 3)
+weighted_sum_kernel(const __grid_constant__ OperandTable ops, int operands,
+                    const Segment* __restrict__ segments, const float* __restrict__ weights,
+                    int groups_total, int group_base, float* __restrict__ dst_base,
+                    int64_t dst_stride)
+{
+    // Segments are taken last to first: pass 1 walked them first to last, so the tail of the
+    // operands is what the L2 still holds when this kernel starts.
+    const Segment seg = segments[gridDim.x - 1 - blockIdx.x];
+    const int first = blockIdx.y * R;
+    const int members = min(R, operands - first);
+    const int group = group_base + blockIdx.y;
+    weighted_sum_of_segment<T, R, VEC>(ops, first, members, seg,
+                                       weights + ((int64_t)seg.tensor * groups_total + group) * R,
+                                       dst_base + (int64_t)group * dst_stride);
+}
+
+// ---- both passes in one launch, for inputs that fit the L2 -------------------------------------
+//
+// One level, one group (n_workers <= 8), few enough segments that every block of the grid is
+// resident at the same time (cooperative launch).  Each block forms the Gram matrix of its
+// segment, the grid synchronises, each block adds up its tensor's partial matrices and derives
+// the weights for itself (the same numbers in every block of a tensor: fixed summation order),
+// and then writes the weighted sum of the segment it has just read, which the 126 MB L2 still
+// holds.  HBM sees the operands once.
+// grid = segments; block = kThreads; partials[segment * E + entry].
+template <typename T, int R, bool VEC>
+__global__ void __launch_bounds__(kThreads, (sizeof(T) == 2 && R == 8) ? 2 : 3)
+fused_small_kernel(const __grid_constant__ OperandTable ops, int operands,
+                   const Segment* __restrict__ segments, float* __restrict__ partials, FinishArgs fin,
+                   float* __restrict__ out)
+{
+    constexpr int E = gram_entries(R);
+    const Segment seg = segments[blockIdx.x];
+    const int members = min(R, operands);
+    gram_of_segment<T, R, VEC>(ops, 0, members, seg, partials + (int64_t)blockIdx.x * E);
+    __threadfence();
+    cooperative_groups::this_grid().sync();
+
+    __shared__ float leaf_weights[R];
+    const int s0 = fin.seg_first[2 * seg.tensor], s1 = fin.seg_first[2 * seg.tensor + 1];
+    TreeOptions opt = fin.tree;
+    if ((int)blockIdx.x != s0) {           // one block per tensor reports the by-products
+        opt.leaf_norm_sums = nullptr;
+        opt.orthogonality = nullptr;
+    }
+    finish_group_in_block<R>(partials, s0, s1, seg.tensor, 0, 1, members, leaf_weights, opt);
+    __syncthreads();
+    weighted_sum_of_segment<T, R, VEC>(ops, 0, members, seg, leaf_weights, out);
 }
 
 // n_workers = 1: the result is the input, converted to fp32.
