@@ -36,10 +36,11 @@ NOMINAL_HBM_GBS = 8000.0
 # kernels as built from the source whose fingerprint is recorded with them; see profiles/.
 # {(workload, kernel, level): bytes}.  Reported only while the kernel source is unchanged.
 NCU_TRAFFIC = {
-    "fingerprint": "072e5b354eb33ba7",
+    "fingerprint": "114ce3fee93026d4",
     "bytes": {
-        "c2/gram_partial/0": 822188032,      # profiles/gram_partial_f32_r8_c2.txt
-        "c2/weighted_sum/0": 874497024,      # profiles/weighted_sum_f32_r8_c2.txt
+        "c2/gram_partial/0": 821598208,      # profiles/gram_partial_mma_f32_r8_c2.txt
+        "c2/weighted_sum/0": 872890880,      # profiles/weighted_sum_f32_r8_c2.txt
+        "c1/fused_small/0": 8037632,         # profiles/fused_small_f32_r2_c1.txt
     },
 }
 
@@ -150,6 +151,8 @@ def algorithmic_bytes(record, plan_levels, total_elems, in_bytes):
         return read
     if record["kernel"] == "weighted_sum":
         return read + level["groups"] * total_elems * 4
+    if record["kernel"] == "fused_small":      # both passes in one launch: HBM sees the operands once
+        return read + total_elems * 4
     if record["kernel"] == "convert":
         return total_elems * (in_bytes + 4)
     return 0

@@ -43,6 +43,8 @@ def test_algorithmic_bytes_per_launch():
     assert bench.algorithmic_bytes({"kernel": "gram_partial", "level": 1}, levels, p, 2) == 16 * p * 4
     assert bench.algorithmic_bytes({"kernel": "weighted_sum", "level": 1}, levels, p, 2) == 16 * p * 4 + p * 4
     assert bench.algorithmic_bytes({"kernel": "tree_weights", "level": 0}, levels, p, 2) == 0
+    one = [{"radix": 2, "operands": 2, "groups": 1}]
+    assert bench.algorithmic_bytes({"kernel": "fused_small", "level": 0}, one, p, 4) == 2 * p * 4 + p * 4
 
 
 def test_oracle_sample_is_bounded_and_whole_tensors():
