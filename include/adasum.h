@@ -89,7 +89,10 @@ typedef enum {
  *                result depends on all earlier workers, so the whole reduce is one level whose
  *                Gram matrix covers every worker: n_workers <= 32 for fp32 inputs, <= 64 for
  *                fp16 / bf16; the radix fields must be 0.  Otherwise ADASUM_ERR_ARG.
+ *   bit 19       ADASUM_FLAG_NO_TCGEN05: form radix-64 Gram matrices with warp-level mma.sync
+ *                instead of tcgen05 and tensor memory; for comparison and debugging
  */
+#define ADASUM_FLAG_NO_TCGEN05 (1u << 19)
 #define ADASUM_FLAG_SIMPLE_KERNELS (1u << 16)
 #define ADASUM_FLAG_SEPARATE_FINISH (1u << 17)
 #define ADASUM_FLAG_LINEAR_ORDER (1u << 18)
@@ -237,6 +240,18 @@ adasum_status_t adasum_pair(const void* a, const void* b, const int64_t* tensor_
 
 adasum_status_t adasum_pair_noalloc(const void* a, const void* b, const int64_t* tensor_offsets,
                                     int32_t num_tensors, adasum_dtype_t dtype, float* out, void* stream);
+
+/*
+ * Device-side status of the last reduce that used this workspace (the paper has no counterpart).
+ * The radix-64 tensor-memory kernel waits, with a limit, for the tensor core to release a
+ * shared-memory stage; if such a wait ever runs out, the kernel records it and finishes (with
+ * wrong numbers) instead of hanging.  This call copies that record back: it synchronises `stream`
+ * and returns ADASUM_OK, ADASUM_ERR_TIMEOUT, or an argument / CUDA error.  Arguments as for the
+ * reduce that is being asked about.
+ */
+adasum_status_t adasum_device_status(int64_t total_elems, int32_t num_tensors, int32_t n_workers,
+                                     adasum_dtype_t dtype, uint32_t flags, const void* workspace,
+                                     void* stream);
 
 /* Static, human-readable name of a status code. */
 const char* adasum_status_string(adasum_status_t status);

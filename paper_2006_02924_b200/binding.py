@@ -24,6 +24,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 
 ADASUM_F32, ADASUM_F16, ADASUM_BF16 = 0, 1, 2
 ADASUM_FLAG_SIMPLE_KERNELS, ADASUM_FLAG_SEPARATE_FINISH, ADASUM_FLAG_LINEAR_ORDER = 1 << 16, 1 << 17, 1 << 18
+ADASUM_FLAG_NO_TCGEN05 = 1 << 19
 ADASUM_OK = 0
 ADASUM_MAX_WORKERS = 4096
 ADASUM_MAX_LEVELS = 12
@@ -97,6 +98,19 @@ def adasum_plan_info(total_elems: int, num_tensors: int, n_workers: int, dtype, 
     if status != ADASUM_OK:
         raise AdasumError(status)
     return {"radices": [int(radices[i]) for i in range(levels.value)], "launches": int(launches.value)}
+
+
+_lib.adasum_device_status.restype = ctypes.c_int
+_lib.adasum_device_status.argtypes = [ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int, ctypes.c_uint32,
+                                      ctypes.c_void_p, ctypes.c_void_p]
+
+
+def adasum_device_status(total_elems: int, num_tensors: int, n_workers: int, dtype, workspace, flags: int = 0,
+                         stream=None) -> int:
+    """``adasum_device_status`` of the C ABI: 0, or 7 (ADASUM_ERR_TIMEOUT) if a bounded device-side
+    wait of the last reduce on ``workspace`` ran out.  Synchronises the stream."""
+    return int(_lib.adasum_device_status(int(total_elems), int(num_tensors), int(n_workers), _dtype_code(dtype),
+                                         int(flags), workspace.data_ptr(), _stream_handle(stream)))
 
 
 def _dtype_code(dtype) -> int:

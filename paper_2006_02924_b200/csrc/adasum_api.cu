@@ -134,7 +134,7 @@ struct LevelPlan {
 bool plan_levels(int n_workers, adasum_dtype_t dtype, uint32_t flags, LevelPlan* plan)
 {
     const int first = (int)(flags & 0xffu), later_flag = (int)((flags >> 8) & 0xffu);
-    if ((flags >> 19) != 0)
+    if ((flags >> 20) != 0)
         return false;
     if (first != 0 && (!valid_radix(first) || first > max_radix_for(dtype)))
         return false;
@@ -171,8 +171,11 @@ bool plan_levels(int n_workers, adasum_dtype_t dtype, uint32_t flags, LevelPlan*
         int radix = want;
         if (radix == 0) {
             // Measured on B200: the tensor-core Gram pass keeps up with HBM at radix 16 for fp32
-            // operands and at radix 32 for fp16 / bf16; beyond that it is bound by the tensor pipe.
+            // operands and at radix 32 for fp16 / bf16; beyond that mma.sync is bound by the tensor pipe.
             radix = (first_level && dtype != ADASUM_F32) ? 32 : 16;
+            // fp16 / bf16 workers in complete groups of 64: the tcgen05 kernel, one level less
+            if (first_level && dtype != ADASUM_F32 && m % 64 == 0 && !(flags & ADASUM_FLAG_NO_TCGEN05))
+                radix = 64;
             radix = radix < cap_auto ? radix : cap_auto;
         }
         if (radix > pow2_ceil(m))
@@ -213,8 +216,8 @@ Layout make_layout(const LevelPlan& plan, int64_t total_elems, int32_t num_tenso
             lay.partials_bytes = p;
         if (w > lay.weights_bytes)
             lay.weights_bytes = w;
-        const size_t c = (size_t)(num_tensors > 0 ? num_tensors : 1) * lv.groups * sizeof(int);
-        if (c > lay.counters_bytes)
+        const size_t c = ((size_t)(num_tensors > 0 ? num_tensors : 1) * lv.groups + 1) * sizeof(int);
+        if (c > lay.counters_bytes)       // + 1: the device status word sits after the ticket counters
             lay.counters_bytes = c;
         const size_t g64 = (size_t)(num_tensors > 0 ? num_tensors : 1) * lv.groups * gram_entries(lv.radix) *
                            sizeof(double);
@@ -379,8 +382,22 @@ cudaError_t allow_dynamic_smem(Kernel kernel, size_t bytes, bool (&configured)[6
 template <typename T, int R, bool VEC>
 cudaError_t launch_gram(GramKind kind, const OperandTable& ops, int operands, int groups_here,
                         const SegmentTable& tab, float* partials, int groups_total, int group_base,
-                        const FinishArgs& fin, cudaStream_t stream)
+                        const FinishArgs& fin, cudaStream_t stream, int* tc_status = nullptr)
 {
+    if constexpr (R == 64 && VEC && sizeof(T) == 2) {
+        // every group complete: the tcgen05 kernel (64 x 64 accumulator in tensor memory)
+        if (kind == GRAM_MMA && tc_status != nullptr && operands == groups_here * 64) {
+            auto kernel = gram_partial_tc64_kernel<T>;
+            static bool configured[64] = {};
+            cudaError_t err = allow_dynamic_smem(kernel, kTcSmemBytes, configured);
+            if (err != cudaSuccess)
+                return err;
+            dim3 grid((unsigned)tab.num_segments, (unsigned)groups_here);
+            kernel<<<grid, kTcThreads, kTcSmemBytes, stream>>>(ops, operands, tab.d_segments, partials, groups_total,
+                                                               group_base, fin, tc_status);
+            return cudaSuccess;
+        }
+    }
     if constexpr (R >= 8) {
         if (kind == GRAM_MMA) {
             if constexpr (R <= 32 || sizeof(T) == 2) {
@@ -541,6 +558,7 @@ struct LevelArgs {
     int* counters;      // ticket counters for finishing inside pass 1, or nullptr
     TreeOptions tree;
     LevelPhase phase;
+    int* tc_status;     // status word for the tcgen05 kernel, or nullptr to keep to mma.sync
     double* gram64;
     float* weights;
     float* dst;
@@ -567,7 +585,7 @@ adasum_status_t run_level_typed(const LevelArgs& a)
             table.ptr[i] = a.operand_ptrs[op0 + (i < ops_here ? i : 0)];
         if (a.vec)
             ADASUM_CUDA_CHECK((launch_gram<T, R, true>(a.kind, table, ops_here, groups_here, *a.gram_tab,
-                                                       a.partials, a.groups, g0, fin, a.stream)));
+                                                       a.partials, a.groups, g0, fin, a.stream, a.tc_status)));
         else
             ADASUM_CUDA_CHECK((launch_gram<T, R, false>(a.kind, table, ops_here, groups_here, *a.gram_tab,
                                                         a.partials, a.groups, g0, fin, a.stream)));
@@ -747,7 +765,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
 
     char* ws = static_cast<char*>(workspace);
     const bool separate_finish = (flags & ADASUM_FLAG_SEPARATE_FINISH) != 0 || sharded;
-    if (!separate_finish && lay.counters_bytes > 0)     // the workspace arrives with unknown contents
+    if (lay.counters_bytes > 0 && phase != PHASE_APPLY)      // the workspace arrives with unknown contents
         ADASUM_CUDA_CHECK(cudaMemsetAsync(ws + lay.counters, 0, lay.counters_bytes, stream));
     if (orthogonality && num_tensors > 0 && (!sharded || (phase == PHASE_APPLY && only_level == 0)))
         ADASUM_CUDA_CHECK(cudaMemsetAsync(orthogonality, 0xff, sizeof(float) * (size_t)num_tensors, stream));
@@ -845,6 +863,10 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         a.gram64 = reinterpret_cast<double*>(ws + lay.gram64);
         a.counters = separate_finish ? nullptr : reinterpret_cast<int*>(ws + lay.counters);
         a.phase = phase;
+        // the status word is the last int of the (zeroed) counter region
+        a.tc_status = (flags & ADASUM_FLAG_NO_TCGEN05)
+                          ? nullptr
+                          : reinterpret_cast<int*>(ws + lay.counters + lay.counters_bytes - sizeof(int));
         a.tree.linear = (flags & ADASUM_FLAG_LINEAR_ORDER) ? 1 : 0;
         a.tree.level_is_first = l == 0;
         a.tree.level_is_last = l + 1 == plan.num_levels;
@@ -1097,6 +1119,34 @@ adasum_status_t adasum_pair_noalloc(const void* a, const void* b, const int64_t*
 {
     return adasum::pair_noalloc_impl(a, b, tensor_offsets, num_tensors, dtype, out,
                                      static_cast<cudaStream_t>(stream));
+}
+
+adasum_status_t adasum_device_status(int64_t total_elems, int32_t num_tensors, int32_t n_workers,
+                                     adasum_dtype_t dtype, uint32_t flags, const void* workspace, void* stream)
+{
+    using namespace adasum;
+    g_error[0] = '\0';
+    if (!workspace)
+        return fail(ADASUM_ERR_NULL, "workspace is NULL");
+    if (total_elems < 0 || num_tensors < 0 || n_workers < 1 || n_workers > ADASUM_MAX_WORKERS)
+        return fail(ADASUM_ERR_ARG, "invalid sizes");
+    if (dtype != ADASUM_F32 && dtype != ADASUM_F16 && dtype != ADASUM_BF16)
+        return fail(ADASUM_ERR_DTYPE, "unknown dtype %d", (int)dtype);
+    LevelPlan plan;
+    if (!plan_levels(n_workers, dtype, flags, &plan))
+        return fail(ADASUM_ERR_ARG, "invalid flags 0x%x", flags);
+    const Layout lay = make_layout(plan, total_elems, num_tensors);
+    if (lay.counters_bytes < sizeof(int))
+        return ADASUM_OK;
+    int word = 0;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    ADASUM_CUDA_CHECK(cudaMemcpyAsync(&word, static_cast<const char*>(workspace) + lay.counters + lay.counters_bytes -
+                                                 sizeof(int),
+                                      sizeof(int), cudaMemcpyDeviceToHost, s));
+    ADASUM_CUDA_CHECK(cudaStreamSynchronize(s));
+    if (word == ADASUM_DEVICE_TIMEOUT)
+        return fail(ADASUM_ERR_TIMEOUT, "a bounded wait on the tensor core ran out");
+    return ADASUM_OK;
 }
 
 const char* adasum_status_string(adasum_status_t status)

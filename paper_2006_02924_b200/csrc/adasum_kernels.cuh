@@ -32,6 +32,7 @@ constexpr int kThreads = 256;               // threads per block of the streamin
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxOperandsPerLaunch = 256;  // operand pointers carried in one kernel argument
 constexpr int kMaxRadix = 64;
+constexpr int ADASUM_DEVICE_TIMEOUT = 7;    // value of ADASUM_ERR_TIMEOUT, written to a status word by a kernel
 
 // A contiguous run of elements of one tensor inside the fused buffers.
 struct Segment {
@@ -709,6 +710,254 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
         dst[gram_index(R, i, j)] = v;
     }
     finish_if_last<R>(fin, partials, seg.tensor, group_base + blockIdx.y, groups_total, members);
+}
+
+// ---- pass 1 for groups of 64 fp16 / bf16 rows: tcgen05 ------------------------------------------
+//
+// At radix 64 the warp-level mma.sync path is bound by the tensor pipe.  The fifth-generation
+// tensor core instruction takes both operands straight from shared memory and keeps the 64 x 64
+// fp32 accumulator in tensor memory, so one thread issues a whole tile's multiplications and the
+// other threads only move data.
+//
+// Tile = 64 rows x 1024 bytes (8 K-blocks of 64 elements), 64 KB, copied with coalesced cp.async
+// (a warp moves 512 contiguous bytes of one row per instruction), laid out as eight
+// [64 rows x 128 bytes] blocks in the 128-byte-swizzle K-major form the instruction's
+// shared-memory descriptor expects: 16-byte chunk c of row r of a block sits at
+// r * 128 + ((c ^ (r & 7)) * 16).  A and B are the SAME block (X X^T): M = N = 64, K = 16 per
+// instruction, 32 instructions per tile.  With M = 64 the accumulator's rows 16 q .. 16 q + 15
+// live in tensor-memory lanes 32 q .. 32 q + 15.
+//
+// Roles: all warps but the last copy (each warp whole half-rows), lane 0 of the last warp
+// multiplies.  Per stage two mbarriers: `full` (the copying threads arrive when their pieces of
+// the tile have landed and are fenced for the tensor core) and `empty` (the tensor core arrives
+// when the multiplications that read the stage are done).  No block-wide barrier inside the loop.
+//
+// Every wait is bounded; if one runs out the thread records ADASUM_ERR_TIMEOUT in *status, stops
+// waiting and keeps going (its block's numbers are then wrong, but every access stays in bounds),
+// the block frees its tensor memory and returns.
+
+constexpr int kTcKBlocks = 8;                 // K-blocks (64 elements, 128 bytes of a row) per tile
+constexpr int kTcStages = 3;
+constexpr int kTcAhead = kTcStages - 1;       // tiles in flight
+constexpr int kTcThreads = 512;
+constexpr int kTcProducerWarps = kTcThreads / 32 - 1;
+constexpr int kTcProducers = kTcProducerWarps * 32;
+constexpr int kTcHalfRows = 64 * kTcKBlocks / 4;                 // 512-byte pieces of rows per tile
+constexpr int kTcRowsPerWarp = (kTcHalfRows + kTcProducerWarps - 1) / kTcProducerWarps;
+constexpr int kTcTileBytes = kTcKBlocks * 8192;
+constexpr int kTcPadBytes = 8 * 1024;         // slack after the last stage
+constexpr size_t kTcSmemBytes = (size_t)kTcStages * kTcTileBytes + kTcPadBytes + 1024;   // + room to align to 1024
+constexpr uint32_t kTcSpinLimit = 1u << 22;   // about a tenth of a second; a real wait is microseconds
+
+__device__ __forceinline__ uint32_t mbarrier_try_wait_parity(uint32_t bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done)
+                 : "r"(bar), "r"(parity)
+                 : "memory");
+    return done;
+}
+
+// Returns false if the barrier did not complete the phase within the spin limit.
+__device__ __forceinline__ bool mbarrier_wait_bounded(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t spin = 0; spin < kTcSpinLimit; ++spin)
+        if (mbarrier_try_wait_parity(bar, parity))
+            return true;
+    return false;
+}
+
+__device__ __forceinline__ void mbarrier_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t tc_smem_descriptor(uint32_t smem_addr)
+{
+    const uint64_t start = (uint64_t)((smem_addr & 0x3ffffu) >> 4);          // bits 0..13
+    const uint64_t leading = (uint64_t)1 << 16;                              // bits 16..29: unused with this swizzle
+    const uint64_t stride = (uint64_t)(1024 >> 4) << 32;                     // bits 32..45: stride byte offset
+    const uint64_t version = (uint64_t)1 << 46;                              // descriptor version of this architecture
+    const uint64_t swizzle_128b = (uint64_t)2 << 61;                         // bits 61..63: layout type
+    return start | leading | stride | version | swizzle_128b;
+}
+
+// grid = (segments, groups in this launch); block = kTcThreads; dynamic shared memory = kTcSmemBytes.
+// Only for 16-byte aligned operands and launches in which every group has all 64 members.
+template <typename T>
+__global__ void __launch_bounds__(kTcThreads, 1)
+gram_partial_tc64_kernel(const __grid_constant__ OperandTable ops, int operands,
+                         const Segment* __restrict__ segments, float* __restrict__ partials,
+                         int groups_total, int group_base, FinishArgs fin, int* __restrict__ status)
+{
+    static_assert(sizeof(T) == 2, "fp16 / bf16 only");
+    constexpr int R = 64;
+    constexpr int E = gram_entries(R);
+    constexpr int V = 8;                                   // elements per 16-byte piece
+    constexpr int TILE_ELEMS = 64 * kTcKBlocks;            // elements of one row in a tile
+    extern __shared__ __align__(1024) unsigned char tc_smem_raw[];
+    __shared__ __align__(8) unsigned long long full_bar[kTcStages], empty_bar[kTcStages];
+    __shared__ uint32_t tmem_base_slot;
+
+    const Segment seg = segments[blockIdx.x];
+    const int first = blockIdx.y * R;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    const int64_t begin = seg.begin, end = seg.begin + seg.len;
+    const int64_t k0 = begin / V * V;
+    const int ntiles = (int)((end - k0 + TILE_ELEMS - 1) / TILE_ELEMS);
+
+    // stage memory, aligned to the 1024 bytes the swizzle pattern repeats with
+    const uint32_t raw_base = static_cast<uint32_t>(__cvta_generic_to_shared(tc_smem_raw));
+    const uint32_t smem_base = (raw_base + 1023u) & ~1023u;
+    const uint32_t full0 = static_cast<uint32_t>(__cvta_generic_to_shared(&full_bar[0]));
+    const uint32_t empty0 = static_cast<uint32_t>(__cvta_generic_to_shared(&empty_bar[0]));
+
+    // ---- set-up: barriers, tensor memory (64 columns of fp32 accumulator)
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int st = 0; st < kTcStages; ++st) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full0 + 8 * st), "r"(kTcProducers));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(empty0 + 8 * st));
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 64;" ::"r"(
+            static_cast<uint32_t>(__cvta_generic_to_shared(&tmem_base_slot))));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_acc = tmem_base_slot;
+
+    bool timed_out = false;
+    if (warp < kTcProducerWarps) {
+        // ---- copying warps: warp w moves rows w, w + 7, ...; lane = 16-byte chunk of the 512-byte row
+        const T* copy_src[kTcRowsPerWarp];
+        uint32_t copy_off[kTcRowsPerWarp];
+#pragma unroll
+        for (int i = 0; i < kTcRowsPerWarp; ++i) {
+            // 512-byte piece h of the tile: row h / (pieces per row), chunks 32 (h % pieces per row) + lane
+            const int h = warp + kTcProducerWarps * i;
+            const int hh = h < kTcHalfRows ? h : 0;
+            const int r = hh / (kTcKBlocks / 4), chunk = (hh % (kTcKBlocks / 4)) * 32 + lane;
+            copy_src[i] = static_cast<const T*>(ops.ptr[first + r]) + chunk * V;
+            copy_off[i] = (chunk >> 3) * 8192 + r * 128 + (((chunk & 7) ^ (r & 7)) << 4);
+        }
+        auto issue_copy = [&](int tile) {
+            if (tile < ntiles) {
+                const int stage = tile % kTcStages;
+                if (tile >= kTcStages && !timed_out) {
+                    // the multiplications of tile - S read this stage: wait for the tensor core
+                    if (!mbarrier_wait_bounded(empty0 + 8 * stage, (uint32_t)((tile / kTcStages - 1) & 1)))
+                        timed_out = true;
+                }
+                const uint32_t dst = smem_base + stage * kTcTileBytes;
+                const int64_t tile_elem0 = k0 + (int64_t)tile * TILE_ELEMS;
+                const bool interior = tile_elem0 >= begin && tile_elem0 + TILE_ELEMS <= end;
+#pragma unroll
+                for (int i = 0; i < kTcRowsPerWarp; ++i) {
+                    const int h = warp + kTcProducerWarps * i;
+                    if (h < kTcHalfRows) {
+                        const int chunk = (h % (kTcKBlocks / 4)) * 32 + lane;
+                        const int64_t e0 = tile_elem0 + (int64_t)chunk * V;
+                        if (interior || (e0 >= begin && e0 + V <= end))
+                            cp_async_16B_shared(dst + copy_off[i], copy_src[i] + tile_elem0);
+                        else
+                            store_shared_16B(dst + copy_off[i],
+                                             load_masked_words<T>(copy_src[i] - chunk * V, e0, begin, end));
+                    }
+                }
+            }
+            cp_async_commit();
+        };
+#pragma unroll
+        for (int tile = 0; tile < kTcAhead; ++tile)
+            issue_copy(tile);
+        for (int tile = 0; tile < ntiles; ++tile) {
+            cp_async_wait<kTcAhead - 1>();                                 // this thread's pieces of `tile` have landed
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // ... and are visible to the tensor core
+            mbarrier_arrive(full0 + 8 * (tile % kTcStages));
+            issue_copy(tile + kTcAhead);
+        }
+        cp_async_wait<0>();
+    } else if (lane == 0) {
+        // ---- multiplying thread
+        // instruction descriptor: fp32 accumulator, A and B of type T, both K-major, N = 64, M = 64
+        constexpr uint32_t kFormat = __is_same(T, __half) ? 0u : 1u;     // 0 = fp16, 1 = bf16
+        constexpr uint32_t kInstr =
+            (1u << 4) | (kFormat << 7) | (kFormat << 10) | ((64u >> 3) << 17) | ((64u >> 4) << 24);
+        for (int tile = 0; tile < ntiles; ++tile) {
+            const int stage = tile % kTcStages;
+            if (!timed_out && !mbarrier_wait_bounded(full0 + 8 * stage, (uint32_t)((tile / kTcStages) & 1)))
+                timed_out = true;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t tile_base = smem_base + stage * kTcTileBytes;
+#pragma unroll
+            for (int kb = 0; kb < kTcKBlocks; ++kb) {
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    // K-block kb, elements 16 ks .. 16 ks + 15 of it: 32 bytes further into the swizzled rows
+                    const uint64_t desc = tc_smem_descriptor(tile_base + kb * 8192 + ks * 32);
+                    const uint32_t accumulate = (tile > 0 || kb > 0 || ks > 0) ? 1u : 0u;
+                    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                                 ::"r"(tmem_acc), "l"(desc), "l"(desc), "r"(kInstr), "r"(accumulate)
+                                 : "memory");
+                }
+            }
+            // arrives on the barrier once everything issued so far has finished reading shared memory
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                             empty0 + 8 * stage)
+                         : "memory");
+        }
+    }
+
+    // ---- epilogue: wait for the last tile's multiplications, read the accumulator rows 0..63
+    {
+        const int last = ntiles - 1;
+        if (!timed_out &&
+            !mbarrier_wait_bounded(empty0 + 8 * (last % kTcStages), (uint32_t)((last / kTcStages) & 1)))
+            timed_out = true;
+    }
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (timed_out)
+        atomicExch(status, (int)ADASUM_DEVICE_TIMEOUT);
+    float* dst = partials + ((int64_t)blockIdx.x * groups_total + group_base + blockIdx.y) * E;
+    if (warp < 4) {
+        // With M = 64 the accumulator's rows 16 w .. 16 w + 15 live in tensor-memory lanes
+        // 32 w .. 32 w + 15, which are the lanes warp w may read: lane l < 16 of warp w gets row
+        // 16 w + l, 16 columns at a time.
+        const int i = 16 * warp + lane;
+#pragma unroll
+        for (int cb = 0; cb < 4; ++cb) {
+            uint32_t r[16];
+            const uint32_t taddr = tmem_acc + ((uint32_t)(32 * warp) << 16) + cb * 16;
+            asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                         : "r"(taddr)
+                         : "memory");
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (lane < 16) {
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    const int j = cb * 16 + c;
+                    if (j >= i)
+                        dst[gram_index(R, i, j)] = __uint_as_float(r[c]);
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 64;" ::"r"(tmem_acc) : "memory");
+    finish_if_last<R>(fin, partials, seg.tensor, group_base + blockIdx.y, groups_total, R);
 }
 
 // ---- coefficients: the binary tree evaluated on a Gram matrix ---------------------------------

@@ -78,9 +78,11 @@ def test_plan_info(binding):
     assert info(0, 0, 4, "f32")["launches"] == 0
     assert info(100, 1, 8, "f32", binding.flags_radix(2, 2))["launches"] == 6
     assert info(100, 1, 8, "f32", binding.flags_radix(2, 2) | (1 << 17))["launches"] == 9
-    assert info(100, 1, 64, "f16")["radices"] == [32, 2]
-    assert info(100, 1, 64, "f16")["launches"] == 4
-    assert info(100, 1, 64, "f16", 1 << 17)["launches"] == 4 + 3
+    assert info(100, 1, 64, "f16")["radices"] == [64]
+    assert info(100, 1, 64, "f16", 1 << 19)["radices"] == [32, 2]
+    assert info(100, 1, 48, "f16")["radices"] == [32, 2]
+    assert info(100, 1, 64, "f16", 1 << 19)["launches"] == 4
+    assert info(100, 1, 64, "f16", (1 << 17) | (1 << 19))["launches"] == 4 + 3
     assert info(100, 1, 256, "f32")["radices"] == [16, 16]
 
 

@@ -131,3 +131,25 @@ def test_reduce_can_be_replayed_from_a_cuda_graph(lib):
     ref = oracle.adasum_reduce([_np(g, "f32") for g in grads], offsets=offsets, threads=0)
     got = out.cpu().numpy().astype(np.float64)
     assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-5
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("n", [64, 128])
+def test_radix_64_tensor_memory_kernel(lib, dtype, n):
+    """Complete groups of 64 fp16 / bf16 workers go through the tcgen05 kernel: same result as the
+    mma.sync kernel (flag bit 19) and as the oracle; no device-side wait ran out."""
+    offsets = workloads.offsets_from_sizes([70_000, 9, 4097, 1, 64, 33_000])
+    total = int(offsets[-1])
+    grads = _correlated(n, total, dtype, seed=1500 + n)
+    flags = lib.flags_radix(64, 0)
+    need = lib.adasum_workspace_bytes(total, 6, n, dtype, flags)
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    out = lib.adasum_reduce(grads, offsets, workspace=ws, flags=flags)
+    assert lib.adasum_device_status(total, 6, n, dtype, ws, flags=flags) == 0
+    other = lib.adasum_reduce(grads, offsets, flags=flags | (1 << 19))
+    ref = oracle.adasum_reduce([_np(g, dtype) for g in grads], offsets=offsets, dtype=dtype, threads=0)
+    got = out.cpu().numpy().astype(np.float64)
+    for t in (0, 2, 4, 5):
+        lo, hi = int(offsets[t]), int(offsets[t + 1])
+        assert np.linalg.norm(got[lo:hi] - ref[lo:hi]) / np.linalg.norm(ref[lo:hi]) <= 2e-3, t
+    assert float(torch.linalg.norm(out - other) / torch.linalg.norm(other)) <= 1e-4
