@@ -2,7 +2,8 @@
 C-ABI library, with a thin Python binding.
 
 ``workloads`` (synthetic inputs) imports without the native library; every compute entry point
-lives in ``binding`` and raises if the library has not been built.
+lives in ``binding`` and raises if the library has not been built.  ``rvh`` runs the reduce with
+one gradient per GPU over a torch.distributed group (recursive vector halving).
 """
 
 _BINDING_NAMES = (
