@@ -208,6 +208,50 @@ def time_reduce(lib, wl, steps, warmup, flags, world=1, sampler=None, flush=True
     return ms, out, ws
 
 
+def time_variants(lib, wl, steps, warmup, flags):
+    """The same workload through adasum_reduce_delta: with a start buffer (the optimizer-delta form,
+    result written over the start buffer) and with bf16 output.  Per-step events, L2 flushed."""
+    dev = wl.grads[0].device
+    dt = wl.grads[0].dtype
+    need = lib.adasum_workspace_bytes(wl.total_elems, wl.num_tensors, wl.n_workers, wl.spec.dtype, flags)
+    ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+    scrub = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(workloads.BASE_SEED + 99)
+    params = torch.randn(wl.total_elems, generator=gen, device=dev).to(dt)
+    out16 = torch.empty(wl.total_elems, dtype=torch.bfloat16, device=dev)
+    b = workloads.DTYPE_BYTES[wl.spec.dtype]
+    cases = [
+        ("delta form, parameters updated in place",
+         lambda: lib.adasum_reduce_delta(wl.grads, params, wl.offsets, out=params, workspace=ws, flags=flags,
+                                         stream=stream),
+         2 * (wl.n_workers + 1) * wl.total_elems * b + wl.total_elems * b),
+        ("plain reduce, bf16 output",
+         lambda: lib.adasum_reduce_delta(wl.grads, None, wl.offsets, out=out16, workspace=ws, flags=flags,
+                                         stream=stream),
+         2 * wl.n_workers * wl.total_elems * b + 2 * wl.total_elems),
+    ]
+    results = []
+    for name, call, two_read_bytes in cases:
+        for _ in range(warmup):
+            call()
+        starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        stops = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        torch.cuda.synchronize()
+        for i in range(steps):
+            scrub.zero_()
+            starts[i].record(stream)
+            call()
+            stops[i].record(stream)
+        torch.cuda.synchronize()
+        ms = sum(a.elapsed_time(c) for a, c in zip(starts, stops)) / steps
+        results.append({"variant": name, "ms_per_reduce": ms, "input_gbs": wl.input_bytes / (ms * 1e-3) / 1e9,
+                        "two_read_bytes": two_read_bytes,
+                        "two_read_gbs": two_read_bytes / (ms * 1e-3) / 1e9})
+    return results
+
+
 class _Null:
     def __enter__(self):
         return self
@@ -486,7 +530,11 @@ def cuda_arm(args):
     summary = summarise(wl, ms, peak)
     spec = wl.spec
     n_workers, total_elems, num_tensors = wl.n_workers, wl.total_elems, wl.num_tensors
-    del wl, out, ws
+    del out, ws
+    variants = []
+    if rank == 0 and world == 1 and not args.no_other_workloads:
+        variants = time_variants(lib, wl, max(3, min(steps, 200)), 3, flags)
+    del wl
     torch.cuda.empty_cache()
 
     others = []
@@ -518,7 +566,7 @@ def cuda_arm(args):
                        "multi_gpu": "independent replicas of the workload, one per GPU, no collective"},
             "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": steps * info["launches"],
             "roofline": roofline, "cpu_baseline": cpu_baseline,
-            "whole_reduce": summary, "other_workloads": others,
+            "whole_reduce": summary, "variants": variants, "other_workloads": others,
         }
         print(json.dumps(line))
     if world > 1:

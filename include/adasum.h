@@ -164,6 +164,38 @@ adasum_status_t adasum_reduce_ex(const void* const* grads, const int64_t* tensor
                                  size_t workspace_bytes, uint32_t flags, void* stream);
 
 /*
+ * The reduce wrapped around a local optimizer step (Section 4.1, the figure that applies the
+ * operator after optimizer.step(); also "Low Precision Support" in Section 4.4.1 and the
+ * delta-from-the-last-allreduce of Section 5.2).  Every worker has taken its own optimizer step
+ * from the common parameters `start` and now holds currents[w]; the operator combines the
+ * effective gradients currents[w] - start and the combination is added back:
+ *
+ *     out = start + Adasum_w(currents[w] - start)              per tensor.
+ *
+ * Nothing is materialised: the differences are formed while the operands stream through both
+ * passes, `start` is added as the result is stored.  The cost over adasum_reduce is one more
+ * operand read per pass ((n_workers + 1) / n_workers of the traffic).
+ *
+ *   currents        host array of n_workers device pointers, as `grads` of adasum_reduce
+ *   start           device, total elements of `dtype`, 16-byte aligned; NULL: no start, the call
+ *                   is adasum_reduce_ex with a choice of output type
+ *   out             device, total elements of out_dtype.  May be `start` itself when out_dtype ==
+ *                   dtype (the parameters are updated in place); may not overlap anything else
+ *   out_dtype       ADASUM_F32, ADASUM_F16 or ADASUM_BF16 (round to nearest even on store)
+ *   everything else as for adasum_reduce_ex, including the workspace size and the plan.
+ *
+ * Each difference currents[w][e] - start[e] is rounded once, to `dtype` (what `current - start`
+ * gives in a framework); all later arithmetic is as in adasum_reduce.  With a start every buffer
+ * must be 16-byte aligned (ADASUM_ERR_ARG otherwise).  The orthogonality measure, if asked for, is
+ * that of the effective gradients.
+ */
+adasum_status_t adasum_reduce_delta(const void* const* currents, const void* start,
+                                    const int64_t* tensor_offsets, int32_t num_tensors,
+                                    int32_t n_workers, adasum_dtype_t dtype, void* out,
+                                    adasum_dtype_t out_dtype, float* orthogonality, void* workspace,
+                                    size_t workspace_bytes, uint32_t flags, void* stream);
+
+/*
  * The same reduce with the ELEMENTS of every tensor spread over several GPUs (one process per GPU).
  *
  * Each GPU holds, for all n_workers workers, its own slice of every tensor: grads[w] is worker w's

@@ -124,3 +124,53 @@ def adasum_reduce(grads, offsets=None, dtype: str | None = None, linear_order: b
 def adasum_pair(a, b, offsets=None, dtype: str | None = None) -> np.ndarray:
     """One application of the operator, per tensor: ``Adasum(a, b)``."""
     return adasum_reduce([a, b], offsets=offsets, dtype=dtype)
+
+
+# ---- the operator wrapped around a local optimizer step -----------------------------------------
+
+def decode(arr: np.ndarray, dtype: str | None = None) -> np.ndarray:
+    """The stored values as fp64, exactly (bf16 travels as uint16 bit patterns)."""
+    arr = np.asarray(arr)
+    if dtype == "bf16":
+        if arr.dtype != np.uint16:
+            raise TypeError("bf16 inputs are passed as their uint16 bit patterns")
+        return (arr.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    return arr.astype(np.float64)
+
+
+def round_to_dtype(x: np.ndarray, dtype: str) -> np.ndarray:
+    """fp64 values rounded ONCE, to nearest even, to f32 / f16 / bf16 (bf16 as uint16 patterns)."""
+    x = np.asarray(x, dtype=np.float64)
+    if dtype == "f32":
+        return x.astype(np.float32)
+    if dtype == "f16":
+        return x.astype(np.float16)
+    if dtype != "bf16":
+        raise ValueError(dtype)
+    # fp64 -> fp32 with round-to-odd (truncate, then set the last bit if anything was lost), so
+    # that the second rounding, fp32 -> bf16 to nearest even, sees whether the value was above or
+    # below a midpoint: together one correct rounding.
+    f = x.astype(np.float32)
+    inexact = f.astype(np.float64) != x
+    too_big = np.abs(f.astype(np.float64)) > np.abs(x)
+    f = np.where(too_big, np.nextafter(f, np.float32(0)), f).astype(np.float32)
+    bits = f.view(np.uint32) | inexact.astype(np.uint32)
+    rounded = (bits.astype(np.uint64) + 0x7FFF + ((bits >> 16) & 1)) >> 16
+    return rounded.astype(np.uint16)
+
+
+def adasum_reduce_delta(currents, start, offsets=None, dtype: str | None = None, linear_order: bool = False,
+                        return_orthogonality: bool = False, threads: int = 1):
+    """``start + Adasum_w(currents[w] - start)`` per tensor (Section 4.1: the operator is applied to
+    the effective gradients of a local optimizer step and the combination is added back to the
+    parameters the step started from).  Each difference is rounded once to the buffers' own type,
+    as ``current - start`` is in a framework; everything after that is fp64.  Returns fp64."""
+    if dtype is None:
+        dtype = {np.dtype(np.float32): "f32", np.dtype(np.float16): "f16"}[np.asarray(start).dtype]
+    s = decode(start, dtype)
+    deltas = [round_to_dtype(decode(c, dtype) - s, dtype) for c in currents]
+    res = adasum_reduce(deltas, offsets=offsets, dtype=dtype, linear_order=linear_order,
+                        return_orthogonality=return_orthogonality, threads=threads)
+    if return_orthogonality:
+        return s + res[0], res[1]
+    return s + res

@@ -7,7 +7,7 @@ one gradient per GPU over a torch.distributed group (recursive vector halving).
 """
 
 _BINDING_NAMES = (
-    "adasum_reduce", "adasum_reduce_ex", "adasum_sharded_gram", "adasum_sharded_apply", "adasum_reduce_sharded",
+    "adasum_reduce", "adasum_reduce_ex", "adasum_reduce_delta", "adasum_sharded_gram", "adasum_sharded_apply", "adasum_reduce_sharded",
     "adasum_pair", "adasum_pair_noalloc", "adasum_workspace_bytes",
     "adasum_plan_info", "adasum_status_string", "adasum_last_error", "adasum_shutdown",
     "adasum_profile_enable", "adasum_profile_collect", "flags_radix", "AdasumError",

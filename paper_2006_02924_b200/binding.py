@@ -47,6 +47,10 @@ _lib.adasum_reduce_ex.restype = ctypes.c_int
 _lib.adasum_reduce_ex.argtypes = [ctypes.POINTER(ctypes.c_void_p), _i64p, ctypes.c_int32, ctypes.c_int32,
                                   ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t,
                                   ctypes.c_uint32, ctypes.c_void_p]
+_lib.adasum_reduce_delta.restype = ctypes.c_int
+_lib.adasum_reduce_delta.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.c_void_p, _i64p, ctypes.c_int32,
+                                     ctypes.c_int32, ctypes.c_int, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p,
+                                     ctypes.c_void_p, ctypes.c_size_t, ctypes.c_uint32, ctypes.c_void_p]
 _lib.adasum_pair.restype = ctypes.c_int
 _lib.adasum_pair.argtypes = [ctypes.c_void_p, ctypes.c_void_p, _i64p, ctypes.c_int32, ctypes.c_int,
                              ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_uint32,
@@ -194,6 +198,34 @@ _lib.adasum_sharded_apply.restype = ctypes.c_int
 _lib.adasum_sharded_apply.argtypes = [ctypes.POINTER(ctypes.c_void_p), _i64p, ctypes.c_int32, ctypes.c_int32,
                                       ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                       ctypes.c_size_t, ctypes.c_uint32, ctypes.c_int32, ctypes.c_void_p]
+
+
+def adasum_reduce_delta(currents, start, tensor_offsets=None, out=None, out_dtype=None, orthogonality=None,
+                        workspace=None, flags: int = 0, stream=None):
+    """``adasum_reduce_delta`` of the C ABI: ``out = start + Adasum_w(currents[w] - start)`` per
+    tensor.  ``start=None`` gives the plain reduce with a choice of output type.  ``out`` may be
+    ``start`` itself (in-place update) when the types agree.  Returns ``out``."""
+    currents = list(currents)
+    first = currents[0]
+    total = first.numel()
+    offs = _offsets_array(tensor_offsets, total)
+    num_tensors = offs.size - 1
+    if out is None:
+        out = torch.empty(total, dtype=out_dtype or torch.float32, device=first.device)
+    need = adasum_workspace_bytes(total, num_tensors, len(currents), first.dtype, flags)
+    workspace, ws_ptr, ws_bytes = _workspace(workspace, need, first.device)
+    ptrs = (ctypes.c_void_p * len(currents))(*[g.data_ptr() for g in currents])
+    if start is not None and (start.dtype != first.dtype or start.numel() != total):
+        raise ValueError("start must have the type and size of the workers' buffers")
+    with torch.cuda.device(first.device):
+        status = _lib.adasum_reduce_delta(ptrs, None if start is None else start.data_ptr(),
+                                          offs.ctypes.data_as(_i64p), num_tensors, len(currents),
+                                          _dtype_code(first.dtype), out.data_ptr(), _dtype_code(out.dtype),
+                                          None if orthogonality is None else orthogonality.data_ptr(),
+                                          ws_ptr, ws_bytes, int(flags), _stream_handle(stream))
+    if status != ADASUM_OK:
+        raise AdasumError(status)
+    return out
 
 
 def adasum_sharded_gram(grads, tensor_offsets, workspace, level: int, flags: int = 0, stream=None):

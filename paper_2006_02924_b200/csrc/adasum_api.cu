@@ -379,12 +379,12 @@ cudaError_t allow_dynamic_smem(Kernel kernel, size_t bytes, bool (&configured)[6
     return cudaSuccess;
 }
 
-template <typename T, int R, bool VEC>
-cudaError_t launch_gram(GramKind kind, const OperandTable& ops, int operands, int groups_here,
-                        const SegmentTable& tab, float* partials, int groups_total, int group_base,
-                        const FinishArgs& fin, cudaStream_t stream, int* tc_status = nullptr)
+template <typename T, int R, bool VEC, bool DELTA>
+cudaError_t launch_gram_variant(GramKind kind, const OperandTable& ops, int operands, int groups_here,
+                                const SegmentTable& tab, float* partials, int groups_total, int group_base,
+                                const FinishArgs& fin, cudaStream_t stream, int* tc_status, const void* start)
 {
-    if constexpr (R == 64 && VEC && sizeof(T) == 2) {
+    if constexpr (R == 64 && VEC && sizeof(T) == 2 && !DELTA) {
         // every group complete: the tcgen05 kernel (64 x 64 accumulator in tensor memory)
         if (kind == GRAM_MMA && tc_status != nullptr && operands == groups_here * 64) {
             auto kernel = gram_partial_tc64_kernel<T>;
@@ -401,15 +401,15 @@ cudaError_t launch_gram(GramKind kind, const OperandTable& ops, int operands, in
     if constexpr (R >= 8) {
         if (kind == GRAM_MMA) {
             if constexpr (R <= 32 || sizeof(T) == 2) {
-                constexpr size_t smem = mma_smem_bytes<T, R>();
-                auto kernel = gram_partial_mma_kernel<T, R, VEC>;
+                constexpr size_t smem = mma_smem_bytes<T, R, DELTA>();
+                auto kernel = gram_partial_mma_kernel<T, R, VEC, DELTA>;
                 static bool configured[64] = {};
                 cudaError_t err = allow_dynamic_smem(kernel, smem, configured);
                 if (err != cudaSuccess)
                     return err;
                 dim3 grid((unsigned)tab.num_segments, (unsigned)groups_here);
                 kernel<<<grid, kThreads, smem, stream>>>(ops, operands, tab.d_segments, partials, groups_total,
-                                                         group_base, fin);
+                                                         group_base, fin, start);
                 return cudaSuccess;
             } else {
                 return cudaErrorInvalidValue;
@@ -419,22 +419,50 @@ cudaError_t launch_gram(GramKind kind, const OperandTable& ops, int operands, in
     if constexpr (R <= 16) {
         if (kind == GRAM_SIMPLE) {
             dim3 grid((unsigned)tab.num_segments, (unsigned)groups_here);
-            gram_partial_kernel<T, R, VEC><<<grid, kThreads, 0, stream>>>(ops, operands, tab.d_segments, partials,
-                                                                          groups_total, group_base, fin);
+            gram_partial_kernel<T, R, VEC, DELTA><<<grid, kThreads, 0, stream>>>(
+                ops, operands, tab.d_segments, partials, groups_total, group_base, fin, start);
             return cudaSuccess;
         }
     }
     return cudaErrorInvalidValue;
 }
 
+// `start` != nullptr selects the kernels that read the operands as (operand - start); those exist
+// for 16-byte aligned buffers only (the caller has checked).
+template <typename T, int R, bool VEC>
+cudaError_t launch_gram(GramKind kind, const OperandTable& ops, int operands, int groups_here,
+                        const SegmentTable& tab, float* partials, int groups_total, int group_base,
+                        const FinishArgs& fin, cudaStream_t stream, int* tc_status = nullptr,
+                        const void* start = nullptr)
+{
+    if constexpr (VEC) {
+        if (start != nullptr)
+            return launch_gram_variant<T, R, true, true>(kind, ops, operands, groups_here, tab, partials, groups_total,
+                                                         group_base, fin, stream, tc_status, start);
+    }
+    if (start != nullptr)
+        return cudaErrorInvalidValue;
+    return launch_gram_variant<T, R, VEC, false>(kind, ops, operands, groups_here, tab, partials, groups_total,
+                                                 group_base, fin, stream, tc_status, nullptr);
+}
+
+constexpr PassExtras kNoExtras{nullptr, nullptr, 0, 0};
+
 template <typename T, int R, bool VEC>
 void launch_wsum(const OperandTable& ops, int operands, int groups_here, const SegmentTable& tab,
-                 const float* weights, int groups_total, int group_base, float* dst, int64_t dst_stride,
-                 cudaStream_t stream)
+                 const float* weights, int groups_total, int group_base, void* dst, int64_t dst_stride,
+                 cudaStream_t stream, const PassExtras& ex = kNoExtras)
 {
     dim3 grid((unsigned)tab.num_segments, (unsigned)groups_here);
-    weighted_sum_kernel<T, R, VEC><<<grid, kThreads, 0, stream>>>(ops, operands, tab.d_segments, weights,
-                                                                  groups_total, group_base, dst, dst_stride);
+    if constexpr (VEC) {
+        if (ex.start != nullptr) {
+            weighted_sum_kernel<T, R, true, true><<<grid, kThreads, 0, stream>>>(
+                ops, operands, tab.d_segments, weights, groups_total, group_base, dst, dst_stride, ex);
+            return;
+        }
+    }
+    weighted_sum_kernel<T, R, VEC, false><<<grid, kThreads, 0, stream>>>(ops, operands, tab.d_segments, weights,
+                                                                         groups_total, group_base, dst, dst_stride, ex);
 }
 
 template <int R>
@@ -506,24 +534,32 @@ bool small_input_plan(const LevelPlan& plan, int64_t total, int32_t num_tensors,
 
 template <typename T, int R, bool VEC>
 cudaError_t launch_fused_small(const OperandTable& ops, int operands, const SegmentTable& tab, float* partials,
-                               const FinishArgs& fin, float* out, cudaStream_t stream)
+                               const FinishArgs& fin, void* out, const PassExtras& ex, cudaStream_t stream)
 {
-    auto kernel = fused_small_kernel<T, R, VEC>;
+    const void* kernel = (const void*)fused_small_kernel<T, R, VEC, false>;
+    if constexpr (VEC) {
+        if (ex.start != nullptr)
+            kernel = (const void*)fused_small_kernel<T, R, true, true>;
+    }
+    if (!VEC && ex.start != nullptr)
+        return cudaErrorInvalidValue;
     int operands_arg = operands;
     const Segment* segments = tab.d_segments;
-    void* args[] = {(void*)&ops, (void*)&operands_arg, (void*)&segments, (void*)&partials, (void*)&fin, (void*)&out};
-    return cudaLaunchCooperativeKernel((const void*)kernel, dim3((unsigned)tab.num_segments), dim3(kThreads), args,
-                                       0, stream);
+    PassExtras ex_arg = ex;
+    void* args[] = {(void*)&ops,      (void*)&operands_arg, (void*)&segments, (void*)&partials,
+                    (void*)&fin,      (void*)&out,          (void*)&ex_arg};
+    return cudaLaunchCooperativeKernel(kernel, dim3((unsigned)tab.num_segments), dim3(kThreads), args, 0, stream);
 }
 
 template <typename T, bool VEC>
 cudaError_t launch_fused_small_radix(int radix, const OperandTable& ops, int operands, const SegmentTable& tab,
-                                     float* partials, const FinishArgs& fin, float* out, cudaStream_t stream)
+                                     float* partials, const FinishArgs& fin, void* out, const PassExtras& ex,
+                                     cudaStream_t stream)
 {
     switch (radix) {
-    case 2: return launch_fused_small<T, 2, VEC>(ops, operands, tab, partials, fin, out, stream);
-    case 4: return launch_fused_small<T, 4, VEC>(ops, operands, tab, partials, fin, out, stream);
-    case 8: return launch_fused_small<T, 8, VEC>(ops, operands, tab, partials, fin, out, stream);
+    case 2: return launch_fused_small<T, 2, VEC>(ops, operands, tab, partials, fin, out, ex, stream);
+    case 4: return launch_fused_small<T, 4, VEC>(ops, operands, tab, partials, fin, out, ex, stream);
+    case 8: return launch_fused_small<T, 8, VEC>(ops, operands, tab, partials, fin, out, ex, stream);
     default: return cudaErrorInvalidValue;
     }
 }
@@ -561,8 +597,9 @@ struct LevelArgs {
     int* tc_status;     // status word for the tcgen05 kernel, or nullptr to keep to mma.sync
     double* gram64;
     float* weights;
-    float* dst;
+    void* dst;
     int64_t dst_stride;
+    PassExtras extras;   // start: this level's operands are (operand - start); base / out_dtype: last level
     bool vec;
     cudaStream_t stream;
     int level;
@@ -585,7 +622,8 @@ adasum_status_t run_level_typed(const LevelArgs& a)
             table.ptr[i] = a.operand_ptrs[op0 + (i < ops_here ? i : 0)];
         if (a.vec)
             ADASUM_CUDA_CHECK((launch_gram<T, R, true>(a.kind, table, ops_here, groups_here, *a.gram_tab,
-                                                       a.partials, a.groups, g0, fin, a.stream, a.tc_status)));
+                                                       a.partials, a.groups, g0, fin, a.stream, a.tc_status,
+                                                       a.extras.start)));
         else
             ADASUM_CUDA_CHECK((launch_gram<T, R, false>(a.kind, table, ops_here, groups_here, *a.gram_tab,
                                                         a.partials, a.groups, g0, fin, a.stream)));
@@ -611,10 +649,10 @@ adasum_status_t run_level_typed(const LevelArgs& a)
             table.ptr[i] = a.operand_ptrs[op0 + (i < ops_here ? i : 0)];
         if (a.vec)
             launch_wsum<T, R, true>(table, ops_here, groups_here, *a.wsum_tab, a.weights, a.groups, g0, a.dst,
-                                    a.dst_stride, a.stream);
+                                    a.dst_stride, a.stream, a.extras);
         else
             launch_wsum<T, R, false>(table, ops_here, groups_here, *a.wsum_tab, a.weights, a.groups, g0, a.dst,
-                                     a.dst_stride, a.stream);
+                                     a.dst_stride, a.stream, a.extras);
         profile_mark(a.stream, ADASUM_KERNEL_WEIGHTED_SUM, a.level, R, false);
     }
     ADASUM_CUDA_CHECK(cudaGetLastError());
@@ -685,11 +723,14 @@ adasum_status_t check_common(const int64_t* offsets, int32_t num_tensors, int32_
     return ADASUM_OK;
 }
 
+// `start` != nullptr: the delta form, out = start + Adasum_i(grads[i] - start).  `out` holds
+// elements of out_dtype.
 adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, int32_t num_tensors,
-                            int32_t n_workers, adasum_dtype_t dtype, float* out, float* orthogonality,
+                            int32_t n_workers, adasum_dtype_t dtype, void* out, float* orthogonality,
                             void* workspace, size_t workspace_bytes, uint32_t flags, cudaStream_t stream,
                             LevelPhase phase = PHASE_WHOLE, int only_level = -1, size_t* sums_offset = nullptr,
-                            int64_t* sums_count = nullptr)
+                            int64_t* sums_count = nullptr, const void* start = nullptr,
+                            adasum_dtype_t out_dtype = ADASUM_F32)
 {
     g_error[0] = '\0';
     if (!grads)
@@ -719,11 +760,24 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     const bool need_out = phase != PHASE_GRAM_SUMS && total > 0;
     if (need_out && !out)
         return fail(ADASUM_ERR_NULL, "out is NULL");
-    if (reinterpret_cast<uintptr_t>(out) & 3u)
-        return fail(ADASUM_ERR_ARG, "out is not 4-byte aligned");
+    if (out_dtype != ADASUM_F32 && out_dtype != ADASUM_F16 && out_dtype != ADASUM_BF16)
+        return fail(ADASUM_ERR_DTYPE, "unknown output dtype %d", (int)out_dtype);
+    if (reinterpret_cast<uintptr_t>(out) & (uintptr_t)(dtype_bytes(out_dtype) - 1))
+        return fail(ADASUM_ERR_ARG, "out is not aligned to its element size");
     const int eb = dtype_bytes(dtype);
-    const size_t in_bytes = (size_t)total * eb, out_bytes = out ? (size_t)total * sizeof(float) : 0;
+    const size_t in_bytes = (size_t)total * eb, out_bytes = out ? (size_t)total * dtype_bytes(out_dtype) : 0;
     bool vec = out ? aligned16(out) : true;
+    if (start != nullptr && total > 0) {
+        if (!aligned16(start))
+            return fail(ADASUM_ERR_ARG, "start is not 16-byte aligned");
+        // the result may be written over start (the parameters are updated in place), nothing else
+        const bool in_place = out == start && out_dtype == dtype;
+        if (out && !in_place && ranges_overlap(start, in_bytes, out, out_bytes))
+            return fail(ADASUM_ERR_ARG, "out overlaps start without being the same buffer of the same type");
+        for (int w = 0; w < n_workers; ++w)
+            if (grads[w] && ranges_overlap(start, in_bytes, grads[w], in_bytes))
+                return fail(ADASUM_ERR_ARG, "start overlaps grads[%d]", w);
+    }
     for (int w = 0; w < n_workers && total > 0; ++w) {
         if (!grads[w])
             return fail(ADASUM_ERR_NULL, "grads[%d] is NULL", w);
@@ -733,6 +787,8 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
             return fail(ADASUM_ERR_ARG, "out overlaps grads[%d]", w);
         vec = vec && aligned16(grads[w]);
     }
+    if (start != nullptr && total > 0 && !vec)
+        return fail(ADASUM_ERR_ARG, "the delta form needs every buffer 16-byte aligned");
     const Layout lay = make_layout(plan, total, num_tensors);
     if (n_workers > 1) {
         if (!workspace)
@@ -746,18 +802,24 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         for (int w = 0; w < n_workers && total > 0; ++w)
             if (ranges_overlap(workspace, lay.total, grads[w], in_bytes))
                 return fail(ADASUM_ERR_ARG, "workspace overlaps grads[%d]", w);
+        if (start != nullptr && total > 0 && ranges_overlap(workspace, lay.total, start, in_bytes))
+            return fail(ADASUM_ERR_ARG, "workspace overlaps start");
     }
+    // what the last level adds and how it stores; the first level gets `start` as well
+    const PassExtras last_extras{nullptr, start, (int)dtype, (int)out_dtype};
 
     profile_mark(stream, -1, 0, 0, true);
     if (n_workers == 1) {
         const int64_t blocks = (total + kThreads - 1) / kThreads;
         const unsigned grid = (unsigned)(blocks < 148 * 16 ? blocks : 148 * 16);
+        PassExtras ex = last_extras;
+        ex.start = start;
         if (dtype == ADASUM_F32)
-            convert_kernel<float><<<grid, kThreads, 0, stream>>>((const float*)grads[0], out, total);
+            convert_kernel<float><<<grid, kThreads, 0, stream>>>((const float*)grads[0], out, total, ex);
         else if (dtype == ADASUM_F16)
-            convert_kernel<__half><<<grid, kThreads, 0, stream>>>((const __half*)grads[0], out, total);
+            convert_kernel<__half><<<grid, kThreads, 0, stream>>>((const __half*)grads[0], out, total, ex);
         else
-            convert_kernel<__nv_bfloat16><<<grid, kThreads, 0, stream>>>((const __nv_bfloat16*)grads[0], out, total);
+            convert_kernel<__nv_bfloat16><<<grid, kThreads, 0, stream>>>((const __nv_bfloat16*)grads[0], out, total, ex);
         ADASUM_CUDA_CHECK(cudaGetLastError());
         profile_mark(stream, ADASUM_KERNEL_CONVERT, 0, 1, false);
         return ADASUM_OK;
@@ -808,16 +870,18 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
                                    orthogonality};
             float* partials = reinterpret_cast<float*>(ws + lay.partials);
             const int radix = plan.level[0].radix;
+            PassExtras ex = last_extras;
+            ex.start = start;
             cudaError_t err;
             if (dtype == ADASUM_F32)
-                err = vec ? launch_fused_small_radix<float, true>(radix, table, n_workers, *tab, partials, fin, out, stream)
-                          : launch_fused_small_radix<float, false>(radix, table, n_workers, *tab, partials, fin, out, stream);
+                err = vec ? launch_fused_small_radix<float, true>(radix, table, n_workers, *tab, partials, fin, out, ex, stream)
+                          : launch_fused_small_radix<float, false>(radix, table, n_workers, *tab, partials, fin, out, ex, stream);
             else if (dtype == ADASUM_F16)
-                err = vec ? launch_fused_small_radix<__half, true>(radix, table, n_workers, *tab, partials, fin, out, stream)
-                          : launch_fused_small_radix<__half, false>(radix, table, n_workers, *tab, partials, fin, out, stream);
+                err = vec ? launch_fused_small_radix<__half, true>(radix, table, n_workers, *tab, partials, fin, out, ex, stream)
+                          : launch_fused_small_radix<__half, false>(radix, table, n_workers, *tab, partials, fin, out, ex, stream);
             else
-                err = vec ? launch_fused_small_radix<__nv_bfloat16, true>(radix, table, n_workers, *tab, partials, fin, out, stream)
-                          : launch_fused_small_radix<__nv_bfloat16, false>(radix, table, n_workers, *tab, partials, fin, out, stream);
+                err = vec ? launch_fused_small_radix<__nv_bfloat16, true>(radix, table, n_workers, *tab, partials, fin, out, ex, stream)
+                          : launch_fused_small_radix<__nv_bfloat16, false>(radix, table, n_workers, *tab, partials, fin, out, ex, stream);
             if (err == cudaSuccess) {
                 profile_mark(stream, ADASUM_KERNEL_FUSED_SMALL, 0, radix, false);
                 return ADASUM_OK;
@@ -873,8 +937,11 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         a.tree.groups_first = plan.level[0].groups;
         a.tree.leaf_norm_sums = orthogonality ? reinterpret_cast<double*>(ws + lay.leaf_sums) : nullptr;
         a.tree.orthogonality = orthogonality;
-        a.dst = last ? out : reinterpret_cast<float*>(ws + lay.buffer[l & 1]);
+        a.dst = last ? out : static_cast<void*>(ws + lay.buffer[l & 1]);
         a.dst_stride = last ? 0 : lay.padded_elems;
+        a.extras = last ? last_extras : kNoExtras;
+        if (l == 0)
+            a.extras.start = start;
         a.vec = vec;
         a.stream = stream;
         a.level = l;
@@ -893,7 +960,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         if (!last) {
             operand_ptrs.resize((size_t)lv.groups);
             for (int g = 0; g < lv.groups; ++g)
-                operand_ptrs[g] = a.dst + (int64_t)g * lay.padded_elems;
+                operand_ptrs[g] = static_cast<float*>(a.dst) + (int64_t)g * lay.padded_elems;
         }
     }
     return ADASUM_OK;
@@ -1084,6 +1151,17 @@ adasum_status_t adasum_reduce_ex(const void* const* grads, const int64_t* tensor
 {
     return adasum::reduce_impl(grads, tensor_offsets, num_tensors, n_workers, dtype, out, orthogonality, workspace,
                                workspace_bytes, flags, static_cast<cudaStream_t>(stream));
+}
+
+adasum_status_t adasum_reduce_delta(const void* const* currents, const void* start,
+                                    const int64_t* tensor_offsets, int32_t num_tensors, int32_t n_workers,
+                                    adasum_dtype_t dtype, void* out, adasum_dtype_t out_dtype,
+                                    float* orthogonality, void* workspace, size_t workspace_bytes, uint32_t flags,
+                                    void* stream)
+{
+    return adasum::reduce_impl(currents, tensor_offsets, num_tensors, n_workers, dtype, out, orthogonality,
+                               workspace, workspace_bytes, flags, static_cast<cudaStream_t>(stream),
+                               adasum::PHASE_WHOLE, -1, nullptr, nullptr, start, out_dtype);
 }
 
 adasum_status_t adasum_sharded_gram(const void* const* grads, const int64_t* tensor_offsets,

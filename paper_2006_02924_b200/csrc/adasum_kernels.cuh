@@ -128,6 +128,39 @@ struct Element<__nv_bfloat16> {
     }
 };
 
+// 16 bytes of T as floats.
+template <typename T>
+__device__ __forceinline__ void decode_vector(const uint4& v, float (&x)[Element<T>::kVec]);
+template <>
+__device__ __forceinline__ void decode_vector<float>(const uint4& v, float (&x)[4])
+{
+    x[0] = __uint_as_float(v.x);
+    x[1] = __uint_as_float(v.y);
+    x[2] = __uint_as_float(v.z);
+    x[3] = __uint_as_float(v.w);
+}
+template <>
+__device__ __forceinline__ void decode_vector<__half>(const uint4& v, float (&x)[8])
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+        x[2 * i] = f.x;
+        x[2 * i + 1] = f.y;
+    }
+}
+template <>
+__device__ __forceinline__ void decode_vector<__nv_bfloat16>(const uint4& v, float (&x)[8])
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        x[2 * i] = __uint_as_float(w[i] << 16);
+        x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+}
+
 // Split a segment [begin, end) into a scalar head, a 16-byte-aligned vector body and a scalar
 // tail.  Without VEC (some buffer is not 16-byte aligned) everything is "tail".
 template <int V, bool VEC>
@@ -142,6 +175,146 @@ __device__ __forceinline__ void split_segment(int64_t begin, int64_t end, int64_
     } else {
         body_begin = begin;
         body_end = begin;
+    }
+}
+
+// ---- the "optimizer delta" form and the output format -------------------------------------------
+//
+// Section 4.1 (the figure that wraps an optimizer): every worker takes a local optimizer step from
+// the common parameters `start`, the operator combines the effective gradients current_i - start,
+// and the combination is added back to `start`.  With DELTA the first level's operands are read as
+// (ptr[i] - start), the difference rounded once to the operands' own type T (what
+// `current - start` gives in a framework); `base` is added to the last level's result; the last
+// level may store fp16 / bf16 instead of fp32.
+struct PassExtras {
+    const void* start;    // DELTA kernels: subtracted from every operand of this level (type T)
+    const void* base;     // last level: result = base + sum (nullptr: nothing added)
+    int base_dtype;       // 0 fp32, 1 fp16, 2 bf16
+    int out_dtype;        // type of the level's destination: 0 fp32 (always, except a last level), 1 fp16, 2 bf16
+};
+
+// Data that the same thread may overwrite later in the same kernel (out == start): a plain load.
+__device__ __forceinline__ uint4 load_plain_16B(const void* p) { return *reinterpret_cast<const uint4*>(p); }
+
+// c - s on the packed words of a 16-byte vector, in T, round to nearest even.
+template <typename T>
+__device__ __forceinline__ uint4 delta_words(const uint4& c, const uint4& s);
+template <>
+__device__ __forceinline__ uint4 delta_words<float>(const uint4& c, const uint4& s)
+{
+    return make_uint4(__float_as_uint(__fsub_rn(__uint_as_float(c.x), __uint_as_float(s.x))),
+                      __float_as_uint(__fsub_rn(__uint_as_float(c.y), __uint_as_float(s.y))),
+                      __float_as_uint(__fsub_rn(__uint_as_float(c.z), __uint_as_float(s.z))),
+                      __float_as_uint(__fsub_rn(__uint_as_float(c.w), __uint_as_float(s.w))));
+}
+template <>
+__device__ __forceinline__ uint4 delta_words<__half>(const uint4& c, const uint4& s)
+{
+    const uint32_t cw[4] = {c.x, c.y, c.z, c.w}, sw[4] = {s.x, s.y, s.z, s.w};
+    uint32_t d[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __half2 r = __hsub2(*reinterpret_cast<const __half2*>(&cw[i]), *reinterpret_cast<const __half2*>(&sw[i]));
+        d[i] = *reinterpret_cast<const uint32_t*>(&r);
+    }
+    return make_uint4(d[0], d[1], d[2], d[3]);
+}
+template <>
+__device__ __forceinline__ uint4 delta_words<__nv_bfloat16>(const uint4& c, const uint4& s)
+{
+    const uint32_t cw[4] = {c.x, c.y, c.z, c.w}, sw[4] = {s.x, s.y, s.z, s.w};
+    uint32_t d[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat162 r = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&cw[i]),
+                                         *reinterpret_cast<const __nv_bfloat162*>(&sw[i]));
+        d[i] = *reinterpret_cast<const uint32_t*>(&r);
+    }
+    return make_uint4(d[0], d[1], d[2], d[3]);
+}
+// One element: c - s in T, as a float.
+__device__ __forceinline__ float delta_one(const float* c, const float* s, int64_t e) { return __fsub_rn(c[e], s[e]); }
+__device__ __forceinline__ float delta_one(const __half* c, const __half* s, int64_t e)
+{
+    return __half2float(__hsub(c[e], s[e]));
+}
+__device__ __forceinline__ float delta_one(const __nv_bfloat16* c, const __nv_bfloat16* s, int64_t e)
+{
+    return __bfloat162float(__hsub(c[e], s[e]));
+}
+
+// Element e of a buffer of the given dtype code, as a float (plain load).
+__device__ __forceinline__ float load_as_float(const void* p, int dtype, int64_t e)
+{
+    if (dtype == 0)
+        return static_cast<const float*>(p)[e];
+    if (dtype == 1)
+        return __half2float(static_cast<const __half*>(p)[e]);
+    return __bfloat162float(static_cast<const __nv_bfloat16*>(p)[e]);
+}
+__device__ __forceinline__ void store_from_float(void* p, int dtype, int64_t e, float y)
+{
+    if (dtype == 0)
+        static_cast<float*>(p)[e] = y;
+    else if (dtype == 1)
+        static_cast<__half*>(p)[e] = __float2half_rn(y);
+    else
+        static_cast<__nv_bfloat16*>(p)[e] = __float2bfloat16_rn(y);
+}
+// N = 4 or 8 consecutive elements starting at element e (e a multiple of N, buffer 16-byte aligned).
+template <int N>
+__device__ __forceinline__ void add_vector_as_float(const void* p, int dtype, int64_t e, float (&y)[N])
+{
+    if (dtype == 0) {
+#pragma unroll
+        for (int j = 0; j < N; j += 4) {
+            const float4 b = *reinterpret_cast<const float4*>(static_cast<const float*>(p) + e + j);
+            y[j] += b.x; y[j + 1] += b.y; y[j + 2] += b.z; y[j + 3] += b.w;
+        }
+    } else {
+        uint32_t w[N / 2];
+        if constexpr (N == 8) {
+            const uint4 b = *reinterpret_cast<const uint4*>(static_cast<const unsigned short*>(p) + e);
+            w[0] = b.x; w[1] = b.y; w[2] = b.z; w[3] = b.w;
+        } else {
+            const uint2 b = *reinterpret_cast<const uint2*>(static_cast<const unsigned short*>(p) + e);
+            w[0] = b.x; w[1] = b.y;
+        }
+#pragma unroll
+        for (int i = 0; i < N / 2; ++i) {
+            if (dtype == 1) {
+                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+                y[2 * i] += f.x; y[2 * i + 1] += f.y;
+            } else {
+                y[2 * i] += __uint_as_float(w[i] << 16);
+                y[2 * i + 1] += __uint_as_float(w[i] & 0xffff0000u);
+            }
+        }
+    }
+}
+template <int N>
+__device__ __forceinline__ void store_vector_from_float(void* p, int dtype, int64_t e, const float (&y)[N])
+{
+    if (dtype == 0) {
+#pragma unroll
+        for (int j = 0; j < N; j += 4)
+            *reinterpret_cast<float4*>(static_cast<float*>(p) + e + j) = make_float4(y[j], y[j + 1], y[j + 2], y[j + 3]);
+    } else {
+        uint32_t w[N / 2];
+#pragma unroll
+        for (int i = 0; i < N / 2; ++i) {
+            if (dtype == 1) {
+                const __half2 h = __floats2half2_rn(y[2 * i], y[2 * i + 1]);
+                w[i] = *reinterpret_cast<const uint32_t*>(&h);
+            } else {
+                const __nv_bfloat162 h = __floats2bfloat162_rn(y[2 * i], y[2 * i + 1]);
+                w[i] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+        }
+        if constexpr (N == 8)
+            *reinterpret_cast<uint4*>(static_cast<unsigned short*>(p) + e) = make_uint4(w[0], w[1], w[2], w[3]);
+        else
+            *reinterpret_cast<uint2*>(static_cast<unsigned short*>(p) + e) = make_uint2(w[0], w[1]);
     }
 }
 
@@ -220,9 +393,11 @@ __device__ __forceinline__ void gram_accumulate(const float (&x)[R], float (&acc
 
 // The Gram matrix of one segment of the group whose first operand is ops.ptr[first], computed by
 // the whole block on the fp32 pipes and written to dst[0 .. E).
-template <typename T, int R, bool VEC>
+// With DELTA the rows are (operand - start), rounded to T.
+template <typename T, int R, bool VEC, bool DELTA = false>
 __device__ __forceinline__ void gram_of_segment(const OperandTable& ops, int first, int members,
-                                                const Segment& seg, float* __restrict__ dst)
+                                                const Segment& seg, float* __restrict__ dst,
+                                                const T* start = nullptr)
 {
     constexpr int E = gram_entries(R);
     constexpr int V = Element<T>::kVec;
@@ -243,10 +418,16 @@ __device__ __forceinline__ void gram_of_segment(const OperandTable& ops, int fir
 
     for (int64_t v = body_begin + (int64_t)threadIdx.x * V; v < body_end; v += (int64_t)kThreads * V) {
         float x[R][V];
+        uint4 sraw = make_uint4(0u, 0u, 0u, 0u);
+        if constexpr (DELTA)
+            sraw = load_plain_16B(start + v);
 #pragma unroll
         for (int i = 0; i < R; ++i) {
             if (i < members) {
-                Element<T>::vec(src[i] + v, x[i]);
+                if constexpr (DELTA)
+                    decode_vector<T>(delta_words<T>(load_keep_16B(src[i] + v), sraw), x[i]);
+                else
+                    Element<T>::vec(src[i] + v, x[i]);
             } else {
 #pragma unroll
                 for (int j = 0; j < V; ++j)
@@ -269,8 +450,12 @@ __device__ __forceinline__ void gram_of_segment(const OperandTable& ops, int fir
         for (int64_t e = lo + threadIdx.x; e < hi; e += kThreads) {
             float col[R];
 #pragma unroll
-            for (int i = 0; i < R; ++i)
-                col[i] = i < members ? Element<T>::one(src[i] + e) : 0.0f;
+            for (int i = 0; i < R; ++i) {
+                if constexpr (DELTA)
+                    col[i] = i < members ? delta_one(src[i], start, e) : 0.0f;
+                else
+                    col[i] = i < members ? Element<T>::one(src[i] + e) : 0.0f;
+            }
             gram_accumulate<R>(col, acc);
         }
     }
@@ -299,18 +484,19 @@ __device__ __forceinline__ void gram_of_segment(const OperandTable& ops, int fir
 
 // grid = (segments, groups in this launch); block = kThreads.
 // partials[(segment * groups_total + group_base + blockIdx.y) * E + entry]
-template <typename T, int R, bool VEC>
+template <typename T, int R, bool VEC, bool DELTA = false>
 __global__ void __launch_bounds__(kThreads)
 gram_partial_kernel(const __grid_constant__ OperandTable ops, int operands,
                     const Segment* __restrict__ segments, float* __restrict__ partials,
-                    int groups_total, int group_base, FinishArgs fin)
+                    int groups_total, int group_base, FinishArgs fin, const void* start)
 {
     constexpr int E = gram_entries(R);
     const Segment seg = segments[blockIdx.x];
     const int first = blockIdx.y * R;
     const int members = min(R, operands - first);
-    gram_of_segment<T, R, VEC>(ops, first, members, seg,
-                               partials + ((int64_t)blockIdx.x * groups_total + group_base + blockIdx.y) * E);
+    gram_of_segment<T, R, VEC, DELTA>(ops, first, members, seg,
+                                      partials + ((int64_t)blockIdx.x * groups_total + group_base + blockIdx.y) * E,
+                                      static_cast<const T*>(start));
     finish_if_last<R>(fin, partials, seg.tensor, group_base + blockIdx.y, groups_total, members);
 }
 
@@ -469,8 +655,12 @@ __host__ __device__ constexpr int mma_min_blocks()
 template <typename T, int R>
 __host__ __device__ constexpr int mma_stages() { return mma_min_blocks<T, R>() == 1 ? 6 : 3; }
 constexpr int kMmaTileBytes = 32 * 1024;
-template <typename T, int R>
-__host__ __device__ constexpr size_t mma_smem_bytes() { return (size_t)mma_stages<T, R>() * kMmaTileBytes; }
+// With DELTA every stage carries one more row: the same columns of `start`.
+template <typename T, int R, bool DELTA = false>
+__host__ __device__ constexpr size_t mma_smem_bytes()
+{
+    return (size_t)mma_stages<T, R>() * (kMmaTileBytes + (DELTA ? kMmaTileBytes / R : 0));
+}
 
 // grid = (segments, groups in this launch); block = kThreads; dynamic shared memory =
 // mma_smem_bytes<T, R>().
@@ -479,11 +669,15 @@ __host__ __device__ constexpr size_t mma_smem_bytes() { return (size_t)mma_stage
 // fragment reads of a quarter warp (two rows, four 16-byte pieces each) fall into distinct banks.
 // The pipeline is the usual multi-stage one: wait for the oldest copy group, one __syncthreads
 // per tile, refill the slot that was consumed in the previous iteration.
-template <typename T, int R, bool VEC>
+//
+// DELTA: the rows are (operand - start), rounded to T.  The tile gets one more row, unswizzled,
+// with the same columns of `start`; a lane subtracts its 16 bytes of it from every fragment it
+// loads.  Rows beyond the group's members are copies of `start`, so that they come out as zero.
+template <typename T, int R, bool VEC, bool DELTA = false>
 __global__ void __launch_bounds__(kThreads, mma_min_blocks<T, R>())
 gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
                         const Segment* __restrict__ segments, float* __restrict__ partials,
-                        int groups_total, int group_base, FinishArgs fin)
+                        int groups_total, int group_base, FinishArgs fin, const void* start_ptr)
 {
     constexpr int E = gram_entries(R);
     constexpr int V = Element<T>::kVec;          // elements per 16-byte vector
@@ -496,6 +690,7 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
     constexpr int DEPTH = mma_depth<T, R>();
     constexpr int STAGES = mma_stages<T, R>();
     constexpr int ROW_BYTES = kMmaTileBytes / R;
+    constexpr int STAGE_BYTES = kMmaTileBytes + (DELTA ? ROW_BYTES : 0);
     constexpr int PIECES_PER_ROW = ROW_BYTES / 16;
     constexpr int TILE_ELEMS = PIECES_PER_ROW * V;               // elements of one row in a tile
     constexpr int PIECES = kMmaTileBytes / 16 / kThreads;        // 16-byte pieces a thread copies per tile
@@ -527,17 +722,22 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
     for (int i = 0; i < PIECES; ++i) {
         const int row = row0 + i * ROWS_PER_PASS;
         copy_src[i] = static_cast<const T*>(ops.ptr[first + (row < members ? row : 0)]) + col0 * V;
+        if (DELTA && row >= members)
+            copy_src[i] = static_cast<const T*>(start_ptr) + col0 * V;
     }
-    const bool full_group = members == R;
+    const T* start_src = static_cast<const T*>(start_ptr) + col0 * V;      // DELTA: threads of row0 == 0 copy it
+    const bool full_group = members == R || DELTA;
 
     auto issue = [&](int tile, int stage) {
         if (tile < ntiles) {
-            const uint32_t dst = smem_base + stage * kMmaTileBytes;
+            const uint32_t dst = smem_base + stage * STAGE_BYTES;
             const int64_t tile_elem0 = k0 + (int64_t)tile * TILE_ELEMS;
             if (VEC && full_group && tile_elem0 >= begin && tile_elem0 + TILE_ELEMS <= end) {
 #pragma unroll
                 for (int i = 0; i < PIECES; ++i)
                     cp_async_16B_shared(dst + copy_off(i), copy_src[i] + tile_elem0);
+                if (DELTA && row0 == 0)
+                    cp_async_16B_shared(dst + kMmaTileBytes + (col0 << 4), start_src + tile_elem0);
             } else {
                 // ragged tile, partial group or unaligned buffers: test every piece
                 const int64_t e0 = tile_elem0 + (int64_t)col0 * V;
@@ -545,12 +745,19 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
 #pragma unroll
                 for (int i = 0; i < PIECES; ++i) {
                     const uint32_t slot = dst + copy_off(i);
-                    if (row0 + i * ROWS_PER_PASS >= members)
+                    if (!DELTA && row0 + i * ROWS_PER_PASS >= members)
                         store_shared_16B(slot, make_uint4(0u, 0u, 0u, 0u));
                     else if (whole)
                         cp_async_16B_shared(slot, copy_src[i] + tile_elem0);
                     else
                         store_shared_16B(slot, load_masked_words<T>(copy_src[i] - col0 * V, e0, begin, end));
+                }
+                if (DELTA && row0 == 0) {
+                    if (whole)
+                        cp_async_16B_shared(dst + kMmaTileBytes + (col0 << 4), start_src + tile_elem0);
+                    else
+                        store_shared_16B(dst + kMmaTileBytes + (col0 << 4),
+                                         load_masked_words<T>(start_src - col0 * V, e0, begin, end));
                 }
             }
         }
@@ -590,7 +797,8 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
             refill -= STAGES;
         issue(tile + STAGES - 1, refill);
 
-        const uint32_t src_stage = smem_base + stage * kMmaTileBytes + frag_off;
+        const uint32_t src_stage = smem_base + stage * STAGE_BYTES + frag_off;
+        const uint32_t start_stage = smem_base + stage * STAGE_BYTES + kMmaTileBytes + (t << 4);
         if (++stage == STAGES)
             stage = 0;
 
@@ -598,10 +806,15 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
 #pragma unroll
             for (int d = 0; d < DEPTH; ++d) {
                 uint32_t w[RBP][4];
+                uint4 sv = make_uint4(0u, 0u, 0u, 0u);
+                if constexpr (DELTA)
+                    sv = load_shared_16B(start_stage + ((warp * DEPTH + d) << 6));
 #pragma unroll
                 for (int rb = 0; rb < RBP; ++rb) {
-                    const uint4 v = rb < RB ? load_shared_16B(src_stage + chunk_off[d] + rb * 8 * ROW_BYTES)
-                                            : make_uint4(0u, 0u, 0u, 0u);
+                    uint4 v = rb < RB ? load_shared_16B(src_stage + chunk_off[d] + rb * 8 * ROW_BYTES)
+                                      : make_uint4(0u, 0u, 0u, 0u);
+                    if (DELTA && rb < RB)
+                        v = delta_words<T>(v, sv);
                     w[rb][0] = v.x; w[rb][1] = v.y; w[rb][2] = v.z; w[rb][3] = v.w;
                 }
 #pragma unroll
@@ -630,10 +843,15 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
 #pragma unroll
             for (int d = 0; d < DEPTH; ++d) {
                 uint32_t hi[RBP][4], lo[RBP][4];
+                uint4 sv = make_uint4(0u, 0u, 0u, 0u);
+                if constexpr (DELTA)
+                    sv = load_shared_16B(start_stage + ((warp * DEPTH + d) << 6));
 #pragma unroll
                 for (int rb = 0; rb < RBP; ++rb) {
-                    const uint4 v = rb < RB ? load_shared_16B(src_stage + chunk_off[d] + rb * 8 * ROW_BYTES)
-                                            : make_uint4(0u, 0u, 0u, 0u);
+                    uint4 v = rb < RB ? load_shared_16B(src_stage + chunk_off[d] + rb * 8 * ROW_BYTES)
+                                      : make_uint4(0u, 0u, 0u, 0u);
+                    if (DELTA && rb < RB)
+                        v = delta_words<T>(v, sv);
                     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
@@ -1209,46 +1427,18 @@ tree_weights_kernel(const double* __restrict__ gram64, int operands, float* __re
 
 // ---- pass 2: weighted sum ---------------------------------------------------------------------
 
-template <typename T>
-__device__ __forceinline__ void decode_vector(const uint4& v, float (&x)[Element<T>::kVec]);
-template <>
-__device__ __forceinline__ void decode_vector<float>(const uint4& v, float (&x)[4])
-{
-    x[0] = __uint_as_float(v.x);
-    x[1] = __uint_as_float(v.y);
-    x[2] = __uint_as_float(v.z);
-    x[3] = __uint_as_float(v.w);
-}
-template <>
-__device__ __forceinline__ void decode_vector<__half>(const uint4& v, float (&x)[8])
-{
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
-        x[2 * i] = f.x;
-        x[2 * i + 1] = f.y;
-    }
-}
-template <>
-__device__ __forceinline__ void decode_vector<__nv_bfloat16>(const uint4& v, float (&x)[8])
-{
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        x[2 * i] = __uint_as_float(w[i] << 16);
-        x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-    }
-}
-
 // The weighted sum of one segment, dst[e] = sum_i w_i x_i[e], by the whole block.  wsrc[0 .. R)
 // are the leaf weights (global or shared memory).  Rows are read eight at a time so that the
 // loads of one batch are in flight together while the register count stays low enough for three
 // blocks per SM.
-template <typename T, int R, bool VEC>
+//
+// DELTA: the rows are (operand - ex.start), rounded to T.  ex.base (if any) is added to the sum
+// and the result is stored in ex.out_dtype; dst may be the same buffer as ex.start / ex.base
+// (every element is read by the thread that writes it, before it writes).
+template <typename T, int R, bool VEC, bool DELTA = false>
 __device__ __forceinline__ void weighted_sum_of_segment(const OperandTable& ops, int first, int members,
                                                         const Segment& seg, const float* wsrc,
-                                                        float* __restrict__ dst)
+                                                        void* dst, const PassExtras& ex)
 {
     constexpr int V = Element<T>::kVec;
     constexpr int BATCH = R < 8 ? R : 8;
@@ -1281,6 +1471,9 @@ __device__ __forceinline__ void weighted_sum_of_segment(const OperandTable& ops,
 #pragma unroll
         for (int j = 0; j < V; ++j)
             y[j] = 0.0f;
+        uint4 sraw = make_uint4(0u, 0u, 0u, 0u);
+        if constexpr (DELTA)
+            sraw = load_plain_16B(static_cast<const T*>(ex.start) + v);
         // Two batches may be unrolled together; beyond that the loop stays rolled so that the
         // compiler cannot hoist every batch's loads and spill.
 #pragma unroll(R / BATCH <= 2 ? 2 : 1)
@@ -1294,7 +1487,10 @@ __device__ __forceinline__ void weighted_sum_of_segment(const OperandTable& ops,
             for (int i = 0; i < BATCH; ++i) {
                 if (b + i < members) {
                     float x[V];
-                    decode_vector<T>(raw[i], x);
+                    if constexpr (DELTA)
+                        decode_vector<T>(delta_words<T>(raw[i], sraw), x);
+                    else
+                        decode_vector<T>(raw[i], x);
                     const float wi = w(b + i);
 #pragma unroll
                     for (int j = 0; j < V; ++j)
@@ -1302,9 +1498,9 @@ __device__ __forceinline__ void weighted_sum_of_segment(const OperandTable& ops,
                 }
             }
         }
-#pragma unroll
-        for (int j = 0; j < V; j += 4)
-            *reinterpret_cast<float4*>(dst + v + j) = make_float4(y[j], y[j + 1], y[j + 2], y[j + 3]);
+        if (ex.base != nullptr)
+            add_vector_as_float<V>(ex.base, ex.base_dtype, v, y);
+        store_vector_from_float<V>(dst, ex.out_dtype, v, y);
     }
     for (int pass = 0; pass < 2; ++pass) {
         const int64_t lo = pass == 0 ? begin : body_end;
@@ -1312,22 +1508,30 @@ __device__ __forceinline__ void weighted_sum_of_segment(const OperandTable& ops,
         for (int64_t e = lo + threadIdx.x; e < hi; e += kThreads) {
             float y = 0.0f;
 #pragma unroll
-            for (int i = 0; i < R; ++i)
-                if (i < members)
-                    y = fmaf(w(i), Element<T>::one(static_cast<const T*>(ops.ptr[first + i]) + e), y);
-            dst[e] = y;
+            for (int i = 0; i < R; ++i) {
+                if (i < members) {
+                    if constexpr (DELTA)
+                        y = fmaf(w(i), delta_one(static_cast<const T*>(ops.ptr[first + i]),
+                                                 static_cast<const T*>(ex.start), e), y);
+                    else
+                        y = fmaf(w(i), Element<T>::one(static_cast<const T*>(ops.ptr[first + i]) + e), y);
+                }
+            }
+            if (ex.base != nullptr)
+                y += load_as_float(ex.base, ex.base_dtype, e);
+            store_from_float(dst, ex.out_dtype, e, y);
         }
     }
 }
 
 // grid = (segments, groups in this launch); block = kThreads.
-// dst_base + (group_base + blockIdx.y) * dst_stride is the group's output buffer (fp32).
-template <typename T, int R, bool VEC>
+// dst_base + (group_base + blockIdx.y) * dst_stride floats is the group's output buffer (fp32; a
+// last level has one group and stride 0, and may store another type: ex.out_dtype).
+template <typename T, int R, bool VEC, bool DELTA = false>
 __global__ void __launch_bounds__(kThreads, 3)
 weighted_sum_kernel(const __grid_constant__ OperandTable ops, int operands,
                     const Segment* __restrict__ segments, const float* __restrict__ weights,
-                    int groups_total, int group_base, float* __restrict__ dst_base,
-                    int64_t dst_stride)
+                    int groups_total, int group_base, void* dst_base, int64_t dst_stride, PassExtras ex)
 {
     // Segments are taken last to first: pass 1 walked them first to last, so the tail of the
     // operands is what the L2 still holds when this kernel starts.
@@ -1335,9 +1539,9 @@ weighted_sum_kernel(const __grid_constant__ OperandTable ops, int operands,
     const int first = blockIdx.y * R;
     const int members = min(R, operands - first);
     const int group = group_base + blockIdx.y;
-    weighted_sum_of_segment<T, R, VEC>(ops, first, members, seg,
-                                       weights + ((int64_t)seg.tensor * groups_total + group) * R,
-                                       dst_base + (int64_t)group * dst_stride);
+    weighted_sum_of_segment<T, R, VEC, DELTA>(ops, first, members, seg,
+                                              weights + ((int64_t)seg.tensor * groups_total + group) * R,
+                                              static_cast<float*>(dst_base) + (int64_t)group * dst_stride, ex);
 }
 
 // ---- both passes in one launch, for inputs that fit the L2 -------------------------------------
@@ -1349,16 +1553,17 @@ weighted_sum_kernel(const __grid_constant__ OperandTable ops, int operands,
 // and then writes the weighted sum of the segment it has just read, which the 126 MB L2 still
 // holds.  HBM sees the operands once.
 // grid = segments; block = kThreads; partials[segment * E + entry].
-template <typename T, int R, bool VEC>
+template <typename T, int R, bool VEC, bool DELTA = false>
 __global__ void __launch_bounds__(kThreads, (sizeof(T) == 2 && R == 8) ? 2 : 3)
 fused_small_kernel(const __grid_constant__ OperandTable ops, int operands,
                    const Segment* __restrict__ segments, float* __restrict__ partials, FinishArgs fin,
-                   float* __restrict__ out)
+                   void* out, PassExtras ex)
 {
     constexpr int E = gram_entries(R);
     const Segment seg = segments[blockIdx.x];
     const int members = min(R, operands);
-    gram_of_segment<T, R, VEC>(ops, 0, members, seg, partials + (int64_t)blockIdx.x * E);
+    gram_of_segment<T, R, VEC, DELTA>(ops, 0, members, seg, partials + (int64_t)blockIdx.x * E,
+                                      static_cast<const T*>(ex.start));
     __threadfence();
     cooperative_groups::this_grid().sync();
 
@@ -1371,17 +1576,22 @@ fused_small_kernel(const __grid_constant__ OperandTable ops, int operands,
     }
     finish_group_in_block<R>(partials, s0, s1, seg.tensor, 0, 1, members, leaf_weights, opt);
     __syncthreads();
-    weighted_sum_of_segment<T, R, VEC>(ops, 0, members, seg, leaf_weights, out);
+    weighted_sum_of_segment<T, R, VEC, DELTA>(ops, 0, members, seg, leaf_weights, out, ex);
 }
 
-// n_workers = 1: the result is the input, converted to fp32.
+// n_workers = 1: the result is the input (with a start: start + (input - start), the difference
+// rounded to T like everywhere else), stored in ex.out_dtype.
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
-convert_kernel(const T* __restrict__ src, float* __restrict__ dst, int64_t n)
+convert_kernel(const T* src, void* dst, int64_t n, PassExtras ex)
 {
     for (int64_t e = (int64_t)blockIdx.x * kThreads + threadIdx.x; e < n;
-         e += (int64_t)gridDim.x * kThreads)
-        dst[e] = Element<T>::one(src + e);
+         e += (int64_t)gridDim.x * kThreads) {
+        float y = ex.start != nullptr ? delta_one(src, static_cast<const T*>(ex.start), e) : Element<T>::one(src + e);
+        if (ex.base != nullptr)
+            y += load_as_float(ex.base, ex.base_dtype, e);
+        store_from_float(dst, ex.out_dtype, e, y);
+    }
 }
 
 }  // namespace adasum

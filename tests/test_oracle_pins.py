@@ -274,3 +274,70 @@ def test_generator_statistics_level_one_coefficient():
     a, b = (g.double().numpy() for g in wl.grads)
     ca, cb = oracle.coefficients(float(a @ b), float(a @ a), float(b @ b))
     assert abs(ca - 0.75) < 0.01 and abs(cb - 0.75) < 0.01
+
+
+# ---- the operator around a local optimizer step (Section 4.1) -------------------------------------
+
+def _nearest_bf16_brute(x: float) -> int:
+    """Nearest bf16 (ties to even) of a positive normal double, by trying both neighbours exactly."""
+    from fractions import Fraction
+
+    m, e = np.frexp(x)                          # x = m 2^e, 0.5 <= m < 1
+    ulp = Fraction(2) ** (int(e) - 8)           # bf16 has 8 significant bits
+    lo = int(Fraction(x) / ulp)                 # truncation, in units of ulp
+    best = None
+    for k in (lo, lo + 1):
+        dist = abs(Fraction(x) - k * ulp)
+        key = (dist, k & 1)                     # nearest, then even
+        if best is None or key < best[0]:
+            best = (key, k)
+    value = float(best[1] * ulp)
+    return int(np.array([value], dtype=np.float32).view(np.uint32)[0] >> 16)
+
+
+def test_round_to_bf16_is_one_correct_rounding():
+    rng = np.random.default_rng(77)
+    xs = list(np.exp(rng.uniform(-20, 20, 400)))
+    # traps for rounding in two steps: just above / below a bf16 midpoint, by less than an fp32 ulp
+    xs += [1.0 + 2.0 ** -8 + 2.0 ** -40, 1.0 + 2.0 ** -8 - 2.0 ** -40, 1.0 + 3 * 2.0 ** -8 + 2.0 ** -45,
+           1.0 + 3 * 2.0 ** -8 - 2.0 ** -45, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8]
+    got = oracle.round_to_dtype(np.array(xs), "bf16")
+    want = [_nearest_bf16_brute(x) for x in xs]
+    assert got.tolist() == want
+    assert oracle.round_to_dtype(-np.array(xs), "bf16").tolist() == [w | 0x8000 for w in want]
+    back = oracle.decode(got, "bf16")
+    assert np.all(np.abs(back - np.array(xs)) <= np.array(xs) * 2.0 ** -8)
+
+
+def test_delta_form_closed_cases():
+    rng = np.random.default_rng(78)
+    offsets = [0, 300, 300, 1000]
+    start = rng.standard_normal(1000).astype(np.float32)
+    # every worker took the same step, exactly representable: the result is that worker's state
+    step = (rng.integers(-8, 9, 1000) * 2.0 ** -10).astype(np.float32)
+    cur = (start.astype(np.float64) + step).astype(np.float32)
+    exact = cur.astype(np.float64) - start == step
+    out = oracle.adasum_reduce_delta([cur] * 4, start, offsets)
+    assert np.allclose(out[exact], cur[exact].astype(np.float64), rtol=0, atol=1e-12)
+    # steps with disjoint supports are orthogonal: the result is start plus all of them
+    curs = []
+    for w in range(4):
+        d = np.zeros(1000, dtype=np.float32)
+        d[w::4] = (rng.integers(1, 9, len(d[w::4])) * 2.0 ** -10).astype(np.float32)
+        curs.append(((start.astype(np.float64) + d).astype(np.float32), d))
+    out = oracle.adasum_reduce_delta([c for c, _ in curs], start, offsets)
+    eff = sum((c.astype(np.float64) - start).astype(np.float32).astype(np.float64) for c, _ in curs)
+    assert np.allclose(out, start + eff, rtol=0, atol=1e-12)
+    # start = 0: the plain reduce
+    g = [rng.standard_normal(1000).astype(np.float32) for _ in range(5)]
+    assert np.array_equal(oracle.adasum_reduce_delta(g, np.zeros(1000, np.float32), offsets),
+                          oracle.adasum_reduce(g, offsets))
+
+
+def test_delta_form_rounds_the_difference_to_the_buffer_type():
+    # 1 + 2^-11 is not an fp16; current - start must be what fp16 subtraction gives
+    start = np.array([1.0, 1024.0, 0.5], dtype=np.float16)
+    cur = np.array([1.001, 1025.0, 0.50049], dtype=np.float16)
+    d = (cur.astype(np.float64) - start.astype(np.float64)).astype(np.float16)
+    out = oracle.adasum_reduce_delta([cur, cur], start, dtype="f16")
+    assert np.allclose(out, start.astype(np.float64) + d.astype(np.float64), rtol=0, atol=1e-15)
