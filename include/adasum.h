@@ -91,8 +91,17 @@ typedef enum {
  *                fp16 / bf16; the radix fields must be 0.  Otherwise ADASUM_ERR_ARG.
  *   bit 19       ADASUM_FLAG_NO_TCGEN05: form radix-64 Gram matrices with warp-level mma.sync
  *                instead of tcgen05 and tensor memory; for comparison and debugging
+ *   bit 20       ADASUM_FLAG_TOP_DOWN_HALVES: the binary tree of Section 3.4 split from the top,
+ *                Adasum(g[lo, hi)) = Adasum(Adasum(g[lo, mid)), Adasum(g[mid, hi))) with mid =
+ *                lo + floor((hi - lo) / 2), instead of paired bottom-up with the odd operand
+ *                carried.  The two are the same tree when n_workers is a power of two (the flag
+ *                then changes nothing) and a DIFFERENT result otherwise; Algorithm 1 itself is
+ *                stated for powers of two only.  For other counts the whole reduce is one level
+ *                (same limits as ADASUM_FLAG_LINEAR_ORDER, radix fields 0); not together with
+ *                ADASUM_FLAG_LINEAR_ORDER.  Otherwise ADASUM_ERR_ARG.
  */
 #define ADASUM_FLAG_NO_TCGEN05 (1u << 19)
+#define ADASUM_FLAG_TOP_DOWN_HALVES (1u << 20)
 #define ADASUM_FLAG_SIMPLE_KERNELS (1u << 16)
 #define ADASUM_FLAG_SEPARATE_FINISH (1u << 17)
 #define ADASUM_FLAG_LINEAR_ORDER (1u << 18)

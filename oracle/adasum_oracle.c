@@ -127,6 +127,19 @@ static void adasum_tree(double **x, int n_operands, int64_t n)
     }
 }
 
+/* The recursion of Section 3.4 taken top-down, Adasum(g[lo, hi)) = Adasum(Adasum(left half),
+ * Adasum(right half)), the left half holding floor(count / 2) operands.  For a power-of-two count
+ * this is the same tree as adasum_tree; otherwise the shapes differ.  Result in x[lo]. */
+static void adasum_halves(double **x, int lo, int hi, int64_t n)
+{
+    if (hi - lo < 2)
+        return;
+    int mid = lo + (hi - lo) / 2;
+    adasum_halves(x, lo, mid, n);
+    adasum_halves(x, mid, hi, n);
+    adasum_two(x[lo], x[mid], n, x[lo]);
+}
+
 /* Linear order of Section 3.4: Adasum(g[0..n+1]) = Adasum(Adasum(g[0..n]), g[n+1]). */
 static void adasum_chain(double **x, int n_operands, int64_t n)
 {
@@ -155,8 +168,10 @@ static int reduce_tensor(const void *const *grads, int dtype, int64_t begin, int
         }
     }
     if (!rc) {
-        if (linear_order)
+        if (linear_order == 1)
             adasum_chain(x, n_workers, n);
+        else if (linear_order == 2)
+            adasum_halves(x, 0, n_workers, n);
         else
             adasum_tree(x, n_workers, n);
         memcpy(out + begin, x[0], (size_t)n * sizeof(double));
@@ -173,7 +188,8 @@ static int reduce_tensor(const void *const *grads, int dtype, int64_t begin, int
  * N-way Adasum of N fused gradient buffers, tensor by tensor.
  *   grads          N host pointers, each a buffer of offsets[num_tensors] elements of `dtype`
  *   offsets        num_tensors+1 element offsets, offsets[0] = 0, non-decreasing
- *   linear_order   0: binary tree (the form used in practice); 1: the sequential recursion
+ *   linear_order   0: binary tree, bottom-up pairs (the form used in practice); 1: the sequential
+ *                  recursion; 2: the binary tree taken top-down by halves
  *   out            offsets[num_tensors] doubles
  *   orthogonality  optional, num_tensors doubles: |Adasum(g_1..g_N)|^2 / sum_i |g_i|^2
  *                  (Section 3.6); NaN for a tensor whose leaves are all zero

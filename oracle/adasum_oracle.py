@@ -85,13 +85,17 @@ def threads_used(threads: int = 0) -> int:
 
 
 def adasum_reduce(grads, offsets=None, dtype: str | None = None, linear_order: bool = False,
-                  return_orthogonality: bool = False, threads: int = 1):
+                  return_orthogonality: bool = False, threads: int = 1, top_down: bool = False):
     """N-way Adasum of ``grads`` (a sequence of N equal-length 1-D arrays), per tensor.
 
     ``offsets`` (``num_tensors + 1`` element offsets) marks the tensors of the fused buffer;
     ``None`` means one tensor.  Returns the fp64 result (and, on request, the per-tensor
-    orthogonality ``|Adasum(g_1..g_N)|^2 / sum_i |g_i|^2`` of Section 3.6).
+    orthogonality ``|Adasum(g_1..g_N)|^2 / sum_i |g_i|^2`` of Section 3.6).  ``linear_order``: the
+    sequential recursion of Section 3.4; ``top_down``: its binary tree split by halves from the top
+    (differs from the default bottom-up pairing only when N is not a power of two).
     """
+    if linear_order and top_down:
+        raise ValueError("choose one order")
     arrs = [np.ascontiguousarray(g).reshape(-1) for g in grads]
     n_workers = len(arrs)
     if n_workers < 1:
@@ -112,7 +116,7 @@ def adasum_reduce(grads, offsets=None, dtype: str | None = None, linear_order: b
     ptrs = (ctypes.c_void_p * n_workers)(*[a.ctypes.data for a in arrs])
     rc = _load().adasum_oracle_reduce(
         ptrs, code, offs.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), num_tensors, n_workers,
-        1 if linear_order else 0, out.ctypes.data_as(ctypes.POINTER(ctypes.c_double)),
+        1 if linear_order else (2 if top_down else 0), out.ctypes.data_as(ctypes.POINTER(ctypes.c_double)),
         ortho.ctypes.data_as(ctypes.POINTER(ctypes.c_double)), threads)
     if rc != 0:
         raise MemoryError("adasum_oracle_reduce failed")

@@ -25,6 +25,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 ADASUM_F32, ADASUM_F16, ADASUM_BF16 = 0, 1, 2
 ADASUM_FLAG_SIMPLE_KERNELS, ADASUM_FLAG_SEPARATE_FINISH, ADASUM_FLAG_LINEAR_ORDER = 1 << 16, 1 << 17, 1 << 18
 ADASUM_FLAG_NO_TCGEN05 = 1 << 19
+ADASUM_FLAG_TOP_DOWN_HALVES = 1 << 20
 ADASUM_OK = 0
 ADASUM_MAX_WORKERS = 4096
 ADASUM_MAX_LEVELS = 12

@@ -131,10 +131,23 @@ struct LevelPlan {
     Level level[ADASUM_MAX_LEVELS];
 };
 
+// TreeOptions::linear for this reduce: 0 bottom-up pairs, 1 sequential, 2 top-down halves (only
+// when that is a different tree, i.e. the count is not a power of two).
+int tree_order(int n_workers, uint32_t flags)
+{
+    if (flags & ADASUM_FLAG_LINEAR_ORDER)
+        return 1;
+    if ((flags & ADASUM_FLAG_TOP_DOWN_HALVES) && n_workers > 1 && (n_workers & (n_workers - 1)) != 0)
+        return 2;
+    return 0;
+}
+
 bool plan_levels(int n_workers, adasum_dtype_t dtype, uint32_t flags, LevelPlan* plan)
 {
     const int first = (int)(flags & 0xffu), later_flag = (int)((flags >> 8) & 0xffu);
-    if ((flags >> 20) != 0)
+    if ((flags >> 21) != 0)
+        return false;
+    if ((flags & ADASUM_FLAG_LINEAR_ORDER) && (flags & ADASUM_FLAG_TOP_DOWN_HALVES))
         return false;
     if (first != 0 && (!valid_radix(first) || first > max_radix_for(dtype)))
         return false;
@@ -146,8 +159,9 @@ bool plan_levels(int n_workers, adasum_dtype_t dtype, uint32_t flags, LevelPlan*
     if (later > max_radix_for(ADASUM_F32))
         later = max_radix_for(ADASUM_F32);      // intermediates are fp32
     const int cap_auto = (flags & ADASUM_FLAG_SIMPLE_KERNELS) ? 16 : 64;
-    if (flags & ADASUM_FLAG_LINEAR_ORDER) {
-        // the running result of the sequential recursion is a combination of ALL earlier leaves:
+    if ((flags & ADASUM_FLAG_LINEAR_ORDER) || tree_order(n_workers, flags) == 2) {
+        // the running result of the sequential recursion is a combination of ALL earlier leaves
+        // (and the halves of a top-down split are not aligned groups of equal size):
         // one level whose Gram matrix covers every worker
         if (first != 0 || later_flag != 0)
             return false;
@@ -865,7 +879,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
             fin.seg_first = tab->d_seg_first;
             fin.counters = nullptr;
             fin.weights = nullptr;
-            fin.tree = TreeOptions{(flags & ADASUM_FLAG_LINEAR_ORDER) ? 1 : 0, 1, 1, 1,
+            fin.tree = TreeOptions{tree_order(n_workers, flags), 1, 1, 1,
                                    orthogonality ? reinterpret_cast<double*>(ws + lay.leaf_sums) : nullptr,
                                    orthogonality};
             float* partials = reinterpret_cast<float*>(ws + lay.partials);
@@ -931,7 +945,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         a.tc_status = (flags & ADASUM_FLAG_NO_TCGEN05)
                           ? nullptr
                           : reinterpret_cast<int*>(ws + lay.counters + lay.counters_bytes - sizeof(int));
-        a.tree.linear = (flags & ADASUM_FLAG_LINEAR_ORDER) ? 1 : 0;
+        a.tree.linear = tree_order(n_workers, flags);
         a.tree.level_is_first = l == 0;
         a.tree.level_is_last = l + 1 == plan.num_levels;
         a.tree.groups_first = plan.level[0].groups;

@@ -330,7 +330,8 @@ __device__ __forceinline__ void store_vector_from_float(void* p, int dtype, int6
 // What the coefficient step produces besides the leaf weights.
 struct TreeOptions {
     int linear;               // 1: the sequential recursion Adasum(Adasum(g[0..n]), g[n+1]) of Section 3.4
-                              //    instead of the binary tree (single-level plans only)
+                              //    instead of the binary tree; 2: the binary tree split by halves
+                              //    from the top instead of paired bottom-up (single-level plans only)
     int level_is_first;       // this level's operands are the workers' gradients
     int level_is_last;        // this level's single group produces the result
     int groups_first;         // number of groups of the first level
@@ -1256,6 +1257,56 @@ __device__ void tree_weights_from_gram(const double* gram, int members, float* _
                 if (mid < members)
                     weight[tid] *= tid < mid ? coef_a[pair] : coef_b[pair];
             }
+            __syncthreads();
+        }
+    } else if (opt.linear == 2) {
+        // The binary tree taken top-down: the node over leaves [lo, hi) combines the results of
+        // [lo, mid) and [mid, hi), mid = lo + (hi - lo) / 2.  Nodes are processed from the deepest
+        // depth up; a thread finds the node of its leaf at a depth by walking down from the root.
+        // A node's squared norm and coefficients are kept at index lo.
+        __shared__ double node_ca[R], node_cb[R];
+        int max_depth = 0;
+        while ((1 << max_depth) < members)
+            ++max_depth;
+        for (int depth = max_depth - 1; depth >= 0; --depth) {
+            int lo = 0, hi = members;
+            bool active = tid < members;
+            for (int t = 0; t < depth && active; ++t) {
+                if (hi - lo < 2) {
+                    active = false;          // this leaf's branch ended above `depth`
+                } else {
+                    const int m = lo + (hi - lo) / 2;
+                    if (tid < m)
+                        hi = m;
+                    else
+                        lo = m;
+                }
+            }
+            active = active && hi - lo >= 2;
+            const int mid = lo + (hi - lo) / 2;
+            if (tid < R) {
+                double acc = 0.0;
+                if (active && tid < mid) {
+                    for (int k = mid; k < hi; ++k)
+                        acc += weight[k] * gram[gram_index(R, tid, k)];
+                    acc *= weight[tid];
+                }
+                row_dot[tid] = acc;
+            }
+            __syncthreads();
+            if (active && tid == lo) {
+                double dot = 0.0;
+                for (int i = lo; i < mid; ++i)
+                    dot += row_dot[i];
+                double ca, cb;
+                pair_coefficients(dot, norm[lo], norm[mid], ca, cb);
+                norm[lo] = ca * ca * norm[lo] + cb * cb * norm[mid] + 2.0 * ca * cb * dot;
+                node_ca[lo] = ca;
+                node_cb[lo] = cb;
+            }
+            __syncthreads();
+            if (active)
+                weight[tid] *= tid < mid ? node_ca[lo] : node_cb[lo];
             __syncthreads();
         }
     } else {

@@ -107,6 +107,50 @@ def test_linear_order_limits(lib):
         lib.adasum_reduce(grads[:8], flags=LINEAR | lib.flags_radix(8, 0))
 
 
+TOP_DOWN = 1 << 20
+
+
+@pytest.mark.parametrize("dtype,n,tol", [("f32", 3, 1e-5), ("f32", 5, 1e-5), ("f32", 6, 1e-5), ("f32", 7, 1e-5),
+                                         ("f32", 13, 1e-5), ("f32", 24, 1e-5), ("f32", 31, 1e-5), ("f16", 11, 2e-3),
+                                         ("f16", 48, 2e-3), ("bf16", 63, 2e-3)])
+def test_top_down_halves(lib, dtype, n, tol):
+    """The tree of Section 3.4 split from the top, for worker counts that are not powers of two."""
+    offsets = workloads.offsets_from_sizes([20_000, 33, 4097, 128])
+    grads = _correlated(n, int(offsets[-1]), dtype, seed=1950 + n, rho=0.6)
+    out, ortho = lib.adasum_reduce_ex(grads, offsets, flags=TOP_DOWN)
+    torch.cuda.synchronize()
+    hosts = [_np(g, dtype) for g in grads]
+    ref, ref_ortho = oracle.adasum_reduce(hosts, offsets=offsets, dtype=dtype, top_down=True,
+                                          return_orthogonality=True, threads=0)
+    got = out.cpu().numpy().astype(np.float64)
+    for t in range(4):
+        lo, hi = int(offsets[t]), int(offsets[t + 1])
+        err = np.linalg.norm(got[lo:hi] - ref[lo:hi]) / np.linalg.norm(ref[lo:hi])
+        assert err <= tol, (t, err)
+        assert abs(float(ortho[t]) - ref_ortho[t]) <= max(10 * tol, 1e-4) * ref_ortho[t]
+    if dtype == "f32":     # the two trees differ by a fraction of a percent: visible above the fp32 tolerance only
+        tree = oracle.adasum_reduce(hosts, offsets=offsets, dtype=dtype, threads=0)
+        assert np.linalg.norm(got - tree) / np.linalg.norm(tree) > 10 * tol      # it really is another tree
+
+
+def test_top_down_halves_limits_and_powers_of_two(lib):
+    offsets = workloads.offsets_from_sizes([9000, 77])
+    grads = _correlated(16, int(offsets[-1]), "f32", seed=1990)
+    same = lib.adasum_reduce(grads, offsets, flags=TOP_DOWN)         # a power of two: the same tree, the same plan
+    want = lib.adasum_reduce(grads, offsets)
+    torch.cuda.synchronize()
+    assert torch.equal(same, want)
+    big = lib.adasum_reduce(_correlated(128, 4096, "f32", seed=1991), flags=TOP_DOWN)     # 128 = 2^7: allowed
+    torch.cuda.synchronize()
+    assert bool(torch.isfinite(big).all())
+    with pytest.raises(lib.AdasumError):                             # 33 fp32 workers do not fit one level
+        lib.adasum_reduce([torch.randn(64, device="cuda") for _ in range(33)], flags=TOP_DOWN)
+    with pytest.raises(lib.AdasumError):
+        lib.adasum_reduce(grads[:6], flags=TOP_DOWN | LINEAR)
+    with pytest.raises(lib.AdasumError):
+        lib.adasum_reduce(grads[:6], flags=TOP_DOWN | lib.flags_radix(8, 0))
+
+
 def test_reduce_can_be_replayed_from_a_cuda_graph(lib):
     """After one ordinary call (which builds the cached segment tables) the reduce is a fixed
     sequence of stream operations: capture it once, replay it on new data."""

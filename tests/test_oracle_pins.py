@@ -154,6 +154,32 @@ def test_brute_force_top_down_tree(n):
         np.testing.assert_allclose(out[lo:hi], ref, rtol=1e-12, atol=1e-14)
 
 
+@pytest.mark.parametrize("n", [3, 5, 6, 7, 11, 13, 24])
+def test_top_down_order_for_any_count(n):
+    """The top-down recursion of Section 3.4 for counts that are not powers of two: the oracle's
+    `top_down` order against the same brute force; and it is a different tree from the bottom-up
+    one with its carried operand (already for n = 3: bottom-up pairs (g0, g1) and carries g2,
+    top-down pairs (g1, g2) first)."""
+    rng = _rng(300 + n)
+    sizes = [5, 40, 1]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    shared = rng.standard_normal(offs[-1])
+    gs = [0.6 * shared + rng.standard_normal(offs[-1]) * (0.1 + w) for w in range(n)]
+    out = oracle.adasum_reduce(gs, offsets=offs, top_down=True)
+    for t in range(len(sizes)):
+        lo, hi = offs[t], offs[t + 1]
+        np.testing.assert_allclose(out[lo:hi], _top_down([g[lo:hi] for g in gs]), rtol=1e-12, atol=1e-14)
+    bottom_up = oracle.adasum_reduce(gs, offsets=offs)
+    assert np.linalg.norm(out - bottom_up) > 1e-3 * np.linalg.norm(bottom_up)
+
+
+@pytest.mark.parametrize("n", [1, 2, 4, 8, 32])
+def test_top_down_equals_bottom_up_for_powers_of_two(n):
+    rng = _rng(400 + n)
+    gs = [rng.standard_normal(50) for _ in range(n)]
+    assert np.array_equal(oracle.adasum_reduce(gs, top_down=True), oracle.adasum_reduce(gs))
+
+
 def test_tree_pairs_adjacent_workers_not_strided():
     """Level 1 pairs workers (0,1) and (2,3): with g0 = g1 and g2 = g3 orthogonal to g0 the
     result is g0 + g2; pairing (0,2),(1,3) would give (g0 + g2) as well only by accident of
