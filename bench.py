@@ -153,6 +153,8 @@ def algorithmic_bytes(record, plan_levels, total_elems, in_bytes):
         return read + level["groups"] * total_elems * 4
     if record["kernel"] == "fused_small":      # both passes in one launch: HBM sees the operands once
         return read + total_elems * 4
+    if record["kernel"] == "wsum_gram":        # pass 2 of this level and pass 1 of the next from the same registers
+        return read + level["groups"] * total_elems * 4
     if record["kernel"] == "convert":
         return total_elems * (in_bytes + 4)
     return 0
@@ -481,6 +483,10 @@ def cuda_arm(args):
     from paper_2006_02924_b200 import binding as lib
 
     flags = lib.flags_radix(args.radix_first, args.radix_later)
+    if args.no_level_fusion:
+        flags |= lib.ADASUM_FLAG_NO_LEVEL_FUSION
+    if args.no_tcgen05:
+        flags |= lib.ADASUM_FLAG_NO_TCGEN05
     peak, peak_kind = measured_peak()
     sampler = ClockSampler(local_rank)
     steps, warmup = max(args.steps, 1), max(args.warmup, 3)
@@ -586,6 +592,9 @@ def main():
                     help="override the configuration's tensor list")
     ap.add_argument("--radix-first", type=int, default=0)
     ap.add_argument("--radix-later", type=int, default=0)
+    ap.add_argument("--no-level-fusion", action="store_true",
+                    help="pass 2 of a level and pass 1 of the next always as separate kernels")
+    ap.add_argument("--no-tcgen05", action="store_true", help="radix-64 Gram matrices with mma.sync")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-other-workloads", action="store_true")
     args = ap.parse_args()

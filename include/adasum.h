@@ -99,7 +99,15 @@ typedef enum {
  *                stated for powers of two only.  For other counts the whole reduce is one level
  *                (same limits as ADASUM_FLAG_LINEAR_ORDER, radix fields 0); not together with
  *                ADASUM_FLAG_LINEAR_ORDER.  Otherwise ADASUM_ERR_ARG.
+ *   bit 21       ADASUM_FLAG_NO_LEVEL_FUSION: always run the second pass of a level and the first
+ *                pass of the next as separate kernels.  Without the flag, when a level has radix 2
+ *                or 4 and so has the next (and the buffers are 16-byte aligned), one kernel writes a level's
+ *                outputs and accumulates the next level's dot products from the same registers
+ *                (Algorithm 1's "apply" of one level and its dot products of the next), so the
+ *                intermediate vectors are read once less.  Same results up to rounding; for
+ *                comparison and debugging.
  */
+#define ADASUM_FLAG_NO_LEVEL_FUSION (1u << 21)
 #define ADASUM_FLAG_NO_TCGEN05 (1u << 19)
 #define ADASUM_FLAG_TOP_DOWN_HALVES (1u << 20)
 #define ADASUM_FLAG_SIMPLE_KERNELS (1u << 16)
@@ -318,6 +326,7 @@ const char* adasum_last_error(void);
 #define ADASUM_KERNEL_WEIGHTED_SUM 2
 #define ADASUM_KERNEL_CONVERT 3
 #define ADASUM_KERNEL_FUSED_SMALL 4   /* both passes in one cooperative launch (inputs that fit the L2) */
+#define ADASUM_KERNEL_WSUM_GRAM 5     /* second pass of `level` and first pass of level + 1 in one kernel */
 
 typedef struct {
     int32_t kernel;

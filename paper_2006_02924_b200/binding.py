@@ -26,6 +26,7 @@ ADASUM_F32, ADASUM_F16, ADASUM_BF16 = 0, 1, 2
 ADASUM_FLAG_SIMPLE_KERNELS, ADASUM_FLAG_SEPARATE_FINISH, ADASUM_FLAG_LINEAR_ORDER = 1 << 16, 1 << 17, 1 << 18
 ADASUM_FLAG_NO_TCGEN05 = 1 << 19
 ADASUM_FLAG_TOP_DOWN_HALVES = 1 << 20
+ADASUM_FLAG_NO_LEVEL_FUSION = 1 << 21
 ADASUM_OK = 0
 ADASUM_MAX_WORKERS = 4096
 ADASUM_MAX_LEVELS = 12
@@ -319,7 +320,8 @@ class _LaunchRecord(ctypes.Structure):
                 ("ms", ctypes.c_float)]
 
 
-KERNEL_NAMES = {0: "gram_partial", 1: "tree_weights", 2: "weighted_sum", 3: "convert", 4: "fused_small"}
+KERNEL_NAMES = {0: "gram_partial", 1: "tree_weights", 2: "weighted_sum", 3: "convert", 4: "fused_small",
+                5: "wsum_gram"}
 
 _lib.adasum_profile_enable.restype = ctypes.c_int
 _lib.adasum_profile_enable.argtypes = [ctypes.c_int32]

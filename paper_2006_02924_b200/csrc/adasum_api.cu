@@ -145,7 +145,7 @@ int tree_order(int n_workers, uint32_t flags)
 bool plan_levels(int n_workers, adasum_dtype_t dtype, uint32_t flags, LevelPlan* plan)
 {
     const int first = (int)(flags & 0xffu), later_flag = (int)((flags >> 8) & 0xffu);
-    if ((flags >> 21) != 0)
+    if ((flags >> 22) != 0)
         return false;
     if ((flags & ADASUM_FLAG_LINEAR_ORDER) && (flags & ADASUM_FLAG_TOP_DOWN_HALVES))
         return false;
@@ -209,7 +209,7 @@ int64_t segment_bound(int64_t total, int32_t num_tensors, int seg_len)
 }
 
 struct Layout {
-    size_t partials = 0, weights = 0, gram64 = 0, counters = 0, leaf_sums = 0, buffer[2] = {0, 0};
+    size_t partials = 0, weights = 0, weights_alt = 0, gram64 = 0, counters = 0, leaf_sums = 0, buffer[2] = {0, 0};
     size_t partials_bytes = 0, weights_bytes = 0, gram64_bytes = 0, counters_bytes = 0, leaf_sums_bytes = 0,
            buffer_bytes[2] = {0, 0};
     int64_t padded_elems = 0;
@@ -247,6 +247,8 @@ Layout make_layout(const LevelPlan& plan, int64_t total_elems, int32_t num_tenso
     lay.partials = off;
     off += align_up(lay.partials_bytes);
     lay.weights = off;
+    off += align_up(lay.weights_bytes);
+    lay.weights_alt = off;          // odd levels: a fused kernel reads one level's weights while it writes the next's
     off += align_up(lay.weights_bytes);
     lay.gram64 = off;
     off += align_up(lay.gram64_bytes);
@@ -617,7 +619,41 @@ struct LevelArgs {
     bool vec;
     cudaStream_t stream;
     int level;
+    // fusion of this level's pass 2 with the next level's pass 1 (wsum_gram_kernel)
+    bool skip_gram;              // this level's Gram sums and weights were produced by the previous level's pass 2
+    int fuse_next_radix;         // 0: plain pass 2; 2 or 4: also pass 1 of the next level, which has this radix
+    const SegmentTable* fuse_tab;
+    int next_groups;
+    float* next_weights;
+    TreeOptions next_tree;
 };
+
+// Measured on a B200: fusing pays while this level's groups are narrow (literal tree 0.60 -> 0.54 ms on
+// the ResNet-50 list with 8 workers, 14.7 -> 13.0 ms on the BERT-Large list with 16); from radix 8 on
+// the plain second pass, which keeps three blocks per SM busy, is faster than the saving.
+bool fusable_radices(int radix, int next_radix) { return radix <= 4 && (next_radix == 2 || next_radix == 4); }
+
+template <typename T, int R1, int R2>
+adasum_status_t launch_wsum_gram(const LevelArgs& a)
+{
+    constexpr int kNextGroupsPerLaunch = kMaxOperandsPerLaunch / (R1 * R2);
+    const FinishArgs next_fin{a.fuse_tab->d_seg_first, a.counters, a.next_weights, a.next_tree};
+    for (int ng0 = 0; ng0 < a.next_groups; ng0 += kNextGroupsPerLaunch) {
+        const int next_here = a.next_groups - ng0 < kNextGroupsPerLaunch ? a.next_groups - ng0 : kNextGroupsPerLaunch;
+        const int g0 = ng0 * R2, op0 = g0 * R1;
+        const int ops_here = a.operands - op0 < kMaxOperandsPerLaunch ? a.operands - op0 : kMaxOperandsPerLaunch;
+        OperandTable table;
+        for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
+            table.ptr[i] = a.operand_ptrs[op0 + (i < ops_here ? i : 0)];
+        dim3 grid((unsigned)a.fuse_tab->num_segments, (unsigned)next_here);
+        wsum_gram_kernel<T, R1, R2, true><<<grid, kThreads, 0, a.stream>>>(
+            table, ops_here, a.fuse_tab->d_segments, a.weights, a.groups, g0, static_cast<float*>(a.dst), a.dst_stride,
+            a.partials, a.next_groups, ng0, next_fin);
+        profile_mark(a.stream, ADASUM_KERNEL_WSUM_GRAM, a.level, R1, false);
+    }
+    ADASUM_CUDA_CHECK(cudaGetLastError());
+    return ADASUM_OK;
+}
 
 template <typename T, int R>
 adasum_status_t run_level_typed(const LevelArgs& a)
@@ -627,7 +663,7 @@ adasum_status_t run_level_typed(const LevelArgs& a)
     const bool fused_finish = a.counters != nullptr && a.phase == PHASE_WHOLE;
     const FinishArgs fin{a.gram_tab->d_seg_first, fused_finish ? a.counters : nullptr, a.weights, a.tree};
     // pass 1
-    for (int g0 = 0; g0 < a.groups && a.phase != PHASE_APPLY; g0 += kGroupsPerLaunch) {
+    for (int g0 = 0; g0 < a.groups && a.phase != PHASE_APPLY && !a.skip_gram; g0 += kGroupsPerLaunch) {
         const int groups_here = a.groups - g0 < kGroupsPerLaunch ? a.groups - g0 : kGroupsPerLaunch;
         const int op0 = g0 * R;
         const int ops_here = a.operands - op0 < kMaxOperandsPerLaunch ? a.operands - op0 : kMaxOperandsPerLaunch;
@@ -646,14 +682,20 @@ adasum_status_t run_level_typed(const LevelArgs& a)
     if (a.phase == PHASE_APPLY) {
         launch_tree_from_sums<R>(a.gram64, a.num_tensors, a.operands, a.groups, a.weights, a.tree, a.stream);
         profile_mark(a.stream, ADASUM_KERNEL_TREE_WEIGHTS, a.level, R, false);
-    } else if (!fused_finish) {
+    } else if (!fused_finish && !a.skip_gram) {
         int weight_launches = 0;
         ADASUM_CUDA_CHECK(launch_weights<R>(a.partials, *a.gram_tab, a.num_tensors, a.operands, a.groups,
                                             a.gram64, a.weights, a.tree, a.stream, &weight_launches,
                                             a.phase == PHASE_GRAM_SUMS));
         profile_mark(a.stream, ADASUM_KERNEL_TREE_WEIGHTS, a.level, R, false);
     }
-    // pass 2
+    // pass 2, together with the next level's pass 1 where that is possible
+    if constexpr (R <= 4) {
+        if (a.fuse_next_radix == 2)
+            return launch_wsum_gram<T, R, 2>(a);
+        if (a.fuse_next_radix == 4)
+            return launch_wsum_gram<T, R, 4>(a);
+    }
     for (int g0 = 0; g0 < a.groups && a.phase != PHASE_GRAM_SUMS; g0 += kGroupsPerLaunch) {
         const int groups_here = a.groups - g0 < kGroupsPerLaunch ? a.groups - g0 : kGroupsPerLaunch;
         const int op0 = g0 * R;
@@ -700,12 +742,24 @@ int launches_of(const LevelPlan& plan, int n_workers, uint32_t flags, int64_t to
     if (small_input_plan(plan, total, num_tensors, n_workers, elem_bytes, flags, 148 * kSmallBlocksPerSm, &seg_len))
         return 1;
     int n = 0;
+    bool gram_done = false;      // by the previous level's pass 2 (16-byte aligned buffers assumed)
     for (int l = 0; l < plan.num_levels; ++l) {
-        const int per_launch = kMaxOperandsPerLaunch / plan.level[l].radix;
+        const int radix = plan.level[l].radix;
+        const int per_launch = kMaxOperandsPerLaunch / radix;
         const int batches = (plan.level[l].groups + per_launch - 1) / per_launch;
-        n += 2 * batches;
-        if (flags & ADASUM_FLAG_SEPARATE_FINISH)        // otherwise done inside pass 1
-            n += plan.level[l].radix >= 32 ? 2 : 1;     // gram_finish (+ tree_weights)
+        if (!gram_done) {
+            n += batches;
+            if (flags & ADASUM_FLAG_SEPARATE_FINISH)        // otherwise done inside pass 1
+                n += radix >= 32 ? 2 : 1;                   // gram_finish (+ tree_weights)
+        }
+        gram_done = l + 1 < plan.num_levels && fusable_radices(radix, plan.level[l + 1].radix) &&
+                    !(flags & (ADASUM_FLAG_SEPARATE_FINISH | ADASUM_FLAG_NO_LEVEL_FUSION));
+        if (gram_done) {
+            const int next_per_launch = kMaxOperandsPerLaunch / (radix * plan.level[l + 1].radix);
+            n += (plan.level[l + 1].groups + next_per_launch - 1) / next_per_launch;
+        } else {
+            n += batches;
+        }
     }
     return n;
 }
@@ -906,6 +960,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         }
     }
 
+    bool gram_done = false;      // the previous level's pass 2 has already produced this level's weights
     for (int l = 0; l < plan.num_levels; ++l) {
         const Level& lv = plan.level[l];
         if (only_level >= 0 && l != only_level) {       // other levels' operands: the intermediates
@@ -937,7 +992,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         a.wsum_tab = wsum_tab;
         a.num_tensors = num_tensors;
         a.partials = reinterpret_cast<float*>(ws + lay.partials);
-        a.weights = reinterpret_cast<float*>(ws + lay.weights);
+        a.weights = reinterpret_cast<float*>(ws + ((l & 1) ? lay.weights_alt : lay.weights));
         a.gram64 = reinterpret_cast<double*>(ws + lay.gram64);
         a.counters = separate_finish ? nullptr : reinterpret_cast<int*>(ws + lay.counters);
         a.phase = phase;
@@ -959,6 +1014,25 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         a.vec = vec;
         a.stream = stream;
         a.level = l;
+        a.skip_gram = gram_done;
+        a.fuse_next_radix = 0;
+        a.fuse_tab = nullptr;
+        a.next_groups = 0;
+        a.next_weights = nullptr;
+        a.next_tree = a.tree;
+        gram_done = false;
+        if (!last && !sharded && !separate_finish && vec && !(flags & ADASUM_FLAG_NO_LEVEL_FUSION) &&
+            a.extras.start == nullptr && fusable_radices(lv.radix, plan.level[l + 1].radix)) {
+            st = get_segment_table(offsets, num_tensors, gram_segment_length(GRAM_SIMPLE, total), &a.fuse_tab);
+            if (st != ADASUM_OK)
+                return st;
+            a.fuse_next_radix = plan.level[l + 1].radix;
+            a.next_groups = plan.level[l + 1].groups;
+            a.next_weights = reinterpret_cast<float*>(ws + (((l + 1) & 1) ? lay.weights_alt : lay.weights));
+            a.next_tree.level_is_first = 0;
+            a.next_tree.level_is_last = l + 2 == plan.num_levels;
+            gram_done = true;
+        }
         if (l == 0) {
             if (dtype == ADASUM_F32)
                 st = run_level<float>(lv.radix, a);

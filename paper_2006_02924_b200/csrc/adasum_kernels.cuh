@@ -1595,6 +1595,142 @@ weighted_sum_kernel(const __grid_constant__ OperandTable ops, int operands,
                                               static_cast<float*>(dst_base) + (int64_t)group * dst_stride, ex);
 }
 
+// ---- pass 2 of a level fused with pass 1 of the next ------------------------------------------
+//
+// Algorithm 1 applied level after level: the combine x' = ca a + cb b of one level writes exactly
+// the vectors whose dot products [a'.b', a'.a', b'.b'] the next level needs.  This kernel forms the
+// weighted sums of R2 adjacent groups of a level (R1 operands each), stores them as the level's
+// outputs, and accumulates, from the same registers, the R2 x R2 Gram matrix of those outputs,
+// which is the next level's pass 1: the intermediates are written once and read once instead of
+// twice.  The next level's sums are finished here as well (last block per (tensor, next group)),
+// so the next level only runs its pass 2.  R2 = 2 or 4: the Gram matrix on the fp32 pipes.
+//
+// grid = (segments, next-level groups in this launch); block = kThreads.
+// weights[(tensor * groups_total + group) * R1 ...]: this level's leaf weights.
+// dst_base + group * dst_stride floats: this level's output buffers (fp32).
+// next_partials[(segment * next_groups_total + next group) * E2 + entry].
+template <typename T, int R1, int R2, bool VEC>
+__global__ void __launch_bounds__(kThreads, 2)
+wsum_gram_kernel(const __grid_constant__ OperandTable ops, int operands,
+                 const Segment* __restrict__ segments, const float* __restrict__ weights,
+                 int groups_total, int group_base, float* __restrict__ dst_base, int64_t dst_stride,
+                 float* __restrict__ next_partials, int next_groups_total, int next_group_base, FinishArgs next_fin)
+{
+    constexpr int V = Element<T>::kVec;
+    constexpr int E2 = gram_entries(R2);
+    constexpr int BATCH = R1 < 8 ? R1 : 8;
+    __shared__ float w_smem[R2][R1];
+    __shared__ float warp_sums[kWarps][E2];
+
+    const Segment seg = segments[blockIdx.x];
+    const int groups_here = (operands + R1 - 1) / R1;                 // this level's groups in this launch
+    const int g_first = blockIdx.y * R2;                              // first of them that this block combines
+    const int members_next = min(R2, groups_here - g_first);
+    for (int k = threadIdx.x; k < R1 * R2; k += kThreads) {
+        const int j = k / R1, i = k % R1;
+        const bool live = j < members_next && (g_first + j) * R1 + i < operands;
+        w_smem[j][i] = live ? weights[((int64_t)seg.tensor * groups_total + group_base + g_first + j) * R1 + i] : 0.0f;
+    }
+    __syncthreads();
+
+    float acc[E2];
+#pragma unroll
+    for (int k = 0; k < E2; ++k)
+        acc[k] = 0.0f;
+
+    const int64_t begin = seg.begin, end = seg.begin + seg.len;
+    int64_t body_begin, body_end;
+    split_segment<V, VEC>(begin, end, body_begin, body_end);
+
+    for (int64_t v = body_begin + (int64_t)threadIdx.x * V; v < body_end; v += (int64_t)kThreads * V) {
+        float y[R2][V];
+#pragma unroll
+        for (int j = 0; j < R2; ++j) {
+#pragma unroll
+            for (int c = 0; c < V; ++c)
+                y[j][c] = 0.0f;
+            if (j < members_next) {
+                const int op0 = (g_first + j) * R1;
+#pragma unroll(R1 / BATCH <= 2 ? 2 : 1)
+                for (int bb = 0; bb < R1; bb += BATCH) {
+                    uint4 raw[BATCH];
+#pragma unroll
+                    for (int i = 0; i < BATCH; ++i)
+                        if (op0 + bb + i < operands)
+                            raw[i] = load_streaming_16B(static_cast<const T*>(ops.ptr[op0 + bb + i]) + v);
+#pragma unroll
+                    for (int i = 0; i < BATCH; ++i) {
+                        if (op0 + bb + i < operands) {
+                            float x[V];
+                            decode_vector<T>(raw[i], x);
+                            const float wi = w_smem[j][bb + i];
+#pragma unroll
+                            for (int c = 0; c < V; ++c)
+                                y[j][c] = fmaf(wi, x[c], y[j][c]);
+                        }
+                    }
+                }
+                float* out = dst_base + (int64_t)(group_base + g_first + j) * dst_stride + v;
+#pragma unroll
+                for (int c = 0; c < V; c += 4)
+                    *reinterpret_cast<float4*>(out + c) = make_float4(y[j][c], y[j][c + 1], y[j][c + 2], y[j][c + 3]);
+            }
+        }
+#pragma unroll
+        for (int c = 0; c < V; ++c) {
+            float col[R2];
+#pragma unroll
+            for (int j = 0; j < R2; ++j)
+                col[j] = y[j][c];
+            gram_accumulate<R2>(col, acc);
+        }
+    }
+    // scalar head [begin, body_begin) and tail [body_end, end)
+    for (int pass = 0; pass < 2; ++pass) {
+        const int64_t lo = pass == 0 ? begin : body_end;
+        const int64_t hi = pass == 0 ? body_begin : end;
+        for (int64_t e = lo + threadIdx.x; e < hi; e += kThreads) {
+            float col[R2];
+#pragma unroll
+            for (int j = 0; j < R2; ++j) {
+                float yy = 0.0f;
+                if (j < members_next) {
+                    const int op0 = (g_first + j) * R1;
+#pragma unroll
+                    for (int i = 0; i < R1; ++i)
+                        if (op0 + i < operands)
+                            yy = fmaf(w_smem[j][i], Element<T>::one(static_cast<const T*>(ops.ptr[op0 + i]) + e), yy);
+                    dst_base[(int64_t)(group_base + g_first + j) * dst_stride + e] = yy;
+                }
+                col[j] = yy;
+            }
+            gram_accumulate<R2>(col, acc);
+        }
+    }
+
+    // block reduction: warp shuffles, then the warps' sums in warp order
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int k = 0; k < E2; ++k) {
+        float sum = acc[k];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1)
+            sum += __shfl_xor_sync(0xffffffffu, sum, d);
+        if (lane == 0)
+            warp_sums[warp][k] = sum;
+    }
+    __syncthreads();
+    float* dst = next_partials + ((int64_t)blockIdx.x * next_groups_total + next_group_base + blockIdx.y) * E2;
+    for (int k = threadIdx.x; k < E2; k += kThreads) {
+        float sum = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w)
+            sum += warp_sums[w][k];
+        dst[k] = sum;
+    }
+    finish_if_last<R2>(next_fin, next_partials, seg.tensor, next_group_base + blockIdx.y, next_groups_total, members_next);
+}
+
 // ---- both passes in one launch, for inputs that fit the L2 -------------------------------------
 //
 // One level, one group (n_workers <= 8), few enough segments that every block of the grid is

@@ -76,7 +76,8 @@ def test_plan_info(binding):
     with pytest.raises(binding.AdasumError):
         info(100, 1, 8, "f32", linear | binding.flags_radix(8, 0))
     assert info(0, 0, 4, "f32")["launches"] == 0
-    assert info(100, 1, 8, "f32", binding.flags_radix(2, 2))["launches"] == 6
+    assert info(100, 1, 8, "f32", binding.flags_radix(2, 2))["launches"] == 4      # pass 1, two fused kernels, pass 2
+    assert info(100, 1, 8, "f32", binding.flags_radix(2, 2) | (1 << 21))["launches"] == 6
     assert info(100, 1, 8, "f32", binding.flags_radix(2, 2) | (1 << 17))["launches"] == 9
     assert info(100, 1, 64, "f16")["radices"] == [64]
     assert info(100, 1, 64, "f16", 1 << 19)["radices"] == [32, 2]
@@ -107,7 +108,7 @@ def test_argument_errors_are_caught_on_the_host(binding):
     assert s(_call_reduce(binding, good, [1, 8], 2)) == "ADASUM_ERR_OFFSETS"
     assert s(_call_reduce(binding, good, [0, 8, 4], 2)) == "ADASUM_ERR_OFFSETS"
     assert s(_call_reduce(binding, good, [0, 8], 2, flags=3)) == "ADASUM_ERR_ARG"
-    assert s(_call_reduce(binding, good, [0, 8], 2, flags=1 << 21)) == "ADASUM_ERR_ARG"
+    assert s(_call_reduce(binding, good, [0, 8], 2, flags=1 << 22)) == "ADASUM_ERR_ARG"
     assert s(_call_reduce(binding, good, [0, 8], 2, flags=64)) == "ADASUM_ERR_ARG"        # radix 64 needs 16-bit inputs
     assert s(_call_reduce(binding, [0x30000000, 0], [0, 8], 2)) == "ADASUM_ERR_NULL"
     assert s(_call_reduce(binding, good, [0, 8], 2, out=0)) == "ADASUM_ERR_NULL"

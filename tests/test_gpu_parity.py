@@ -162,7 +162,7 @@ def test_more_operands_than_one_launch_carries(lib, dtype, n, first):
     offsets = workloads.offsets_from_sizes([2000, 5, 777, 64])
     grads = _correlated(n, int(offsets[-1]), dtype, seed=280 + n, rho=0.7)
     info = lib.adasum_plan_info(int(offsets[-1]), 4, n, dtype, lib.flags_radix(first, 0))
-    assert info["launches"] > 2 * len(info["radices"])
+    assert info["launches"] > len(info["radices"]) + 1      # more than one launch per pass somewhere
     _run_and_check(lib, grads, offsets, dtype, flags=lib.flags_radix(first, 0))
 
 
