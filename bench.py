@@ -234,6 +234,21 @@ def time_variants(lib, wl, steps, warmup, flags):
                                          stream=stream),
          2 * wl.n_workers * wl.total_elems * b + 2 * wl.total_elems),
     ]
+    if wl.spec.dtype == "f32" and wl.input_bytes <= 4e9:
+        # the same values as fp64 buffers: the fp64 kernels (levels of radix 4 / 2, doubles throughout)
+        grads64 = [g.double() for g in wl.grads]
+        out64 = torch.empty(wl.total_elems, dtype=torch.float64, device=dev)
+        info64 = lib.adasum_plan_info(wl.total_elems, wl.num_tensors, wl.n_workers, "f64", 0)
+        ws64 = torch.empty(max(lib.adasum_workspace_bytes(wl.total_elems, wl.num_tensors, wl.n_workers, "f64", 0), 256),
+                           dtype=torch.uint8, device=dev)
+        moved, m = 0, wl.n_workers
+        for r in info64["radices"]:             # every level: operands read twice, outputs written once
+            g = (m + r - 1) // r
+            moved += (2 * m + g) * wl.total_elems * 8
+            m = g
+        cases.append((f"fp64 buffers, fp64 output, radices {info64['radices']}",
+                      lambda: lib.adasum_reduce_delta(grads64, None, wl.offsets, out=out64, workspace=ws64,
+                                                      stream=stream), moved))
     results = []
     for name, call, two_read_bytes in cases:
         for _ in range(warmup):
@@ -248,7 +263,8 @@ def time_variants(lib, wl, steps, warmup, flags):
             stops[i].record(stream)
         torch.cuda.synchronize()
         ms = sum(a.elapsed_time(c) for a, c in zip(starts, stops)) / steps
-        results.append({"variant": name, "ms_per_reduce": ms, "input_gbs": wl.input_bytes / (ms * 1e-3) / 1e9,
+        in_bytes = wl.input_bytes * (2 if name.startswith("fp64") else 1)
+        results.append({"variant": name, "ms_per_reduce": ms, "input_gbs": in_bytes / (ms * 1e-3) / 1e9,
                         "two_read_bytes": two_read_bytes,
                         "two_read_gbs": two_read_bytes / (ms * 1e-3) / 1e9})
     return results

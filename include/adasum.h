@@ -44,11 +44,22 @@
 extern "C" {
 #endif
 
-/* Element type of the worker gradients.  The output is fp32 for every input type. */
+/* Element type of the worker gradients.  adasum_reduce, adasum_reduce_ex and adasum_pair write
+ * fp32 for every input type; adasum_reduce_delta takes the output type as an argument.
+ *
+ * ADASUM_F64 (the paper's implementation serves fp16, fp32 and fp64 tensors, Section 4.4): such
+ * buffers are reduced in doubles throughout (fp64 products and sums, leaf weights, intermediates)
+ * by kernels of their own, in levels of radix 2 or 4 (radix fields 0, 2 or 4; 0 = 4), as the
+ * bottom-up binary tree only: ADASUM_FLAG_LINEAR_ORDER, ADASUM_FLAG_TOP_DOWN_HALVES,
+ * ADASUM_FLAG_SEPARATE_FINISH and ADASUM_FLAG_SIMPLE_KERNELS are refused with ADASUM_ERR_ARG.
+ * The output is fp64 or fp32 (adasum_reduce_delta with out_dtype ADASUM_F64 or ADASUM_F32; the
+ * calls with a float* out store fp32).  The sharded calls and adasum_pair_noalloc refuse
+ * ADASUM_F64 with ADASUM_ERR_DTYPE. */
 typedef enum {
     ADASUM_F32 = 0,
     ADASUM_F16 = 1,   /* IEEE binary16 */
-    ADASUM_BF16 = 2
+    ADASUM_BF16 = 2,
+    ADASUM_F64 = 3
 } adasum_dtype_t;
 
 typedef enum {
@@ -198,7 +209,8 @@ adasum_status_t adasum_reduce_ex(const void* const* grads, const int64_t* tensor
  *                   is adasum_reduce_ex with a choice of output type
  *   out             device, total elements of out_dtype.  May be `start` itself when out_dtype ==
  *                   dtype (the parameters are updated in place); may not overlap anything else
- *   out_dtype       ADASUM_F32, ADASUM_F16 or ADASUM_BF16 (round to nearest even on store)
+ *   out_dtype       ADASUM_F32, ADASUM_F16 or ADASUM_BF16 (round to nearest even on store); for
+ *                   ADASUM_F64 inputs ADASUM_F64 or ADASUM_F32
  *   everything else as for adasum_reduce_ex, including the workspace size and the plan.
  *
  * Each difference currents[w][e] - start[e] is rounded once, to `dtype` (what `current - start`

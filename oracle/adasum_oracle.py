@@ -143,8 +143,11 @@ def decode(arr: np.ndarray, dtype: str | None = None) -> np.ndarray:
 
 
 def round_to_dtype(x: np.ndarray, dtype: str) -> np.ndarray:
-    """fp64 values rounded ONCE, to nearest even, to f32 / f16 / bf16 (bf16 as uint16 patterns)."""
+    """fp64 values rounded ONCE, to nearest even, to f32 / f16 / bf16 (bf16 as uint16 patterns);
+    f64 is returned as it is."""
     x = np.asarray(x, dtype=np.float64)
+    if dtype == "f64":
+        return x
     if dtype == "f32":
         return x.astype(np.float32)
     if dtype == "f16":
@@ -170,7 +173,8 @@ def adasum_reduce_delta(currents, start, offsets=None, dtype: str | None = None,
     parameters the step started from).  Each difference is rounded once to the buffers' own type,
     as ``current - start`` is in a framework; everything after that is fp64.  Returns fp64."""
     if dtype is None:
-        dtype = {np.dtype(np.float32): "f32", np.dtype(np.float16): "f16"}[np.asarray(start).dtype]
+        dtype = {np.dtype(np.float32): "f32", np.dtype(np.float16): "f16",
+                 np.dtype(np.float64): "f64"}[np.asarray(start).dtype]
     s = decode(start, dtype)
     deltas = [round_to_dtype(decode(c, dtype) - s, dtype) for c in currents]
     res = adasum_reduce(deltas, offsets=offsets, dtype=dtype, linear_order=linear_order,

@@ -22,7 +22,7 @@ if not os.path.exists(LIB_PATH):
 
 _lib = ctypes.CDLL(LIB_PATH)
 
-ADASUM_F32, ADASUM_F16, ADASUM_BF16 = 0, 1, 2
+ADASUM_F32, ADASUM_F16, ADASUM_BF16, ADASUM_F64 = 0, 1, 2, 3
 ADASUM_FLAG_SIMPLE_KERNELS, ADASUM_FLAG_SEPARATE_FINISH, ADASUM_FLAG_LINEAR_ORDER = 1 << 16, 1 << 17, 1 << 18
 ADASUM_FLAG_NO_TCGEN05 = 1 << 19
 ADASUM_FLAG_TOP_DOWN_HALVES = 1 << 20
@@ -30,7 +30,8 @@ ADASUM_FLAG_NO_LEVEL_FUSION = 1 << 21
 ADASUM_OK = 0
 ADASUM_MAX_WORKERS = 4096
 ADASUM_MAX_LEVELS = 12
-_DTYPES = {torch.float32: ADASUM_F32, torch.float16: ADASUM_F16, torch.bfloat16: ADASUM_BF16}
+_DTYPES = {torch.float32: ADASUM_F32, torch.float16: ADASUM_F16, torch.bfloat16: ADASUM_BF16,
+           torch.float64: ADASUM_F64}
 
 _i64p = ctypes.POINTER(ctypes.c_int64)
 _i32p = ctypes.POINTER(ctypes.c_int32)
@@ -123,7 +124,7 @@ def _dtype_code(dtype) -> int:
     if isinstance(dtype, int):
         return dtype
     if isinstance(dtype, str):
-        return {"f32": ADASUM_F32, "f16": ADASUM_F16, "bf16": ADASUM_BF16}[dtype]
+        return {"f32": ADASUM_F32, "f16": ADASUM_F16, "bf16": ADASUM_BF16, "f64": ADASUM_F64}[dtype]
     return _DTYPES[dtype]
 
 

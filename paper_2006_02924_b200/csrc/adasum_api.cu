@@ -13,6 +13,7 @@
 #include <vector>
 
 #include "adasum_kernels.cuh"
+#include "adasum_f64.cuh"
 
 namespace adasum {
 namespace {
@@ -76,7 +77,12 @@ void profile_mark(cudaStream_t stream, int kernel, int level, int radix, bool st
 constexpr size_t kAlign = 256;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
-int dtype_bytes(adasum_dtype_t dtype) { return dtype == ADASUM_F32 ? 4 : 2; }
+int dtype_bytes(adasum_dtype_t dtype) { return dtype == ADASUM_F64 ? 8 : (dtype == ADASUM_F32 ? 4 : 2); }
+
+bool known_dtype(adasum_dtype_t dtype)
+{
+    return dtype == ADASUM_F32 || dtype == ADASUM_F16 || dtype == ADASUM_BF16 || dtype == ADASUM_F64;
+}
 
 int max_radix_for(adasum_dtype_t dtype) { return dtype == ADASUM_F32 ? 32 : 64; }
 
@@ -777,7 +783,7 @@ adasum_status_t check_common(const int64_t* offsets, int32_t num_tensors, int32_
 {
     if (!offsets)
         return fail(ADASUM_ERR_NULL, "tensor_offsets is NULL");
-    if (dtype != ADASUM_F32 && dtype != ADASUM_F16 && dtype != ADASUM_BF16)
+    if (!known_dtype(dtype))
         return fail(ADASUM_ERR_DTYPE, "unknown dtype %d", (int)dtype);
     if (n_workers < 1 || n_workers > ADASUM_MAX_WORKERS)
         return fail(ADASUM_ERR_ARG, "n_workers = %d outside 1..%d", n_workers, ADASUM_MAX_WORKERS);
@@ -801,6 +807,8 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
                             adasum_dtype_t out_dtype = ADASUM_F32)
 {
     g_error[0] = '\0';
+    if (dtype == ADASUM_F64)       // whole reduces of fp64 buffers go to reduce_f64_impl
+        return fail(ADASUM_ERR_DTYPE, "the sharded calls take fp32, fp16 or bf16 gradients");
     if (!grads)
         return fail(ADASUM_ERR_NULL, "grads is NULL");
     if (orthogonality && n_workers < 2)
@@ -829,7 +837,8 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     if (need_out && !out)
         return fail(ADASUM_ERR_NULL, "out is NULL");
     if (out_dtype != ADASUM_F32 && out_dtype != ADASUM_F16 && out_dtype != ADASUM_BF16)
-        return fail(ADASUM_ERR_DTYPE, "unknown output dtype %d", (int)out_dtype);
+        return fail(ADASUM_ERR_DTYPE, out_dtype == ADASUM_F64 ? "an fp64 output needs fp64 inputs" : "unknown output dtype %d",
+                    (int)out_dtype);
     if (reinterpret_cast<uintptr_t>(out) & (uintptr_t)(dtype_bytes(out_dtype) - 1))
         return fail(ADASUM_ERR_ARG, "out is not aligned to its element size");
     const int eb = dtype_bytes(dtype);
@@ -1054,6 +1063,260 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     return ADASUM_OK;
 }
 
+// ---- fp64 gradients ------------------------------------------------------------------------------
+//
+// A family of its own (adasum_f64.cuh): levels of radix 2 or 4 on the fp64 pipes, doubles throughout.
+
+// flags of an fp64 reduce: radix fields 0 (= 4), 2 or 4; the switches that select fp32 / 16-bit
+// kernels are accepted and change nothing; the orders that need one Gram matrix over all workers
+// are not offered.
+bool plan_levels_f64(int n_workers, uint32_t flags, LevelPlan* plan)
+{
+    const int first = (int)(flags & 0xffu), later_flag = (int)((flags >> 8) & 0xffu);
+    if ((flags >> 22) != 0)
+        return false;
+    if (flags & (ADASUM_FLAG_LINEAR_ORDER | ADASUM_FLAG_TOP_DOWN_HALVES | ADASUM_FLAG_SEPARATE_FINISH |
+                 ADASUM_FLAG_SIMPLE_KERNELS))
+        return false;
+    if ((first != 0 && first != 2 && first != 4) || (later_flag != 0 && later_flag != 2 && later_flag != 4))
+        return false;
+    const int later = later_flag != 0 ? later_flag : first;
+    int m = n_workers;
+    plan->num_levels = 0;
+    while (m > 1) {
+        if (plan->num_levels == ADASUM_MAX_LEVELS)
+            return false;
+        int radix = plan->num_levels == 0 ? first : later;
+        if (radix == 0)
+            radix = 4;
+        if (radix > pow2_ceil(m))
+            radix = pow2_ceil(m);
+        Level& lv = plan->level[plan->num_levels++];
+        lv.radix = radix;
+        lv.operands = m;
+        lv.groups = (m + radix - 1) / radix;
+        m = lv.groups;
+    }
+    return true;
+}
+
+int segment_length_f64(int64_t total) { return total >= (int64_t(1) << 22) ? 4096 : 1024; }
+
+Layout make_layout_f64(const LevelPlan& plan, int64_t total_elems, int32_t num_tensors)
+{
+    Layout lay;
+    lay.padded_elems = (total_elems + 63) / 64 * 64;
+    const size_t tensors = (size_t)(num_tensors > 0 ? num_tensors : 1);
+    for (int l = 0; l < plan.num_levels; ++l) {
+        const Level& lv = plan.level[l];
+        const size_t p = (size_t)segment_bound(total_elems, num_tensors, segment_length_f64(total_elems)) * lv.groups *
+                         gram_entries(lv.radix) * sizeof(double);
+        const size_t w = tensors * lv.groups * lv.radix * sizeof(double);
+        const size_t c = (tensors * lv.groups + 1) * sizeof(int);
+        lay.partials_bytes = p > lay.partials_bytes ? p : lay.partials_bytes;
+        lay.weights_bytes = w > lay.weights_bytes ? w : lay.weights_bytes;
+        lay.counters_bytes = c > lay.counters_bytes ? c : lay.counters_bytes;
+        if (l + 1 < plan.num_levels) {
+            const size_t b = (size_t)lv.groups * lay.padded_elems * sizeof(double);
+            if (b > lay.buffer_bytes[l & 1])
+                lay.buffer_bytes[l & 1] = b;
+        }
+    }
+    if (plan.num_levels > 0)
+        lay.leaf_sums_bytes = tensors * plan.level[0].groups * sizeof(double);
+    size_t off = 0;
+    lay.partials = off;
+    off += align_up(lay.partials_bytes);
+    lay.weights = off;
+    off += align_up(lay.weights_bytes);
+    lay.counters = off;
+    off += align_up(lay.counters_bytes);
+    lay.leaf_sums = off;
+    off += align_up(lay.leaf_sums_bytes);
+    lay.buffer[0] = off;
+    off += align_up(lay.buffer_bytes[0]);
+    lay.buffer[1] = off;
+    off += align_up(lay.buffer_bytes[1]);
+    lay.total = off > 0 ? off : kAlign;
+    return lay;
+}
+
+struct LevelArgsF64 {
+    const void* const* operand_ptrs;
+    int operands, groups;
+    const SegmentTable* tab;
+    double* partials;
+    FinishArgsF64 fin;
+    void* dst;
+    int64_t dst_stride;
+    const double* start;     // first level of the delta form
+    const double* base;      // last level of the delta form
+    int out_f32;             // last level storing floats
+    bool vec;
+    cudaStream_t stream;
+    int level;
+};
+
+template <int R>
+adasum_status_t run_level_f64(const LevelArgsF64& a)
+{
+    constexpr int kGroupsPerLaunch = kMaxOperandsPerLaunch / R;
+    for (int pass = 0; pass < 2; ++pass) {
+        for (int g0 = 0; g0 < a.groups; g0 += kGroupsPerLaunch) {
+            const int groups_here = a.groups - g0 < kGroupsPerLaunch ? a.groups - g0 : kGroupsPerLaunch;
+            const int op0 = g0 * R;
+            const int ops_here = a.operands - op0 < kMaxOperandsPerLaunch ? a.operands - op0 : kMaxOperandsPerLaunch;
+            OperandTable table;
+            for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
+                table.ptr[i] = a.operand_ptrs[op0 + (i < ops_here ? i : 0)];
+            dim3 grid((unsigned)a.tab->num_segments, (unsigned)groups_here);
+            if (pass == 0) {
+                if (a.vec)
+                    gram_partial_f64_kernel<R, true><<<grid, kThreads, 0, a.stream>>>(
+                        table, ops_here, a.tab->d_segments, a.partials, a.groups, g0, a.fin, a.start);
+                else
+                    gram_partial_f64_kernel<R, false><<<grid, kThreads, 0, a.stream>>>(
+                        table, ops_here, a.tab->d_segments, a.partials, a.groups, g0, a.fin, a.start);
+                profile_mark(a.stream, ADASUM_KERNEL_GRAM_PARTIAL, a.level, R, false);
+            } else {
+                if (a.vec)
+                    weighted_sum_f64_kernel<R, true><<<grid, kThreads, 0, a.stream>>>(
+                        table, ops_here, a.tab->d_segments, a.fin.weights, a.groups, g0, a.dst, a.dst_stride, a.start,
+                        a.base, a.out_f32);
+                else
+                    weighted_sum_f64_kernel<R, false><<<grid, kThreads, 0, a.stream>>>(
+                        table, ops_here, a.tab->d_segments, a.fin.weights, a.groups, g0, a.dst, a.dst_stride, a.start,
+                        a.base, a.out_f32);
+                profile_mark(a.stream, ADASUM_KERNEL_WEIGHTED_SUM, a.level, R, false);
+            }
+        }
+    }
+    ADASUM_CUDA_CHECK(cudaGetLastError());
+    return ADASUM_OK;
+}
+
+// grads, start and (unless out_dtype is fp32) out hold doubles.
+adasum_status_t reduce_f64_impl(const void* const* grads, const int64_t* offsets, int32_t num_tensors,
+                                int32_t n_workers, void* out, adasum_dtype_t out_dtype, float* orthogonality,
+                                void* workspace, size_t workspace_bytes, uint32_t flags, cudaStream_t stream,
+                                const void* start)
+{
+    g_error[0] = '\0';
+    if (!grads)
+        return fail(ADASUM_ERR_NULL, "grads is NULL");
+    if (orthogonality && n_workers < 2)
+        return fail(ADASUM_ERR_ARG, "the orthogonality measure needs at least two workers");
+    if (reinterpret_cast<uintptr_t>(orthogonality) & 3u)
+        return fail(ADASUM_ERR_ARG, "orthogonality is not 4-byte aligned");
+    adasum_status_t st = check_common(offsets, num_tensors, n_workers, ADASUM_F64);
+    if (st != ADASUM_OK)
+        return st;
+    if (out_dtype != ADASUM_F64 && out_dtype != ADASUM_F32)
+        return fail(ADASUM_ERR_DTYPE, "fp64 inputs are reduced to an fp64 or fp32 output");
+    LevelPlan plan;
+    if (!plan_levels_f64(n_workers, flags, &plan))
+        return fail(ADASUM_ERR_ARG, "invalid flags 0x%x for %d fp64 workers (radix 2 or 4, binary tree only)", flags,
+                    n_workers);
+    const int64_t total = offsets[num_tensors];
+    if (total == 0)
+        return ADASUM_OK;
+    if (!out)
+        return fail(ADASUM_ERR_NULL, "out is NULL");
+    const int out_f32 = out_dtype == ADASUM_F32;
+    if (reinterpret_cast<uintptr_t>(out) & (uintptr_t)(out_f32 ? 3 : 7))
+        return fail(ADASUM_ERR_ARG, "out is not aligned to its element size");
+    const size_t in_bytes = (size_t)total * 8, out_bytes = (size_t)total * (out_f32 ? 4 : 8);
+    bool vec = aligned16(out);
+    if (start != nullptr) {
+        if (reinterpret_cast<uintptr_t>(start) & 7u)
+            return fail(ADASUM_ERR_ARG, "start is not 8-byte aligned");
+        const bool in_place = out == start && !out_f32;
+        if (!in_place && ranges_overlap(start, in_bytes, out, out_bytes))
+            return fail(ADASUM_ERR_ARG, "out overlaps start without being the same buffer of the same type");
+        vec = vec && aligned16(start);
+    }
+    for (int w = 0; w < n_workers; ++w) {
+        if (!grads[w])
+            return fail(ADASUM_ERR_NULL, "grads[%d] is NULL", w);
+        if (reinterpret_cast<uintptr_t>(grads[w]) & 7u)
+            return fail(ADASUM_ERR_ARG, "grads[%d] is not aligned to its element size", w);
+        if (ranges_overlap(grads[w], in_bytes, out, out_bytes))
+            return fail(ADASUM_ERR_ARG, "out overlaps grads[%d]", w);
+        if (start != nullptr && ranges_overlap(start, in_bytes, grads[w], in_bytes))
+            return fail(ADASUM_ERR_ARG, "start overlaps grads[%d]", w);
+        vec = vec && aligned16(grads[w]);
+    }
+    const Layout lay = make_layout_f64(plan, total, num_tensors);
+    if (n_workers > 1) {
+        if (!workspace)
+            return fail(ADASUM_ERR_WORKSPACE, "workspace is NULL");
+        if (workspace_bytes < lay.total)
+            return fail(ADASUM_ERR_WORKSPACE, "workspace has %zu bytes, need %zu", workspace_bytes, lay.total);
+        if (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1))
+            return fail(ADASUM_ERR_ARG, "workspace is not %zu-byte aligned", kAlign);
+        if (ranges_overlap(workspace, lay.total, out, out_bytes))
+            return fail(ADASUM_ERR_ARG, "workspace overlaps out");
+        for (int w = 0; w < n_workers; ++w)
+            if (ranges_overlap(workspace, lay.total, grads[w], in_bytes))
+                return fail(ADASUM_ERR_ARG, "workspace overlaps grads[%d]", w);
+        if (start != nullptr && ranges_overlap(workspace, lay.total, start, in_bytes))
+            return fail(ADASUM_ERR_ARG, "workspace overlaps start");
+    }
+    profile_mark(stream, -1, 0, 0, true);
+    if (n_workers == 1) {
+        const int64_t blocks = (total + kThreads - 1) / kThreads;
+        const unsigned grid = (unsigned)(blocks < 148 * 16 ? blocks : 148 * 16);
+        convert_f64_kernel<<<grid, kThreads, 0, stream>>>(static_cast<const double*>(grads[0]), out, total,
+                                                          static_cast<const double*>(start), out_f32);
+        ADASUM_CUDA_CHECK(cudaGetLastError());
+        profile_mark(stream, ADASUM_KERNEL_CONVERT, 0, 1, false);
+        return ADASUM_OK;
+    }
+    char* ws = static_cast<char*>(workspace);
+    ADASUM_CUDA_CHECK(cudaMemsetAsync(ws + lay.counters, 0, lay.counters_bytes, stream));
+    if (orthogonality && num_tensors > 0)
+        ADASUM_CUDA_CHECK(cudaMemsetAsync(orthogonality, 0xff, sizeof(float) * (size_t)num_tensors, stream));
+    if (num_tensors == 0)
+        return ADASUM_OK;
+    const SegmentTable* tab = nullptr;
+    st = get_segment_table(offsets, num_tensors, segment_length_f64(total), &tab);
+    if (st != ADASUM_OK)
+        return st;
+    std::vector<const void*> operand_ptrs(grads, grads + n_workers);
+    for (int l = 0; l < plan.num_levels; ++l) {
+        const Level& lv = plan.level[l];
+        const bool last = l + 1 == plan.num_levels;
+        LevelArgsF64 a;
+        a.operand_ptrs = operand_ptrs.data();
+        a.operands = lv.operands;
+        a.groups = lv.groups;
+        a.tab = tab;
+        a.partials = reinterpret_cast<double*>(ws + lay.partials);
+        a.fin.seg_first = tab->d_seg_first;
+        a.fin.counters = reinterpret_cast<int*>(ws + lay.counters);
+        a.fin.weights = reinterpret_cast<double*>(ws + lay.weights);
+        a.fin.tree = TreeOptions{0, l == 0, last, plan.level[0].groups,
+                                 orthogonality ? reinterpret_cast<double*>(ws + lay.leaf_sums) : nullptr, orthogonality};
+        a.dst = last ? out : static_cast<void*>(ws + lay.buffer[l & 1]);
+        a.dst_stride = last ? 0 : lay.padded_elems;
+        a.start = l == 0 ? static_cast<const double*>(start) : nullptr;
+        a.base = last ? static_cast<const double*>(start) : nullptr;
+        a.out_f32 = last ? out_f32 : 0;
+        a.vec = vec;
+        a.stream = stream;
+        a.level = l;
+        st = lv.radix == 2 ? run_level_f64<2>(a) : run_level_f64<4>(a);
+        if (st != ADASUM_OK)
+            return st;
+        if (!last) {
+            operand_ptrs.resize((size_t)lv.groups);
+            for (int g = 0; g < lv.groups; ++g)
+                operand_ptrs[g] = static_cast<double*>(a.dst) + (int64_t)g * lay.padded_elems;
+        }
+    }
+    return ADASUM_OK;
+}
+
 // ---- pair operator without any device allocation -------------------------------------------------
 //
 // Scratch for adasum_pair_noalloc: the segment table, the per-segment partial sums and the
@@ -1125,6 +1388,8 @@ adasum_status_t pair_noalloc_impl(const void* a, const void* b, const int64_t* o
     adasum_status_t st = check_common(offsets, num_tensors, 2, dtype);
     if (st != ADASUM_OK)
         return st;
+    if (dtype == ADASUM_F64)
+        return fail(ADASUM_ERR_DTYPE, "adasum_pair_noalloc takes fp32, fp16 or bf16 inputs");
     const int64_t total = offsets[num_tensors];
     if (num_tensors > kNoallocMaxTensors)
         return fail(ADASUM_ERR_ARG, "num_tensors = %d exceeds the static scratch limit of %d tensors", num_tensors,
@@ -1192,9 +1457,11 @@ size_t adasum_workspace_bytes(int64_t total_elems, int32_t num_tensors, int32_t 
     using namespace adasum;
     if (total_elems < 0 || num_tensors < 0 || n_workers < 1 || n_workers > ADASUM_MAX_WORKERS)
         return 0;
-    if (dtype != ADASUM_F32 && dtype != ADASUM_F16 && dtype != ADASUM_BF16)
+    if (!known_dtype(dtype))
         return 0;
     LevelPlan plan;
+    if (dtype == ADASUM_F64)
+        return plan_levels_f64(n_workers, flags, &plan) ? make_layout_f64(plan, total_elems, num_tensors).total : 0;
     if (!plan_levels(n_workers, dtype, flags, &plan))
         return 0;
     return make_layout(plan, total_elems, num_tensors).total;
@@ -1208,18 +1475,23 @@ adasum_status_t adasum_plan_info(int64_t total_elems, int32_t num_tensors, int32
     g_error[0] = '\0';
     if (total_elems < 0 || num_tensors < 0 || n_workers < 1 || n_workers > ADASUM_MAX_WORKERS)
         return fail(ADASUM_ERR_ARG, "invalid sizes");
-    if (dtype != ADASUM_F32 && dtype != ADASUM_F16 && dtype != ADASUM_BF16)
+    if (!known_dtype(dtype))
         return fail(ADASUM_ERR_DTYPE, "unknown dtype %d", (int)dtype);
     LevelPlan plan;
-    if (!plan_levels(n_workers, dtype, flags, &plan))
+    if (dtype == ADASUM_F64 ? !plan_levels_f64(n_workers, flags, &plan) : !plan_levels(n_workers, dtype, flags, &plan))
         return fail(ADASUM_ERR_ARG, "invalid flags 0x%x", flags);
     if (radices)
         for (int l = 0; l < plan.num_levels; ++l)
             radices[l] = plan.level[l].radix;
     if (num_levels)
         *num_levels = plan.num_levels;
-    if (num_launches)
-        *num_launches = total_elems == 0 ? 0 : launches_of(plan, n_workers, flags, total_elems, num_tensors, dtype_bytes(dtype));
+    if (num_launches) {
+        // fp64: every level is two passes, nothing fused
+        const uint32_t count_flags = dtype == ADASUM_F64 ? (flags | ADASUM_FLAG_NO_LEVEL_FUSION) : flags;
+        *num_launches = total_elems == 0 ? 0
+                                         : launches_of(plan, n_workers, count_flags, dtype == ADASUM_F64 ? -1 : total_elems,
+                                                       num_tensors, dtype_bytes(dtype));
+    }
     return ADASUM_OK;
 }
 
@@ -1228,6 +1500,9 @@ adasum_status_t adasum_reduce(const void* const* grads, const int64_t* tensor_of
                               float* out, void* workspace, size_t workspace_bytes, uint32_t flags,
                               void* stream)
 {
+    if (dtype == ADASUM_F64)
+        return adasum::reduce_f64_impl(grads, tensor_offsets, num_tensors, n_workers, out, ADASUM_F32, nullptr,
+                                       workspace, workspace_bytes, flags, static_cast<cudaStream_t>(stream), nullptr);
     return adasum::reduce_impl(grads, tensor_offsets, num_tensors, n_workers, dtype, out, nullptr, workspace,
                                workspace_bytes, flags, static_cast<cudaStream_t>(stream));
 }
@@ -1237,6 +1512,9 @@ adasum_status_t adasum_reduce_ex(const void* const* grads, const int64_t* tensor
                                  float* out, float* orthogonality, void* workspace, size_t workspace_bytes,
                                  uint32_t flags, void* stream)
 {
+    if (dtype == ADASUM_F64)
+        return adasum::reduce_f64_impl(grads, tensor_offsets, num_tensors, n_workers, out, ADASUM_F32, orthogonality,
+                                       workspace, workspace_bytes, flags, static_cast<cudaStream_t>(stream), nullptr);
     return adasum::reduce_impl(grads, tensor_offsets, num_tensors, n_workers, dtype, out, orthogonality, workspace,
                                workspace_bytes, flags, static_cast<cudaStream_t>(stream));
 }
@@ -1247,6 +1525,9 @@ adasum_status_t adasum_reduce_delta(const void* const* currents, const void* sta
                                     float* orthogonality, void* workspace, size_t workspace_bytes, uint32_t flags,
                                     void* stream)
 {
+    if (dtype == ADASUM_F64)
+        return adasum::reduce_f64_impl(currents, tensor_offsets, num_tensors, n_workers, out, out_dtype, orthogonality,
+                                       workspace, workspace_bytes, flags, static_cast<cudaStream_t>(stream), start);
     return adasum::reduce_impl(currents, tensor_offsets, num_tensors, n_workers, dtype, out, orthogonality,
                                workspace, workspace_bytes, flags, static_cast<cudaStream_t>(stream),
                                adasum::PHASE_WHOLE, -1, nullptr, nullptr, start, out_dtype);
@@ -1276,6 +1557,9 @@ adasum_status_t adasum_pair(const void* a, const void* b, const int64_t* tensor_
                             size_t workspace_bytes, uint32_t flags, void* stream)
 {
     const void* grads[2] = {a, b};
+    if (dtype == ADASUM_F64)
+        return adasum::reduce_f64_impl(grads, tensor_offsets, num_tensors, 2, out, ADASUM_F32, nullptr, workspace,
+                                       workspace_bytes, flags, static_cast<cudaStream_t>(stream), nullptr);
     return adasum::reduce_impl(grads, tensor_offsets, num_tensors, 2, dtype, out, nullptr, workspace,
                                workspace_bytes, flags, static_cast<cudaStream_t>(stream));
 }
@@ -1296,8 +1580,10 @@ adasum_status_t adasum_device_status(int64_t total_elems, int32_t num_tensors, i
         return fail(ADASUM_ERR_NULL, "workspace is NULL");
     if (total_elems < 0 || num_tensors < 0 || n_workers < 1 || n_workers > ADASUM_MAX_WORKERS)
         return fail(ADASUM_ERR_ARG, "invalid sizes");
-    if (dtype != ADASUM_F32 && dtype != ADASUM_F16 && dtype != ADASUM_BF16)
+    if (!known_dtype(dtype))
         return fail(ADASUM_ERR_DTYPE, "unknown dtype %d", (int)dtype);
+    if (dtype == ADASUM_F64)        // the fp64 kernels have no bounded waits
+        return ADASUM_OK;
     LevelPlan plan;
     if (!plan_levels(n_workers, dtype, flags, &plan))
         return fail(ADASUM_ERR_ARG, "invalid flags 0x%x", flags);

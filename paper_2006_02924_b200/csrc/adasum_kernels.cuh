@@ -1203,8 +1203,8 @@ __device__ __forceinline__ void pair_coefficients(double dot, double norm_a, dou
 // Also written, when asked for: the sum of the leaves' squared norms (first level) and the
 // orthogonality measure |result|^2 / sum_i |g_i|^2 of Section 3.6 (last level; NaN when every
 // leaf is zero).
-template <int R>
-__device__ void tree_weights_from_gram(const double* gram, int members, float* __restrict__ dst,
+template <int R, typename W = float>
+__device__ void tree_weights_from_gram(const double* gram, int members, W* __restrict__ dst,
                                        const TreeOptions& opt, int tensor, int group)
 {
     __shared__ double weight[R], norm[R], row_dot[R], coef_a[R / 2 > 0 ? R / 2 : 1], coef_b[R / 2 > 0 ? R / 2 : 1];
@@ -1333,7 +1333,7 @@ __device__ void tree_weights_from_gram(const double* gram, int members, float* _
         }
     }
     if (tid < R)
-        dst[tid] = tid < members ? (float)weight[tid] : 0.0f;
+        dst[tid] = tid < members ? (W)weight[tid] : (W)0;
     if (tid == 0) {
         if (opt.leaf_norm_sums != nullptr && opt.level_is_first)
             opt.leaf_norm_sums[(int64_t)tensor * opt.groups_first + group] = leaf_sum;

@@ -84,8 +84,8 @@ SPECS = {
                        zero_tensor_fraction=0.05, seed_index=5),
 }
 
-TORCH_DTYPES = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}
-DTYPE_BYTES = {"f32": 4, "f16": 2, "bf16": 2}
+TORCH_DTYPES = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16, "f64": torch.float64}
+DTYPE_BYTES = {"f32": 4, "f16": 2, "bf16": 2, "f64": 8}
 
 
 @dataclasses.dataclass

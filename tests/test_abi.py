@@ -52,6 +52,8 @@ def test_workspace_bytes(binding):
     assert ws(10, 1, 0, "f32") == 0
     assert ws(10, 1, 2, 7) == 0
     assert ws(10, 1, 2, "f32", 3) == 0                       # radix 3 is not a power of two
+    assert ws(1_000_000, 4, 16, "f64") >= 4 * 1_000_000 * 8      # four fp64 intermediates after a radix-4 level
+    assert ws(10, 1, 2, "f64", 8) == 0                           # fp64: radix 2 or 4 only
     small, big = ws(1_000_000, 1, 2, "f32"), ws(100_000_000, 1, 2, "f32")
     assert 0 < small <= big
     # the literal tree keeps N/2 + N/4 intermediates, the radix-16 plan only N/16
@@ -85,6 +87,13 @@ def test_plan_info(binding):
     assert info(100, 1, 64, "f16", 1 << 19)["launches"] == 4
     assert info(100, 1, 64, "f16", (1 << 17) | (1 << 19))["launches"] == 4 + 3
     assert info(100, 1, 256, "f32")["radices"] == [16, 16]
+    # fp64 buffers: levels of radix 2 or 4, two launches each
+    assert info(100, 1, 64, "f64")["radices"] == [4, 4, 4]
+    assert info(100, 1, 64, "f64")["launches"] == 6
+    assert info(100, 1, 5, "f64", binding.flags_radix(2, 0))["radices"] == [2, 2, 2]
+    for bad in (binding.flags_radix(8, 0), 1 << 18, 1 << 20, 1 << 17):
+        with pytest.raises(binding.AdasumError):
+            info(100, 1, 8, "f64", bad)
 
 
 def _call_reduce(binding, ptrs, offsets, n, dtype=0, out=0x10000000, ws=0x20000000, ws_bytes=1 << 40, flags=0,
