@@ -279,6 +279,15 @@ def test_c2_full_size_every_tensor(lib):
     print(f"c2 full: global {glob:.2e} worst tensor {worst:.2e}")
 
 
+def test_c2_full_size_literal_tree(lib):
+    """The same workload as the level-by-level tree of Algorithm 1 (radix 2 everywhere), where every
+    level's combine is fused with the next level's dot products; and the same with separate kernels."""
+    wl = workloads.generate("c2", device="cuda")
+    for flags in (lib.flags_radix(2, 2), lib.flags_radix(2, 2) | lib.ADASUM_FLAG_NO_LEVEL_FUSION):
+        glob, worst = _run_and_check(lib, wl.grads, wl.offsets, "f32", flags=flags, strict=True)
+        print(f"c2 full, literal tree (flags {flags:#x}): global {glob:.2e} worst tensor {worst:.2e}")
+
+
 def _sampled_tensor_check(lib, name, sample_count, max_len):
     """Full-size run in the launch configuration the benchmark uses; a sample of tensors (every
     size class up to max_len elements, seeded choice) is reduced by the oracle and compared."""
