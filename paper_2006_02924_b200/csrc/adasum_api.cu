@@ -556,7 +556,7 @@ bool small_input_plan(const LevelPlan& plan, int64_t total, int32_t num_tensors,
 
 template <typename T, int R, bool VEC>
 cudaError_t launch_fused_small(const OperandTable& ops, int operands, const SegmentTable& tab, float* partials,
-                               const FinishArgs& fin, void* out, const PassExtras& ex, cudaStream_t stream)
+                               const FinishArgs& fin, void* out, const PassExtras& ex, int* status, cudaStream_t stream)
 {
     const void* kernel = (const void*)fused_small_kernel<T, R, VEC, false>;
     if constexpr (VEC) {
@@ -568,20 +568,20 @@ cudaError_t launch_fused_small(const OperandTable& ops, int operands, const Segm
     int operands_arg = operands;
     const Segment* segments = tab.d_segments;
     PassExtras ex_arg = ex;
-    void* args[] = {(void*)&ops,      (void*)&operands_arg, (void*)&segments, (void*)&partials,
-                    (void*)&fin,      (void*)&out,          (void*)&ex_arg};
+    void* args[] = {(void*)&ops, (void*)&operands_arg, (void*)&segments, (void*)&partials,
+                    (void*)&fin, (void*)&out,          (void*)&ex_arg,   (void*)&status};
     return cudaLaunchCooperativeKernel(kernel, dim3((unsigned)tab.num_segments), dim3(kThreads), args, 0, stream);
 }
 
 template <typename T, bool VEC>
 cudaError_t launch_fused_small_radix(int radix, const OperandTable& ops, int operands, const SegmentTable& tab,
                                      float* partials, const FinishArgs& fin, void* out, const PassExtras& ex,
-                                     cudaStream_t stream)
+                                     int* status, cudaStream_t stream)
 {
     switch (radix) {
-    case 2: return launch_fused_small<T, 2, VEC>(ops, operands, tab, partials, fin, out, ex, stream);
-    case 4: return launch_fused_small<T, 4, VEC>(ops, operands, tab, partials, fin, out, ex, stream);
-    case 8: return launch_fused_small<T, 8, VEC>(ops, operands, tab, partials, fin, out, ex, stream);
+    case 2: return launch_fused_small<T, 2, VEC>(ops, operands, tab, partials, fin, out, ex, status, stream);
+    case 4: return launch_fused_small<T, 4, VEC>(ops, operands, tab, partials, fin, out, ex, status, stream);
+    case 8: return launch_fused_small<T, 8, VEC>(ops, operands, tab, partials, fin, out, ex, status, stream);
     default: return cudaErrorInvalidValue;
     }
 }
@@ -904,8 +904,15 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
 
     char* ws = static_cast<char*>(workspace);
     const bool separate_finish = (flags & ADASUM_FLAG_SEPARATE_FINISH) != 0 || sharded;
-    if (lay.counters_bytes > 0 && phase != PHASE_APPLY)      // the workspace arrives with unknown contents
-        ADASUM_CUDA_CHECK(cudaMemsetAsync(ws + lay.counters, 0, lay.counters_bytes, stream));
+    // Inputs that fit the L2 are served by one cooperative launch that needs no ticket counters.
+    int small_seg_len = 0;
+    const int small_blocks = (sharded || total == 0 || num_tensors == 0) ? 0 : resident_small_blocks();
+    const bool small_candidate =
+        small_blocks > 0 && small_input_plan(plan, total, num_tensors, n_workers, eb, flags, small_blocks, &small_seg_len);
+    // the workspace arrives with unknown contents
+    auto clear_counters = [&]() { return cudaMemsetAsync(ws + lay.counters, 0, lay.counters_bytes, stream); };
+    if (lay.counters_bytes > 0 && phase != PHASE_APPLY && !small_candidate)
+        ADASUM_CUDA_CHECK(clear_counters());
     if (orthogonality && num_tensors > 0 && (!sharded || (phase == PHASE_APPLY && only_level == 0)))
         ADASUM_CUDA_CHECK(cudaMemsetAsync(orthogonality, 0xff, sizeof(float) * (size_t)num_tensors, stream));
     if (phase == PHASE_GRAM_SUMS) {
@@ -926,10 +933,8 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     std::vector<const void*> operand_ptrs(grads, grads + n_workers);
 
     // Inputs that fit the L2: one cooperative launch does both passes and HBM sees the operands once.
-    int small_seg_len = 0;
-    const int small_blocks = sharded ? 0 : resident_small_blocks();
-    if (small_blocks > 0 &&
-        small_input_plan(plan, total, num_tensors, n_workers, eb, flags, small_blocks, &small_seg_len)) {
+    if (small_candidate) {
+        int* dev_status = reinterpret_cast<int*>(ws + lay.counters + lay.counters_bytes - sizeof(int));
         const SegmentTable* tab = nullptr;
         st = get_segment_table(offsets, num_tensors, small_seg_len, &tab);
         if (st != ADASUM_OK)
@@ -951,14 +956,14 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
             ex.start = start;
             cudaError_t err;
             if (dtype == ADASUM_F32)
-                err = vec ? launch_fused_small_radix<float, true>(radix, table, n_workers, *tab, partials, fin, out, ex, stream)
-                          : launch_fused_small_radix<float, false>(radix, table, n_workers, *tab, partials, fin, out, ex, stream);
+                err = vec ? launch_fused_small_radix<float, true>(radix, table, n_workers, *tab, partials, fin, out, ex, dev_status, stream)
+                          : launch_fused_small_radix<float, false>(radix, table, n_workers, *tab, partials, fin, out, ex, dev_status, stream);
             else if (dtype == ADASUM_F16)
-                err = vec ? launch_fused_small_radix<__half, true>(radix, table, n_workers, *tab, partials, fin, out, ex, stream)
-                          : launch_fused_small_radix<__half, false>(radix, table, n_workers, *tab, partials, fin, out, ex, stream);
+                err = vec ? launch_fused_small_radix<__half, true>(radix, table, n_workers, *tab, partials, fin, out, ex, dev_status, stream)
+                          : launch_fused_small_radix<__half, false>(radix, table, n_workers, *tab, partials, fin, out, ex, dev_status, stream);
             else
-                err = vec ? launch_fused_small_radix<__nv_bfloat16, true>(radix, table, n_workers, *tab, partials, fin, out, ex, stream)
-                          : launch_fused_small_radix<__nv_bfloat16, false>(radix, table, n_workers, *tab, partials, fin, out, ex, stream);
+                err = vec ? launch_fused_small_radix<__nv_bfloat16, true>(radix, table, n_workers, *tab, partials, fin, out, ex, dev_status, stream)
+                          : launch_fused_small_radix<__nv_bfloat16, false>(radix, table, n_workers, *tab, partials, fin, out, ex, dev_status, stream);
             if (err == cudaSuccess) {
                 profile_mark(stream, ADASUM_KERNEL_FUSED_SMALL, 0, radix, false);
                 return ADASUM_OK;
@@ -967,6 +972,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
                 return fail(ADASUM_ERR_CUDA, "cooperative launch: %s", cudaGetErrorString(err));
             (void)cudaGetLastError();       // too many blocks for this device after all: the two-pass path serves it
         }
+        ADASUM_CUDA_CHECK(clear_counters());      // the two-pass path draws tickets
     }
 
     bool gram_done = false;      // the previous level's pass 2 has already produced this level's weights

@@ -1744,9 +1744,14 @@ template <typename T, int R, bool VEC, bool DELTA = false>
 __global__ void __launch_bounds__(kThreads, (sizeof(T) == 2 && R == 8) ? 2 : 3)
 fused_small_kernel(const __grid_constant__ OperandTable ops, int operands,
                    const Segment* __restrict__ segments, float* __restrict__ partials, FinishArgs fin,
-                   void* out, PassExtras ex)
+                   void* out, PassExtras ex, int* __restrict__ status)
 {
     constexpr int E = gram_entries(R);
+    // This path uses no ticket counters, so the host does not clear them (one operation less in
+    // front of a reduce that takes microseconds); the device status word, which lives beside
+    // them and which adasum_device_status reads, is cleared here instead.
+    if (blockIdx.x == 0 && threadIdx.x == 0)
+        *status = 0;
     const Segment seg = segments[blockIdx.x];
     const int members = min(R, operands);
     gram_of_segment<T, R, VEC, DELTA>(ops, 0, members, seg, partials + (int64_t)blockIdx.x * E,

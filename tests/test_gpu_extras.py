@@ -197,3 +197,21 @@ def test_radix_64_tensor_memory_kernel(lib, dtype, n):
         lo, hi = int(offsets[t]), int(offsets[t + 1])
         assert np.linalg.norm(got[lo:hi] - ref[lo:hi]) / np.linalg.norm(ref[lo:hi]) <= 2e-3, t
     assert float(torch.linalg.norm(out - other) / torch.linalg.norm(other)) <= 1e-4
+
+
+@pytest.mark.parametrize("n,total", [(2, 1_000_000), (8, 300_000), (8, 40_000_000)])
+def test_device_status_is_clean_on_a_dirty_workspace(lib, n, total):
+    """The workspace arrives with arbitrary contents; after a reduce the status word reads 0, on the
+    single-launch path (which clears it in the kernel) as on the two-pass path (cleared by the host)."""
+    grads = _correlated(n, total, "f32", seed=1700 + n)
+    need = lib.adasum_workspace_bytes(total, 1, n, "f32")
+    ws = torch.full((need,), 0xAB, dtype=torch.uint8, device="cuda")
+    lib.adasum_profile_enable(16)
+    out = lib.adasum_reduce(grads, workspace=ws)
+    assert lib.adasum_device_status(total, 1, n, "f32", ws) == 0
+    kinds = {r["kernel"] for r in lib.adasum_profile_collect(16)}
+    assert ("fused_small" in kinds) == (n * total * 4 <= 96 << 20), kinds
+    ref = oracle.adasum_reduce([_np(g, "f32") for g in grads], dtype="f32", threads=0)
+    assert np.linalg.norm(out.cpu().numpy() - ref) / np.linalg.norm(ref) <= 1e-5
+    again = lib.adasum_reduce(grads, workspace=ws)             # the same workspace a second time
+    assert torch.equal(out, again)
