@@ -14,11 +14,17 @@
 //   weighted_sum   stream the operands a second time; out = sum_i weight_i x_i.
 //
 // The Gram matrix of a group is a dense contraction X X^T (R x P times P x R).  For R <= 8 it is
-// cheap enough for the fp32 pipes (gram_partial_kernel); for R >= 8 it runs on the tensor cores (gram_partial_mma_kernel): fp16 / bf16 products are exact in
-// the fp32 accumulator, fp32 inputs are split into two tf32 terms (three products).
+// cheap enough for the fp32 pipes (gram_partial_kernel); for R >= 8 it runs on the tensor cores
+// (gram_partial_mma_kernel; gram_partial_tc64_kernel for 64 fp16 / bf16 rows): fp16 / bf16 products
+// are exact in the fp32 accumulator, fp32 inputs are split into two tf32 terms (three products).
 //
-// The kernels never wait on one another and use no floating-point atomics, so results are
-// deterministic and there is nothing that can spin.
+// Two more kernels merge neighbouring steps: fused_small_kernel (both passes of a small input in
+// one cooperative launch) and wsum_gram_kernel (pass 2 of a level with pass 1 of the next).
+//
+// No kernel waits on another kernel and none uses floating-point atomics, so results are
+// deterministic.  The only waits are inside a launch: the grid barrier of the cooperative
+// fused_small_kernel, and the bounded mbarrier waits between the copying warps and the tensor
+// core in gram_partial_tc64_kernel.
 #pragma once
 
 #include <cooperative_groups.h>
