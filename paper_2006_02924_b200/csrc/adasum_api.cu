@@ -930,6 +930,8 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     }
     if (total == 0 || num_tensors == 0)
         return ADASUM_OK;
+    // per-launch timing: the first kernel's interval starts here, after the clearing of counters above
+    profile_mark(stream, -1, 0, 0, true);
     std::vector<const void*> operand_ptrs(grads, grads + n_workers);
 
     // Inputs that fit the L2: one cooperative launch does both passes and HBM sees the operands once.
@@ -1288,6 +1290,8 @@ adasum_status_t reduce_f64_impl(const void* const* grads, const int64_t* offsets
     st = get_segment_table(offsets, num_tensors, segment_length_f64(total), &tab);
     if (st != ADASUM_OK)
         return st;
+    // per-launch timing: the first kernel's interval starts here, after the clearing of counters above
+    profile_mark(stream, -1, 0, 0, true);
     std::vector<const void*> operand_ptrs(grads, grads + n_workers);
     for (int l = 0; l < plan.num_levels; ++l) {
         const Level& lv = plan.level[l];
@@ -1632,7 +1636,7 @@ adasum_status_t adasum_profile_enable(int32_t max_launches)
         return fail(ADASUM_ERR_ARG, "max_launches must be positive");
     std::lock_guard<std::mutex> lock(g_profiler_mutex);
     g_profiler.enabled = false;
-    const size_t want = (size_t)max_launches * 2;    // room for the call-opening events too
+    const size_t want = (size_t)max_launches * 3;    // room for the two call-opening events of every reduce too
     while (g_profiler.events.size() < want) {
         cudaEvent_t ev;
         cudaError_t err = cudaEventCreate(&ev);
