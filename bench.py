@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the N-way Adasum combine.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4] [--impl reference]
 
 A step is one whole reduce (every level: partial Gram matrices, tree weights, weighted sum) of one
 synthetic workload.  Prints ONE JSON line.  `value` is input GB/s (N_workers * elements * bytes
@@ -37,10 +37,16 @@ NOMINAL_HBM_GBS = 8000.0
 # {(workload, kernel, level): bytes}.  Reported only while the kernel source is unchanged.
 NCU_TRAFFIC = {
     "fingerprint": "c99f9f3e55777864",
-    "bytes": {
-        "c2/gram_partial/0": 822090496,      # profiles/gram_partial_mma_f32_r8_c2.txt
-        "c2/weighted_sum/0": 874237696,      # profiles/weighted_sum_f32_r8_c2.txt
-        "c1/fused_small/0": 8040448,         # profiles/fused_small_f32_r2_c1.txt
+    # "<workload>/<kernel>/<level>": DRAM bytes of the captured launch and the algorithmic bytes of that
+    # same launch (captures of the larger configurations are taken on a smaller case of the same kernel
+    # and scaled by algorithmic bytes)
+    "captures": {
+        "c2/gram_partial/0": {"dram_bytes": 822090496, "algorithmic_bytes": 817825024,
+                              "profile": "profiles/gram_partial_mma_f32_r8_c2.txt"},
+        "c2/weighted_sum/0": {"dram_bytes": 874237696, "algorithmic_bytes": 920053152,
+                              "profile": "profiles/weighted_sum_f32_r8_c2.txt"},
+        "c1/fused_small/0": {"dram_bytes": 8040448, "algorithmic_bytes": 12000000,
+                             "profile": "profiles/fused_small_f32_r2_c1.txt"},
     },
 }
 
@@ -49,9 +55,11 @@ def kernel_source_fingerprint() -> str:
     import hashlib
 
     h = hashlib.sha256()
-    for name in ("adasum_kernels.cuh", "adasum_f64.cuh", "adasum_api.cu"):
-        with open(os.path.join(ROOT, "paper_2006_02924_b200", "csrc", name), "rb") as fh:
-            h.update(fh.read())
+    csrc = os.path.join(ROOT, "paper_2006_02924_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        if name.endswith((".cu", ".cuh", ".h")):
+            with open(os.path.join(csrc, name), "rb") as fh:
+                h.update(fh.read())
     return h.hexdigest()[:16]
 
 
@@ -144,15 +152,17 @@ class ClockSampler:
 
 def algorithmic_bytes(record, plan_levels, total_elems, in_bytes):
     """Bytes one launch must move: its operands once, plus its output for the weighted sum."""
-    level = plan_levels[record["level"]]
+    level = plan_levels[record["level"]] if record["level"] < len(plan_levels) else None
+    if record["kernel"] == "short_tensors" or level is None:
+        return 0                                # a few hundred elements per worker
     elem_bytes = in_bytes if record["level"] == 0 else 4
     read = level["operands"] * total_elems * elem_bytes
     if record["kernel"] == "gram_partial":
         return read
     if record["kernel"] == "weighted_sum":
         return read + level["groups"] * total_elems * 4
-    if record["kernel"] == "fused_small":      # both passes in one launch: HBM sees the operands once
-        return read + total_elems * 4
+    if record["kernel"] in ("fused_small", "fused_l2"):   # both passes in one launch: HBM sees the operands once
+        return read + level["groups"] * total_elems * 4
     if record["kernel"] == "wsum_gram":        # pass 2 of this level and pass 1 of the next from the same registers
         return read + level["groups"] * total_elems * 4
     if record["kernel"] == "convert":
@@ -173,21 +183,40 @@ def plan_levels_of(lib, wl, flags):
 L2_FLUSH_BYTES = 512 * 1024 * 1024      # four times the 126 MB L2
 
 
-def time_reduce(lib, wl, steps, warmup, flags, world=1, sampler=None, flush=True):
+class Reducer:
+    """One workload on this rank with its output and workspace, and the call that reduces it:
+    adasum_reduce, or (several GPUs, every rank holding a slice of every tensor) the element-sharded
+    reduce whose Gram sums are all-reduced over NCCL between the two passes of every level."""
+
+    def __init__(self, lib, wl, flags, sharded_group=None, sharded=False):
+        self.lib, self.wl, self.flags, self.sharded, self.group = lib, wl, flags, sharded, sharded_group
+        dev = wl.grads[0].device
+        self.out = torch.empty(wl.total_elems, dtype=torch.float32, device=dev)
+        need = lib.adasum_workspace_bytes(wl.total_elems, wl.num_tensors, wl.n_workers, wl.spec.dtype, flags)
+        self.ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+        self.stream = torch.cuda.current_stream()
+
+    def __call__(self, grads=None):
+        grads = self.wl.grads if grads is None else grads
+        if self.sharded:
+            self.lib.adasum_reduce_sharded(grads, self.wl.offsets, group=self.group, out=self.out, workspace=self.ws,
+                                           flags=self.flags, stream=self.stream)
+        else:
+            self.lib.adasum_reduce(grads, self.wl.offsets, out=self.out, workspace=self.ws, flags=self.flags,
+                                   stream=self.stream)
+
+
+def time_steps(call, steps, warmup, world=1, sampler=None, flush=True, device="cuda"):
     """W warm-up steps, then K timed steps bracketed by barrier + synchronize.  Every step is timed
     with its own pair of CUDA events on the launching stream; between steps a buffer four times the
     size of L2 is overwritten (outside the events), so no step finds its inputs cached by the
     previous one.  Returns ms per step (local): the mean of the K event intervals."""
     import torch.distributed as dist
 
-    dev = wl.grads[0].device
-    out = torch.empty(wl.total_elems, dtype=torch.float32, device=dev)
-    need = lib.adasum_workspace_bytes(wl.total_elems, wl.num_tensors, wl.n_workers, wl.spec.dtype, flags)
-    ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
-    scrub = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev) if flush else None
+    scrub = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device) if flush else None
     stream = torch.cuda.current_stream()
     for _ in range(warmup):
-        lib.adasum_reduce(wl.grads, wl.offsets, out=out, workspace=ws, flags=flags, stream=stream)
+        call()
     starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
     stops = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
     if world > 1:
@@ -199,15 +228,14 @@ def time_reduce(lib, wl, steps, warmup, flags, world=1, sampler=None, flush=True
             if scrub is not None:
                 scrub.zero_()
             starts[i].record(stream)
-            lib.adasum_reduce(wl.grads, wl.offsets, out=out, workspace=ws, flags=flags, stream=stream)
+            call()
             stops[i].record(stream)
         if sampler is not None:
             sampler.sample_once()
         torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
-    ms = sum(a.elapsed_time(b) for a, b in zip(starts, stops)) / steps
-    return ms, out, ws
+    return sum(a.elapsed_time(b) for a, b in zip(starts, stops)) / steps
 
 
 def time_variants(lib, wl, steps, warmup, flags):
@@ -217,7 +245,6 @@ def time_variants(lib, wl, steps, warmup, flags):
     dt = wl.grads[0].dtype
     need = lib.adasum_workspace_bytes(wl.total_elems, wl.num_tensors, wl.n_workers, wl.spec.dtype, flags)
     ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
-    scrub = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
     gen = torch.Generator(device=dev)
     gen.manual_seed(workloads.BASE_SEED + 99)
@@ -251,18 +278,7 @@ def time_variants(lib, wl, steps, warmup, flags):
                                                       stream=stream), moved))
     results = []
     for name, call, two_read_bytes in cases:
-        for _ in range(warmup):
-            call()
-        starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
-        stops = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
-        torch.cuda.synchronize()
-        for i in range(steps):
-            scrub.zero_()
-            starts[i].record(stream)
-            call()
-            stops[i].record(stream)
-        torch.cuda.synchronize()
-        ms = sum(a.elapsed_time(c) for a, c in zip(starts, stops)) / steps
+        ms = time_steps(call, steps, warmup, device=dev)
         in_bytes = wl.input_bytes * (2 if name.startswith("fp64") else 1)
         results.append({"variant": name, "ms_per_reduce": ms, "input_gbs": in_bytes / (ms * 1e-3) / 1e9,
                         "two_read_bytes": two_read_bytes,
@@ -278,23 +294,22 @@ class _Null:
         return False
 
 
-def kernel_breakdown(lib, wl, steps, flags, out, ws):
+def kernel_breakdown(lib, reducer, steps):
     """The same K steps again with an event after every launch; per (kernel, level): launches,
-    mean ms, total ms."""
-    info, levels = plan_levels_of(lib, wl, flags)
-    stream = torch.cuda.current_stream()
-    lib.adasum_profile_enable(steps * max(info["launches"], 1) + 8)
+    mean ms, total ms.  Returns (rows sorted by total time, instrumented ms per step, plan info,
+    plan levels, launches of this library's kernels per step)."""
+    wl = reducer.wl
+    info, levels = plan_levels_of(lib, wl, reducer.flags)
+    capacity = steps * (max(info["launches"], 1) + 4 * len(levels) + 4) + 8
+    lib.adasum_profile_enable(capacity)
     torch.cuda.synchronize()
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    scrub = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=out.device)
-    t0.record(stream)
+    scrub = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=reducer.out.device)
     for _ in range(steps):
         scrub.zero_()
-        lib.adasum_reduce(wl.grads, wl.offsets, out=out, workspace=ws, flags=flags, stream=stream)
-    t1.record(stream)
+        reducer()
     torch.cuda.synchronize()
     del scrub
-    records = lib.adasum_profile_collect(steps * max(info["launches"], 1) + 8)
+    records = lib.adasum_profile_collect(capacity)
     groups = {}
     for r in records:
         key = (r["kernel"], r["level"])
@@ -310,26 +325,30 @@ def kernel_breakdown(lib, wl, steps, flags, out, ws):
         g["gbs"] = g["bytes_per_launch"] / (g["mean_ms"] * 1e-3) / 1e9 if g["mean_ms"] > 0 else 0.0
         rows.append(g)
     rows.sort(key=lambda g: -g["total_ms"])
-    return rows, sum(g["total_ms"] for g in rows) / steps, info, levels
+    return rows, sum(g["total_ms"] for g in rows) / steps, info, levels, len(records) / steps
 
 
-def time_e2e(lib, wl, steps, flags, out, ws):
-    """Inputs start in pinned host memory every step and the result is read back to the host."""
-    dev = wl.grads[0].device
+def time_e2e(reducer, steps, world=1):
+    """Inputs start in pinned host memory every step and the result is read back to the host: per
+    step one host-to-device copy per worker buffer (into the buffers the reduce reads), the reduce,
+    one device-to-host copy of the result.  Returns (ms per step, H2D bytes, D2H bytes, check)."""
+    import torch.distributed as dist
+
+    wl = reducer.wl
     host_in = [torch.empty(g.shape, dtype=g.dtype, pin_memory=True).copy_(g) for g in wl.grads]
     host_out = torch.empty(wl.total_elems, dtype=torch.float32, pin_memory=True)
-    staging = [torch.empty_like(g) for g in wl.grads]
     stream = torch.cuda.current_stream()
 
     def step():
-        for d, h in zip(staging, host_in):
+        for d, h in zip(wl.grads, host_in):
             d.copy_(h, non_blocking=True)
-        lib.adasum_reduce(staging, wl.offsets, out=out, workspace=ws, flags=flags, stream=stream)
-        host_out.copy_(out, non_blocking=True)
+        reducer()
+        host_out.copy_(reducer.out, non_blocking=True)
 
-    for _ in range(2):
-        step()
+    step()
     torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     wall0 = time.perf_counter()
     t0.record(stream)
@@ -339,22 +358,28 @@ def time_e2e(lib, wl, steps, flags, out, ws):
     torch.cuda.synchronize()
     wall = (time.perf_counter() - wall0) * 1e3 / steps
     ms = max(t0.elapsed_time(t1) / steps, wall)
-    del dev
-    return ms, wl.input_bytes, wl.total_elems * 4, float(host_out[:8].abs().sum())
+    check = float(host_out[:8].abs().sum())
+    del host_in
+    return ms, wl.input_bytes, wl.total_elems * 4, check
 
 
 # ---- the CPU oracle arm ------------------------------------------------------------------------------
 
-def oracle_sample(wl_cpu, budget_elem_ops: float):
-    """A prefix-free sample of whole tensors (largest first until the budget is used) whose
-    reduction costs about budget_elem_ops = 2 (N-1) * elements."""
+def oracle_sample(wl_cpu, budget_elem_ops: float, threads: int = 1):
+    """A sample of whole tensors (largest first until the budget is used) whose reduction costs
+    about budget_elem_ops = 2 (N-1) * elements.  The oracle's threads each take whole tensors, so
+    with `threads` > 1 tensors larger than a thread's share of the budget are passed over (as long
+    as smaller ones exist): the sample then keeps every core busy."""
     sizes = np.diff(wl_cpu.offsets)
     per_elem = 2.0 * max(wl_cpu.n_workers - 1, 1)
     order = np.argsort(-sizes, kind="stable")
+    share = budget_elem_ops / max(threads, 1)
+    if threads > 1 and np.any((sizes > 0) & (per_elem * sizes <= share)):
+        order = [t for t in order if per_elem * float(sizes[t]) <= share]
     chosen, used = [], 0.0
     for t in order:
         cost = per_elem * float(sizes[t])
-        if chosen and used + cost > budget_elem_ops:
+        if sizes[t] == 0 or (chosen and used + cost > budget_elem_ops):
             continue
         chosen.append(int(t))
         used += cost
@@ -408,14 +433,17 @@ def reference_arm(args):
     wl = workloads.generate(spec, device="cpu", tensor_sizes=[sizes[t] for t in keep])
     all_tensors = list(range(wl.num_tensors))
     # calibrate on a small sample, then size each step so that the whole run stays near two minutes
-    probe = oracle_sample(wl, 2e8)
+    from oracle import adasum_oracle as oracle
+
+    cores = oracle.threads_used(0)
+    probe = oracle_sample(wl, 4e8, cores)
     dt, nbytes, threads = run_oracle(wl, probe)
     per_elem = 2.0 * max(spec.n_workers - 1, 1)
     probe_ops = per_elem * sum(int(wl.offsets[t + 1] - wl.offsets[t]) for t in probe)
     rate = probe_ops / max(dt, 1e-6)
     budget = rate * min(120.0 / (steps + warmup), 20.0)
     full_ops = per_elem * wl.total_elems
-    tensors = all_tensors if budget >= full_ops else oracle_sample(wl, budget)
+    tensors = all_tensors if budget >= full_ops else oracle_sample(wl, budget, cores)
     times = []
     for i in range(steps + warmup):
         dt, nbytes, threads = run_oracle(wl, tensors)
@@ -467,22 +495,122 @@ def resolve_spec(name, n_workers=None, tensor_list=None):
     return spec
 
 
-def measure_workload(lib, name, steps, warmup, flags, replica, world, sampler=None):
-    wl = workloads.generate(name, device="cuda", replica=replica)
-    ms, out, ws = time_reduce(lib, wl, steps, warmup, flags, world=world, sampler=sampler)
-    return wl, ms, out, ws
+def sharded_local_sizes(spec, world: int, rank: int):
+    """Tensor sizes of rank `rank`'s slice when every tensor of the configuration is cut into
+    `world` element ranges (workloads.element_shards); a tensor may be empty on the last ranks."""
+    offsets = workloads.offsets_from_sizes(spec.tensor_sizes())
+    local_offsets, _ = workloads.element_shards(offsets, world)[rank]
+    return [int(v) for v in np.diff(local_offsets)]
 
 
-def summarise(wl, ms, peak):
-    p, b, n = wl.total_elems, workloads.DTYPE_BYTES[wl.spec.dtype], wl.n_workers
-    one_read = n * p * b + 4 * p
+def allreduce_bytes_per_level(num_tensors: int, levels):
+    """Bytes of fp64 Gram sums every rank contributes to the all-reduce of each level."""
+    return [num_tensors * lv["groups"] * (lv["radix"] * (lv["radix"] + 1) // 2) * 8 for lv in levels]
+
+
+def whole_reduce_summary(n_workers, total_elems, elem_bytes, ms, peak):
+    """Both readings of "fraction of the HBM roofline" for the whole reduce: the one-read formula
+    (N P b read + 4 P written, at peak), which a two-phase method cannot reach for tensors that do
+    not fit on chip, and the two-read bound (dot products complete before any output)."""
+    one_read = n_workers * total_elems * elem_bytes + 4 * total_elems
+    two_read = 2 * n_workers * total_elems * elem_bytes + 4 * total_elems
+    per_s = 1.0 / (ms * 1e-3) / 1e9
     return {
         "ms_per_reduce": ms,
-        "input_gbs": wl.input_bytes / (ms * 1e-3) / 1e9,
-        "one_read_roofline_frac_measured_peak": one_read / (ms * 1e-3) / 1e9 / peak,
-        "one_read_roofline_frac_nominal_8TBs": one_read / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
-        "two_read_roofline_frac_measured_peak": (2 * n * p * b + 4 * p) / (ms * 1e-3) / 1e9 / peak,
+        "input_gbs": n_workers * total_elems * elem_bytes * per_s,
+        "one_read_bytes": one_read, "two_read_bytes": two_read,
+        "one_read_roofline_frac_measured_peak": one_read * per_s / peak,
+        "one_read_roofline_frac_nominal_8TBs": one_read * per_s / NOMINAL_HBM_GBS,
+        "two_read_roofline_frac_measured_peak": two_read * per_s / peak,
+        "two_read_roofline_frac_nominal_8TBs": two_read * per_s / NOMINAL_HBM_GBS,
     }
+
+
+def traffic_of(workload_key: str, row) -> dict:
+    """ncu DRAM bytes per launch for this kernel, scaled from the captured case by algorithmic
+    bytes (traffic grows in proportion: every operand byte crosses HBM once per pass); None once
+    the kernel sources have changed since the counters were taken."""
+    if NCU_TRAFFIC["fingerprint"] != kernel_source_fingerprint():
+        return None
+    entry = NCU_TRAFFIC["captures"].get(f"{workload_key}/{row['kernel']}/{row['level']}")
+    if entry is None or entry["algorithmic_bytes"] <= 0:
+        return None
+    return int(round(entry["dram_bytes"] * row["bytes_per_launch"] / entry["algorithmic_bytes"]))
+
+
+def cpu_baseline_of(wl, name: str, seconds: float):
+    """The fp64 oracle, as it stands, on a bounded sample of the workload (whole tensors), sized from
+    a short calibration run so that it takes about `seconds` on this host."""
+    from oracle import adasum_oracle as oracle
+
+    threads = oracle.threads_used(0)
+    per_elem = 2.0 * max(wl.n_workers - 1, 1)
+    full_ops = per_elem * wl.total_elems
+    probe = oracle_sample(wl, min(full_ops, 4e8), threads)
+    dt, _, _ = run_oracle(wl, probe)
+    probe_ops = per_elem * sum(int(wl.offsets[t + 1] - wl.offsets[t]) for t in probe)
+    budget = probe_ops / max(dt, 1e-6) * seconds
+    # at most 16 GB of inputs are staged on the host
+    budget = min(budget, per_elem * 16e9 / (wl.n_workers * workloads.DTYPE_BYTES[wl.spec.dtype]))
+    tensors = list(range(wl.num_tensors)) if budget >= full_ops else oracle_sample(wl, budget, threads)
+    dt, nbytes, used = run_oracle(wl, tensors)
+    elems = sum(int(wl.offsets[t + 1] - wl.offsets[t]) for t in tensors)
+    return {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": used, "kind": "oracle",
+            "sample": f"{len(tensors)} of {wl.num_tensors} tensors of {name}, {elems} elements x "
+                      f"{wl.n_workers} workers ({nbytes / 1e9:.2f} GB of inputs), {dt:.2f} s"}
+
+
+def measure_config(lib, name, spec, steps, warmup, flags, peak, peak_kind, *, world=1, rank=0, mode="single",
+                   sampler=None, e2e_steps=3, cpu_seconds=10.0, tensor_sizes=None, traffic_key=None):
+    """One configuration end to end: the timed steps, the per-launch breakdown with the roofline of
+    the dominant kernel, the end-to-end leg and (one GPU only) the CPU oracle beside it."""
+    sharded = mode == "sharded" and world > 1
+    wl = workloads.generate(spec, device="cuda", tensor_sizes=tensor_sizes, replica=rank)
+    reducer = Reducer(lib, wl, flags, sharded=sharded)
+    ms_local = time_steps(reducer, steps, warmup, world=world, sampler=sampler)
+    eb = workloads.DTYPE_BYTES[spec.dtype]
+    if sharded:          # strong scaling: the job is the whole configuration, the time the slowest rank's
+        job_elems = sum(spec.tensor_sizes())
+        ms, _ = aggregate_over_ranks(ms_local, 0.0, world, "cuda")
+        job_bytes = float(spec.n_workers * job_elems * eb)
+    else:
+        job_elems = wl.total_elems * world
+        ms, job_bytes = aggregate_over_ranks(ms_local, float(wl.input_bytes), world, "cuda")
+    rows, ms_instrumented, info, levels, launches_per_step = kernel_breakdown(lib, reducer, steps)
+    top = rows[0]
+    total_rows_ms = sum(r["total_ms"] for r in rows)
+    roofline = {
+        "bound": "hbm", "kernel": f"{top['kernel']}<radix {top['radix']}> level {top['level']}",
+        "achieved": top["gbs"], "peak": peak, "unit": "GB/s", "frac": top["gbs"] / peak,
+        "peak_kind": f"of {peak_kind}", "traffic": traffic_of(traffic_key or name, top),
+        "bytes_per_launch": top["bytes_per_launch"], "mean_launch_ms": top["mean_ms"],
+        "share_of_step": top["total_ms"] / total_rows_ms if total_rows_ms > 0 else None,
+        "timing": "CUDA event after every launch, same K steps (L2 flushed between them) repeated right "
+                  "after the timed region",
+        "instrumented_ms_per_step": ms_instrumented,
+        "kernels": [dict({k: r[k] for k in ("kernel", "level", "radix", "launches", "mean_ms", "gbs")},
+                         frac=r["gbs"] / peak, traffic=traffic_of(traffic_key or name, r)) for r in rows],
+        "whole_reduce": whole_reduce_summary(spec.n_workers, job_elems if sharded else wl.total_elems, eb,
+                                             ms if sharded else ms_local, peak),
+    }
+    e2e_ms_local, h2d, d2h, _ = time_e2e(reducer, e2e_steps, world=world)
+    e2e_ms, _ = aggregate_over_ranks(e2e_ms_local, 0.0, world, "cuda")
+    e2e = {"value": job_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps,
+           "bytes_are": "per rank" if world > 1 else "whole job"}
+    cpu_baseline = None
+    if rank == 0 and world == 1 and cpu_seconds > 0:
+        cpu_baseline = cpu_baseline_of(wl, name, cpu_seconds)
+    entry = {
+        "workload": name, "n_workers": spec.n_workers, "dtype": spec.dtype, "tensor_list": spec.tensor_list,
+        "num_tensors": wl.num_tensors, "elements_per_worker": job_elems if sharded else wl.total_elems,
+        "steps": steps, "radices": info["radices"], "ms_per_reduce": ms,
+        "input_gbs": job_bytes / (ms * 1e-3) / 1e9, "launches_per_step": launches_per_step,
+        "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu_baseline,
+    }
+    if sharded:
+        entry["allreduce_bytes_per_level"] = allreduce_bytes_per_level(wl.num_tensors, levels)
+    return entry, wl, reducer
 
 
 def cuda_arm(args):
@@ -506,90 +634,66 @@ def cuda_arm(args):
     peak, peak_kind = measured_peak()
     sampler = ClockSampler(local_rank)
     steps, warmup = max(args.steps, 1), max(args.warmup, 3)
+    mode = "single" if world == 1 else args.multi
+    single = rank == 0 and world == 1
 
     main_spec = resolve_spec(args.workload, args.n_workers, args.tensor_list)
-    wl, ms_local, out, ws = measure_workload(lib, main_spec, steps, warmup, flags, rank, world, sampler)
-    ms, job_bytes = aggregate_over_ranks(ms_local, float(wl.input_bytes), world, "cuda")
-    value = job_bytes / (ms * 1e-3) / 1e9
-
-    rows, ms_instrumented, info, levels = kernel_breakdown(lib, wl, steps, flags, out, ws)
-    top = rows[0]
-    traffic = None
-    if NCU_TRAFFIC["fingerprint"] == kernel_source_fingerprint():
-        traffic = NCU_TRAFFIC["bytes"].get(f"{args.workload}/{top['kernel']}/{top['level']}")
-    roofline = {
-        "bound": "hbm", "kernel": f"{top['kernel']}<radix {top['radix']}> level {top['level']}",
-        "achieved": top["gbs"], "peak": peak, "unit": "GB/s", "frac": top["gbs"] / peak,
-        "peak_kind": f"of {peak_kind}", "traffic": traffic,
-        "bytes_per_launch": top["bytes_per_launch"], "mean_launch_ms": top["mean_ms"],
-        "share_of_step": top["total_ms"] / sum(r["total_ms"] for r in rows),
-        "timing": "CUDA event after every launch, same K steps (L2 flushed between them) repeated right "
-                  "after the timed region",
-        "instrumented_ms_per_step": ms_instrumented,
-        "kernels": [{k: r[k] for k in ("kernel", "level", "radix", "launches", "mean_ms", "gbs")} for r in rows],
-    }
-
-    e2e_steps = min(steps, 20)
-    e2e_ms_local, h2d, d2h, _ = time_e2e(lib, wl, e2e_steps, flags, out, ws)
-    e2e_ms, _ = aggregate_over_ranks(e2e_ms_local, float(wl.input_bytes), world, "cuda")
-    e2e = {"value": job_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
-           "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps}
-
-    cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        budget = 4e9
-        tensors = oracle_sample(wl, budget)
-        if 2.0 * (wl.n_workers - 1) * wl.total_elems <= budget:
-            tensors = list(range(wl.num_tensors))
-        dt, nbytes, threads = run_oracle(wl, tensors)
-        cpu_baseline = {
-            "value": nbytes / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
-            "sample": f"{len(tensors)} of {wl.num_tensors} tensors of {args.workload}, "
-                      f"{sum(int(wl.offsets[t + 1] - wl.offsets[t]) for t in tensors)} elements x "
-                      f"{wl.n_workers} workers, {dt:.2f} s",
-        }
-
-    summary = summarise(wl, ms, peak)
-    spec = wl.spec
-    n_workers, total_elems, num_tensors = wl.n_workers, wl.total_elems, wl.num_tensors
-    del out, ws
+    sizes = sharded_local_sizes(main_spec, world, rank) if mode == "sharded" else None
+    overridden = bool(args.n_workers or args.tensor_list)
+    traffic_key = args.workload if not overridden else \
+        f"{args.workload}:{main_spec.tensor_list}:n{main_spec.n_workers}"
+    head, wl, reducer = measure_config(
+        lib, args.workload, main_spec, steps, warmup, flags, peak, peak_kind, world=world, rank=rank, mode=mode,
+        sampler=sampler, e2e_steps=args.e2e_steps, cpu_seconds=0.0 if args.no_cpu_baseline else args.cpu_seconds,
+        tensor_sizes=sizes, traffic_key=traffic_key)
     variants = []
-    if rank == 0 and world == 1 and not args.no_other_workloads:
-        variants = time_variants(lib, wl, max(3, min(steps, 200)), 3, flags)
+    if single and not args.no_other_workloads:
+        del reducer
+        variants = time_variants(lib, wl, max(3, min(steps, 50)), 3, flags)
+    reducer = None
     del wl
     torch.cuda.empty_cache()
 
     others = []
-    if rank == 0 and world == 1 and not args.no_other_workloads:
+    if single and not args.no_other_workloads:
         for name in ("c1", "c2", "c3", "c4", "c5"):
-            if name == args.workload and not (args.n_workers or args.tensor_list):
+            if name == args.workload and not overridden:
                 continue
-            k = max(3, min(steps, 10 if name in ("c3", "c4", "c5") else 200))
-            owl, oms, oout, ows = measure_workload(lib, name, k, 3, flags, 0, 1)
-            orows, _, oinfo, _ = kernel_breakdown(lib, owl, k, flags, oout, ows)
-            entry = {"workload": name, "n_workers": owl.n_workers, "dtype": owl.spec.dtype,
-                     "steps": k, "radices": oinfo["radices"], **summarise(owl, oms, peak),
-                     "kernels": [{kk: r[kk] for kk in ("kernel", "level", "radix", "mean_ms", "gbs")} for r in orows]}
+            k = max(3, min(steps, 20 if name in ("c3", "c4", "c5") else 200))
+            entry, owl, ored = measure_config(lib, name, workloads.SPECS[name], k, 3, flags, peak, peak_kind,
+                                              e2e_steps=args.e2e_steps,
+                                              cpu_seconds=0.0 if args.no_cpu_baseline else min(args.cpu_seconds, 6.0))
             others.append(entry)
-            del owl, oout, ows
+            del owl, ored
             torch.cuda.empty_cache()
 
     if rank == 0:
+        spec = main_spec
+        scaling = "strong" if mode == "sharded" else "weak"
+        multi = {"single": "one GPU",
+                 "sharded": "every rank holds one element range of every tensor; per level the fp64 Gram sums are "
+                            "all-reduced over NCCL between the two passes (no other exchange)",
+                 "replicas": "independent replicas of the workload, one per GPU, no collective"}[mode]
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
-            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": spec.dtype, "data": "synthetic",
-            "config": {"workload": args.workload, "n_workers": n_workers, "tensor_list": spec.tensor_list,
-                       "num_tensors": num_tensors, "elements_per_worker": total_elems,
-                       "radices": info["radices"], "l2": "flushed between steps (512 MB overwritten outside the per-step events)" +
-                       ("; inputs also larger than L2" if n_workers * total_elems *
-                        workloads.DTYPE_BYTES[spec.dtype] > 2 * 126e6 else ""),
-                       "timing": "mean of K per-step CUDA-event intervals on the launching stream",
-                       "multi_gpu": "independent replicas of the workload, one per GPU, no collective"},
-            "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": steps * info["launches"],
-            "roofline": roofline, "cpu_baseline": cpu_baseline,
-            "whole_reduce": summary, "variants": variants, "other_workloads": others,
+            "metric": METRIC, "value": head["input_gbs"], "unit": UNIT, "n_gpus": world, "steps": steps,
+            "warmup": warmup, "ms_per_step": head["ms_per_reduce"], "higher_is_better": True, "scaling": scaling,
+            "vs_baseline": None, "dtype": spec.dtype, "data": "synthetic",
+            "config": {"workload": args.workload, "n_workers": spec.n_workers, "tensor_list": spec.tensor_list,
+                       "num_tensors": head["num_tensors"], "elements_per_worker": head["elements_per_worker"],
+                       "radices": head["radices"],
+                       "l2": "flushed between steps (512 MB overwritten outside the per-step events); inputs are also "
+                             "larger than L2" if spec.n_workers * head["elements_per_worker"] *
+                             workloads.DTYPE_BYTES[spec.dtype] > 2 * 126e6 else
+                             "flushed between steps (512 MB overwritten outside the per-step events)",
+                       "timing": "mean of K per-step CUDA-event intervals on the launching stream, max over ranks",
+                       "multi_gpu": multi},
+            "clocks": sampler.summary(), "e2e": head["e2e"],
+            "gpu_launches": int(round(steps * head["launches_per_step"])),
+            "roofline": head["roofline"], "cpu_baseline": head["cpu_baseline"],
+            "variants": variants, "other_workloads": others,
         }
+        if "allreduce_bytes_per_level" in head:
+            line["config"]["allreduce_bytes_per_level"] = head["allreduce_bytes_per_level"]
         print(json.dumps(line))
     if world > 1:
         dist.barrier()
@@ -599,10 +703,16 @@ def cuda_arm(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
-    ap.add_argument("--workload", default="c2", choices=sorted(workloads.SPECS))
+    ap.add_argument("--workload", default="c4", choices=sorted(workloads.SPECS))
+    ap.add_argument("--multi", default="sharded", choices=["sharded", "replicas"],
+                    help="with several GPUs: every rank holds a slice of every tensor and the Gram sums are "
+                         "all-reduced (sharded), or every rank reduces an independent copy of the workload (replicas)")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0,
+                    help="about how long the CPU oracle runs on its sample of the headline workload")
     ap.add_argument("--n-workers", type=int, default=0, help="override the configuration's worker count")
     ap.add_argument("--tensor-list", default="", choices=["", "single", "resnet50", "bert_large"],
                     help="override the configuration's tensor list")

@@ -16,6 +16,12 @@
  * in fp32 inside blocks of at most a few thousand elements per thread block and in fp64 across
  * blocks (Section 4.4.1 asks for accumulation wider than the gradient type); all coefficient
  * arithmetic is fp64 on the device; intermediates between levels and the output are fp32.
+ * Tensors of at most 64 elements are the exception: their result can be a small difference of
+ * large terms (a one-element tensor whose workers disagree in sign), so adasum_reduce,
+ * adasum_reduce_ex, adasum_reduce_delta and adasum_pair apply the operator to them literally, pair
+ * by pair and level by level, in fp64 from the loads to the one rounding of the stored result (one
+ * more small kernel launch when a buffer has such tensors; the sharded calls, whose tensors are
+ * spread over several GPUs, keep to the general path).
  *
  * Conventions for every entry point:
  *   - plain C, no exceptions; every call returns a status, and on any status other than
@@ -28,10 +34,14 @@
  *     default stream) and never synchronise it;
  *   - the library allocates nothing per call.  The first call with a tensor-offset table it
  *     has not seen on the current device builds a small segment table on the device
- *     (cudaMalloc plus a blocking copy); later calls with the same table reuse it.  Up to 64
- *     tables are kept; beyond that the oldest is freed.  adasum_shutdown() frees them all.
- *     That first call must therefore not be made while the stream is being captured into a
- *     CUDA graph;
+ *     (cudaMalloc plus a blocking copy); later calls with the same table reuse it.  The cache
+ *     keeps the most recently used tables, up to 256 of them and 256 MB of device memory; a
+ *     call that needs a new table beyond that drops the least recently used ones, and freeing
+ *     them (cudaFree) waits for all work already submitted to the device.  A caller whose
+ *     tensor grouping changes on every call therefore pays an allocation, a blocking copy and,
+ *     once the cache is full, a device-wide wait per call; keep the set of offset tables small
+ *     where that matters.  adasum_shutdown() frees them all.  A call that builds a table must
+ *     not be made while the stream is being captured into a CUDA graph;
  *   - results are deterministic: the same inputs, sizes and flags give the same bits.
  */
 #ifndef ADASUM_H_
@@ -70,8 +80,10 @@ typedef enum {
     ADASUM_ERR_DTYPE = 4,       /* unknown dtype */
     ADASUM_ERR_WORKSPACE = 5,   /* workspace NULL or smaller than adasum_workspace_bytes() */
     ADASUM_ERR_CUDA = 6,        /* a CUDA runtime call or a launch failed (see adasum_last_error) */
-    ADASUM_ERR_TIMEOUT = 7      /* reserved for bounded device-side waits; unused by the
-                                   current kernels, which never wait on one another */
+    ADASUM_ERR_TIMEOUT = 7      /* a bounded device-side wait ran out (the waits between the copying
+                                   warps and the tensor core inside the tcgen05 Gram kernel, and
+                                   the flag waits inside the single-launch kernels); reported by
+                                   adasum_device_status, never by the call that launched */
 } adasum_status_t;
 
 /*
@@ -141,7 +153,8 @@ size_t adasum_workspace_bytes(int64_t total_elems, int32_t num_tensors, int32_t 
 /*
  * How a reduce with these sizes will run: writes the radix of each level into radices[]
  * (room for ADASUM_MAX_LEVELS entries), the number of levels into *num_levels and the number
- * of kernel launches on a B200 into *num_launches (each may be NULL).  Host-only.  A one-level
+ * of kernel launches on a B200 into *num_launches (each may be NULL; a buffer that has tensors of
+ * at most 64 elements takes one launch more, which this call cannot know).  Host-only.  A one-level
  * reduce of at most 8 workers whose operands total at most 96 MB is a single cooperative launch that
  * reads the operands from HBM once (the second pass finds them in the L2) unless flag bit 16 or 17
  * is set.
@@ -277,7 +290,7 @@ adasum_status_t adasum_pair(const void* a, const void* b, const int64_t* tensor_
  * allocator at start-up, a real-time loop that forbids driver allocations after initialisation.
  * adasum_pair needs a workspace from its caller and builds a cached segment table with cudaMalloc
  * on first use; this entry point needs neither.  Its scratch (segment table, per-segment partial
- * sums, per-tensor coefficients; about 0.5 MB) is a fixed array inside the library's device
+ * sums, per-tensor coefficients, the list of short tensors; about 0.6 MB) is a fixed array inside the library's device
  * image, so every GPU that loads the library carries it until the process exits.
  *
  *   a, b, tensor_offsets, num_tensors, dtype, out, stream   as for adasum_pair
@@ -287,9 +300,12 @@ adasum_status_t adasum_pair(const void* a, const void* b, const int64_t* tensor_
  * equals adasum_pair's with default flags.
  *
  * The call performs no cudaMalloc / cudaFree and uses no allocating library routine; it enqueues
- * two small host-to-device copies (the segment table of this call) and three kernels on `stream`.
- * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
- * that device current); make that first call before any stream capture begins.
+ * up to three small host-to-device copies (the segment table of this call, up to about 0.3 MB, staged
+ * from ordinary host memory, so the call can briefly wait for the copy engine) and three or four
+ * kernels on `stream`.  The first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress, with that device current); make that first call before any stream capture
+ * begins.  Because the table is copied from host memory that lives only for the duration of the
+ * call, a `stream` that is being captured is refused with ADASUM_ERR_ARG and nothing is recorded.
  *
  * All calls on a device share the one scratch array, which keeps the previous call's contents.
  * Every entry that a call reads is first rewritten by the same call, so nothing has to be
@@ -339,6 +355,7 @@ const char* adasum_last_error(void);
 #define ADASUM_KERNEL_CONVERT 3
 #define ADASUM_KERNEL_FUSED_SMALL 4   /* both passes in one cooperative launch (inputs that fit the L2) */
 #define ADASUM_KERNEL_WSUM_GRAM 5     /* second pass of `level` and first pass of level + 1 in one kernel */
+#define ADASUM_KERNEL_SHORT_TENSORS 6 /* the whole tree of the tensors of at most 64 elements, in fp64 */
 
 typedef struct {
     int32_t kernel;

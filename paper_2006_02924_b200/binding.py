@@ -322,7 +322,7 @@ class _LaunchRecord(ctypes.Structure):
 
 
 KERNEL_NAMES = {0: "gram_partial", 1: "tree_weights", 2: "weighted_sum", 3: "convert", 4: "fused_small",
-                5: "wsum_gram"}
+                5: "wsum_gram", 6: "short_tensors"}
 
 _lib.adasum_profile_enable.restype = ctypes.c_int
 _lib.adasum_profile_enable.argtypes = [ctypes.c_int32]

@@ -12,11 +12,11 @@
 #include <mutex>
 #include <vector>
 
+#include "adasum_internal.h"
 #include "adasum_kernels.cuh"
 #include "adasum_f64.cuh"
 
 namespace adasum {
-namespace {
 
 thread_local char g_error[512] = "";
 
@@ -29,12 +29,7 @@ adasum_status_t fail(adasum_status_t status, const char* fmt, ...)
     return status;
 }
 
-#define ADASUM_CUDA_CHECK(expr)                                                                  \
-    do {                                                                                         \
-        cudaError_t err__ = (expr);                                                              \
-        if (err__ != cudaSuccess)                                                                \
-            return fail(ADASUM_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(err__));            \
-    } while (0)
+namespace {
 
 // ---- optional per-launch timing ---------------------------------------------------------------
 // When enabled, an event is recorded on the caller's stream before the first launch of a reduce
@@ -57,6 +52,8 @@ struct Profiler {
 Profiler g_profiler;
 std::mutex g_profiler_mutex;
 
+}  // namespace
+
 void profile_mark(cudaStream_t stream, int kernel, int level, int radix, bool starts_call)
 {
     if (!g_profiler.enabled)
@@ -73,6 +70,8 @@ void profile_mark(cudaStream_t stream, int kernel, int level, int radix, bool st
     g_profiler.marks[g_profiler.used] = ProfileMark{kernel, level, radix, starts_call};
     ++g_profiler.used;
 }
+
+namespace {
 
 constexpr size_t kAlign = 256;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -94,17 +93,6 @@ int pow2_ceil(int x)
     while (p < x)
         p *= 2;
     return p;
-}
-
-// Which Gram kernel serves a level.
-enum GramKind {
-    GRAM_SIMPLE,      // fp32 pipes, operands in registers (radix <= 4; radix 8 and 16 on request)
-    GRAM_MMA          // tensor cores (radix >= 8)
-};
-
-GramKind gram_kind(int radix, bool simple_kernels)
-{
-    return (radix >= 32 || (radix >= 8 && !simple_kernels)) ? GRAM_MMA : GRAM_SIMPLE;
 }
 
 // Elements per segment.  One block accumulates a whole segment in fp32 (per thread: segment /
@@ -218,14 +206,26 @@ struct Layout {
     size_t partials = 0, weights = 0, weights_alt = 0, gram64 = 0, counters = 0, leaf_sums = 0, buffer[2] = {0, 0};
     size_t partials_bytes = 0, weights_bytes = 0, gram64_bytes = 0, counters_bytes = 0, leaf_sums_bytes = 0,
            buffer_bytes[2] = {0, 0};
+    // short tensors of reduces with more workers than one launch carries: per launch an fp64 vector
+    // over the short tensors' elements and the sum of its leaves' squared norms
+    size_t short_vecs = 0, short_sums = 0, short_vecs_bytes = 0, short_sums_bytes = 0;
+    int64_t short_vec_stride = 0, short_sum_stride = 0;      // doubles between two launches' arrays
     int64_t padded_elems = 0;
     size_t total = 0;
 };
 
-Layout make_layout(const LevelPlan& plan, int64_t total_elems, int32_t num_tensors)
+Layout make_layout(const LevelPlan& plan, int64_t total_elems, int32_t num_tensors, int n_workers)
 {
     Layout lay;
     lay.padded_elems = (total_elems + 63) / 64 * 64;
+    if (n_workers > kMaxOperandsPerLaunch) {
+        const int64_t launches = (n_workers + kMaxOperandsPerLaunch - 1) / kMaxOperandsPerLaunch;
+        const int64_t bound = (int64_t)num_tensors * kShortTensorElems;
+        lay.short_vec_stride = total_elems < bound ? total_elems : bound;
+        lay.short_sum_stride = num_tensors;
+        lay.short_vecs_bytes = (size_t)(launches * lay.short_vec_stride) * sizeof(double);
+        lay.short_sums_bytes = (size_t)(launches * lay.short_sum_stride) * sizeof(double);
+    }
     for (int l = 0; l < plan.num_levels; ++l) {
         const Level& lv = plan.level[l];
         const size_t p = (size_t)segment_bound(total_elems, num_tensors,
@@ -268,34 +268,54 @@ Layout make_layout(const LevelPlan& plan, int64_t total_elems, int32_t num_tenso
     off += align_up(lay.buffer_bytes[0]);
     lay.buffer[1] = off;
     off += align_up(lay.buffer_bytes[1]);
+    lay.short_vecs = off;
+    off += align_up(lay.short_vecs_bytes);
+    lay.short_sums = off;
+    off += align_up(lay.short_sums_bytes);
     lay.total = off > 0 ? off : kAlign;
     return lay;
 }
 
 // ---- cached segment tables ---------------------------------------------------------------------
+//
+// A table is shared between the cache and every call that is using it (TableRef), so dropping it
+// from the cache never frees device memory that a call still intends to launch with: the device
+// arrays go when the last reference does, and cudaFree then waits for the kernels that were
+// enqueued with them.
 
-struct SegmentTable {
-    int device = -1;
-    int seg_len = 0;
-    std::vector<int64_t> offsets;
-    Segment* d_segments = nullptr;
-    int32_t* d_seg_first = nullptr;
-    int32_t num_segments = 0;
-    int32_t max_segments_per_tensor = 0;
-    std::vector<Segment> h_segments;
-    std::vector<int32_t> h_seg_first;
-};
+using TableRef = std::shared_ptr<const SegmentTable>;
 
+// Least recently used first.  The cache is bounded both by the number of tables and by the device
+// bytes they hold.
 std::mutex g_tables_mutex;
-std::vector<std::unique_ptr<SegmentTable>> g_tables;
-constexpr size_t kMaxCachedTables = 64;
+std::vector<std::shared_ptr<SegmentTable>> g_tables;
+constexpr size_t kMaxCachedTables = 256;
+constexpr size_t kMaxCachedTableBytes = size_t(256) << 20;
+
+size_t table_device_bytes(const SegmentTable& tab)
+{
+    return sizeof(Segment) * (tab.h_segments.size() + 1) + sizeof(int32_t) * tab.h_seg_first.size() +
+           sizeof(ShortTensor) * (tab.h_short.size() + 1);
+}
 
 // Segments are listed tensor by tensor, LARGEST tensor first (ties in index order): the blocks of
 // pass 1 that run last then belong to small tensors, whose per-tensor finish (adding the partial
 // matrices, tree weights) is short, instead of leaving one SM busy with a long tensor's finish
 // while the rest of the GPU idles.  Each tensor's segments stay contiguous, in element order.
-void build_segments(const int64_t* offsets, int32_t num_tensors, int seg_len, SegmentTable* tab)
+void build_segments(const int64_t* offsets, int32_t num_tensors, int seg_len, bool skip_short, SegmentTable* tab)
 {
+    tab->skip_short = skip_short;
+    tab->h_short.clear();
+    tab->short_elems = 0;
+    if (skip_short) {
+        for (int32_t t = 0; t < num_tensors; ++t) {
+            const int64_t len = offsets[t + 1] - offsets[t];
+            if (len > 0 && len <= kShortTensorElems) {
+                tab->h_short.push_back(ShortTensor{offsets[t], (int32_t)len, t, tab->short_elems});
+                tab->short_elems += len;
+            }
+        }
+    }
     std::vector<int32_t> order((size_t)num_tensors);
     for (int32_t t = 0; t < num_tensors; ++t)
         order[t] = t;
@@ -310,6 +330,8 @@ void build_segments(const int64_t* offsets, int32_t num_tensors, int seg_len, Se
         tab->h_seg_first[2 * (size_t)t] = (int32_t)tab->h_segments.size();
         int64_t b = offsets[t];
         const int64_t e = offsets[t + 1];
+        if (skip_short && e - b <= kShortTensorElems)
+            b = e;
         while (b < e) {
             // cut on a 64-element grid of the fused buffer so that interior cuts keep 16-byte
             // alignment whatever the tensor's own start
@@ -327,201 +349,68 @@ void build_segments(const int64_t* offsets, int32_t num_tensors, int seg_len, Se
     tab->num_segments = (int32_t)tab->h_segments.size();
 }
 
-adasum_status_t get_segment_table(const int64_t* offsets, int32_t num_tensors, int seg_len,
-                                  const SegmentTable** out)
+// The table for (current device, offsets, seg_len), built and uploaded on first use.  The caller
+// keeps the returned reference until it has enqueued its last launch that reads the table.
+adasum_status_t get_segment_table(const int64_t* offsets, int32_t num_tensors, int seg_len, bool skip_short,
+                                  TableRef* out)
 {
     int device = 0;
     ADASUM_CUDA_CHECK(cudaGetDevice(&device));
+    std::vector<std::shared_ptr<SegmentTable>> dropped;      // destroyed after the lock is released
     std::lock_guard<std::mutex> lock(g_tables_mutex);
-    for (const auto& tab : g_tables) {
-        if (tab->device == device && tab->seg_len == seg_len &&
-            tab->offsets.size() == (size_t)num_tensors + 1 &&
-            std::memcmp(tab->offsets.data(), offsets, sizeof(int64_t) * tab->offsets.size()) == 0) {
-            *out = tab.get();
+    for (size_t i = 0; i < g_tables.size(); ++i) {
+        const SegmentTable& tab = *g_tables[i];
+        if (tab.device == device && tab.seg_len == seg_len && tab.skip_short == skip_short &&
+            tab.offsets.size() == (size_t)num_tensors + 1 &&
+            std::memcmp(tab.offsets.data(), offsets, sizeof(int64_t) * tab.offsets.size()) == 0) {
+            // most recently used last
+            std::rotate(g_tables.begin() + (ptrdiff_t)i, g_tables.begin() + (ptrdiff_t)i + 1, g_tables.end());
+            *out = g_tables.back();
             return ADASUM_OK;
         }
     }
-    if (g_tables.size() >= kMaxCachedTables) {
-        // Drop the oldest table.  cudaFree waits for work already submitted to the device, so
-        // kernels still reading the table finish first.
-        SegmentTable* oldest = g_tables.front().get();
-        int current = device;
-        if (oldest->device != current)
-            ADASUM_CUDA_CHECK(cudaSetDevice(oldest->device));
-        cudaError_t e1 = cudaFree(oldest->d_segments), e2 = cudaFree(oldest->d_seg_first);
-        if (oldest->device != current)
-            ADASUM_CUDA_CHECK(cudaSetDevice(current));
-        g_tables.erase(g_tables.begin());
-        if (e1 != cudaSuccess || e2 != cudaSuccess)
-            return fail(ADASUM_ERR_CUDA, "freeing an evicted segment table failed");
-    }
-    auto tab = std::make_unique<SegmentTable>();
+    auto tab = std::make_shared<SegmentTable>();
     tab->device = device;
     tab->seg_len = seg_len;
     tab->offsets.assign(offsets, offsets + num_tensors + 1);
-    build_segments(offsets, num_tensors, seg_len, tab.get());
+    build_segments(offsets, num_tensors, seg_len, skip_short, tab.get());
     const size_t seg_bytes = sizeof(Segment) * (tab->h_segments.size() + 1);
     const size_t first_bytes = sizeof(int32_t) * tab->h_seg_first.size();
-    ADASUM_CUDA_CHECK(cudaMalloc(&tab->d_segments, seg_bytes));
-    cudaError_t err = cudaMalloc(&tab->d_seg_first, first_bytes);
+    const size_t short_bytes = sizeof(ShortTensor) * (tab->h_short.size() + 1);
+    // Make room: least recently used tables leave the cache.  One that a call in flight still holds
+    // lives on until that call lets go of it.
+    size_t held = 0;
+    for (const auto& t : g_tables)
+        held += table_device_bytes(*t);
+    while (!g_tables.empty() &&
+           (g_tables.size() >= kMaxCachedTables ||
+            held + seg_bytes + first_bytes + short_bytes > kMaxCachedTableBytes)) {
+        held -= table_device_bytes(*g_tables.front());
+        dropped.push_back(std::move(g_tables.front()));
+        g_tables.erase(g_tables.begin());
+    }
+    tab->owns_device_arrays = true;
+    cudaError_t err = cudaMalloc(&tab->d_segments, seg_bytes);
+    if (err == cudaSuccess)
+        err = cudaMalloc(&tab->d_seg_first, first_bytes);
     // Blocking copies: the table may be used from any stream afterwards.
     if (err == cudaSuccess && !tab->h_segments.empty())
         err = cudaMemcpy(tab->d_segments, tab->h_segments.data(),
                          sizeof(Segment) * tab->h_segments.size(), cudaMemcpyHostToDevice);
     if (err == cudaSuccess)
         err = cudaMemcpy(tab->d_seg_first, tab->h_seg_first.data(), first_bytes, cudaMemcpyHostToDevice);
-    if (err != cudaSuccess) {
-        cudaFree(tab->d_segments);
-        cudaFree(tab->d_seg_first);
-        return fail(ADASUM_ERR_CUDA, "segment table upload: %s", cudaGetErrorString(err));
+    if (err == cudaSuccess && !tab->h_short.empty()) {
+        err = cudaMalloc(&tab->d_short, short_bytes);
+        if (err == cudaSuccess)
+            err = cudaMemcpy(tab->d_short, tab->h_short.data(), sizeof(ShortTensor) * tab->h_short.size(),
+                             cudaMemcpyHostToDevice);
     }
-    *out = tab.get();
-    g_tables.push_back(std::move(tab));
+    if (err != cudaSuccess)
+        return fail(ADASUM_ERR_CUDA, "segment table upload: %s", cudaGetErrorString(err));
+    g_tables.push_back(tab);
+    *out = std::move(tab);
     return ADASUM_OK;
 }
-
-// ---- launches ----------------------------------------------------------------------------------
-
-// Opt a kernel in to `bytes` of dynamic shared memory, once per device.
-template <typename Kernel>
-cudaError_t allow_dynamic_smem(Kernel kernel, size_t bytes, bool (&configured)[64])
-{
-    int device = 0;
-    cudaError_t err = cudaGetDevice(&device);
-    if (err != cudaSuccess)
-        return err;
-    if (device < 0 || device >= 64)
-        return cudaErrorInvalidDevice;
-    if (!configured[device]) {
-        err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-        if (err != cudaSuccess)
-            return err;
-        configured[device] = true;
-    }
-    return cudaSuccess;
-}
-
-template <typename T, int R, bool VEC, bool DELTA>
-cudaError_t launch_gram_variant(GramKind kind, const OperandTable& ops, int operands, int groups_here,
-                                const SegmentTable& tab, float* partials, int groups_total, int group_base,
-                                const FinishArgs& fin, cudaStream_t stream, int* tc_status, const void* start)
-{
-    if constexpr (R == 64 && VEC && sizeof(T) == 2 && !DELTA) {
-        // every group complete: the tcgen05 kernel (64 x 64 accumulator in tensor memory)
-        if (kind == GRAM_MMA && tc_status != nullptr && operands == groups_here * 64) {
-            auto kernel = gram_partial_tc64_kernel<T>;
-            static bool configured[64] = {};
-            cudaError_t err = allow_dynamic_smem(kernel, kTcSmemBytes, configured);
-            if (err != cudaSuccess)
-                return err;
-            dim3 grid((unsigned)tab.num_segments, (unsigned)groups_here);
-            kernel<<<grid, kTcThreads, kTcSmemBytes, stream>>>(ops, operands, tab.d_segments, partials, groups_total,
-                                                               group_base, fin, tc_status);
-            return cudaSuccess;
-        }
-    }
-    if constexpr (R >= 8) {
-        if (kind == GRAM_MMA) {
-            if constexpr (R <= 32 || sizeof(T) == 2) {
-                constexpr size_t smem = mma_smem_bytes<T, R, DELTA>();
-                auto kernel = gram_partial_mma_kernel<T, R, VEC, DELTA>;
-                static bool configured[64] = {};
-                cudaError_t err = allow_dynamic_smem(kernel, smem, configured);
-                if (err != cudaSuccess)
-                    return err;
-                dim3 grid((unsigned)tab.num_segments, (unsigned)groups_here);
-                kernel<<<grid, kThreads, smem, stream>>>(ops, operands, tab.d_segments, partials, groups_total,
-                                                         group_base, fin, start);
-                return cudaSuccess;
-            } else {
-                return cudaErrorInvalidValue;
-            }
-        }
-    }
-    if constexpr (R <= 16) {
-        if (kind == GRAM_SIMPLE) {
-            dim3 grid((unsigned)tab.num_segments, (unsigned)groups_here);
-            gram_partial_kernel<T, R, VEC, DELTA><<<grid, kThreads, 0, stream>>>(
-                ops, operands, tab.d_segments, partials, groups_total, group_base, fin, start);
-            return cudaSuccess;
-        }
-    }
-    return cudaErrorInvalidValue;
-}
-
-// `start` != nullptr selects the kernels that read the operands as (operand - start); those exist
-// for 16-byte aligned buffers only (the caller has checked).
-template <typename T, int R, bool VEC>
-cudaError_t launch_gram(GramKind kind, const OperandTable& ops, int operands, int groups_here,
-                        const SegmentTable& tab, float* partials, int groups_total, int group_base,
-                        const FinishArgs& fin, cudaStream_t stream, int* tc_status = nullptr,
-                        const void* start = nullptr)
-{
-    if constexpr (VEC) {
-        if (start != nullptr)
-            return launch_gram_variant<T, R, true, true>(kind, ops, operands, groups_here, tab, partials, groups_total,
-                                                         group_base, fin, stream, tc_status, start);
-    }
-    if (start != nullptr)
-        return cudaErrorInvalidValue;
-    return launch_gram_variant<T, R, VEC, false>(kind, ops, operands, groups_here, tab, partials, groups_total,
-                                                 group_base, fin, stream, tc_status, nullptr);
-}
-
-constexpr PassExtras kNoExtras{nullptr, nullptr, 0, 0};
-
-template <typename T, int R, bool VEC>
-void launch_wsum(const OperandTable& ops, int operands, int groups_here, const SegmentTable& tab,
-                 const float* weights, int groups_total, int group_base, void* dst, int64_t dst_stride,
-                 cudaStream_t stream, const PassExtras& ex = kNoExtras)
-{
-    dim3 grid((unsigned)tab.num_segments, (unsigned)groups_here);
-    if constexpr (VEC) {
-        if (ex.start != nullptr) {
-            weighted_sum_kernel<T, R, true, true><<<grid, kThreads, 0, stream>>>(
-                ops, operands, tab.d_segments, weights, groups_total, group_base, dst, dst_stride, ex);
-            return;
-        }
-    }
-    weighted_sum_kernel<T, R, VEC, false><<<grid, kThreads, 0, stream>>>(ops, operands, tab.d_segments, weights,
-                                                                         groups_total, group_base, dst, dst_stride, ex);
-}
-
-template <int R>
-cudaError_t launch_weights(const float* partials, const SegmentTable& tab, int32_t num_tensors, int operands,
-                           int groups, double* gram64, float* weights, const TreeOptions& opt, cudaStream_t stream,
-                           int* launches, bool sums_only = false)
-{
-    dim3 grid((unsigned)num_tensors, (unsigned)groups, (unsigned)tree_entry_blocks(R));
-    // wide blocks only pay off when some tensor has many per-segment partials to add
-    const int threads = tab.max_segments_per_tensor > 64 ? kTreeThreadsMax : 256;
-    gram_finish_kernel<R><<<grid, threads, threads * sizeof(double), stream>>>(partials, tab.d_seg_first, operands,
-                                                                                gram64, weights, opt, sums_only ? 1 : 0);
-    *launches = 1;
-    if (sums_only)
-        return cudaSuccess;
-    if constexpr (tree_entry_blocks(R) > 1) {
-        dim3 grid2((unsigned)num_tensors, (unsigned)groups);
-        tree_weights_kernel<R><<<grid2, kThreads, 0, stream>>>(gram64, operands, weights, opt);
-        *launches = 2;
-    }
-    return cudaSuccess;
-}
-
-template <int R>
-void launch_tree_from_sums(const double* gram64, int32_t num_tensors, int operands, int groups, float* weights,
-                           const TreeOptions& opt, cudaStream_t stream)
-{
-    dim3 grid((unsigned)num_tensors, (unsigned)groups);
-    tree_weights_kernel<R><<<grid, kThreads, 0, stream>>>(gram64, operands, weights, opt);
-}
-
-// Which part of a level a call runs.
-enum LevelPhase {
-    PHASE_WHOLE = 0,        // pass 1, coefficients, pass 2
-    PHASE_GRAM_SUMS = 1,    // pass 1, then this GPU's fp64 Gram sums to gram64 (to be added across GPUs)
-    PHASE_APPLY = 2         // coefficients from gram64, then pass 2
-};
 
 // ---- single-launch path for inputs that fit the L2 ------------------------------------------------
 
@@ -554,38 +443,6 @@ bool small_input_plan(const LevelPlan& plan, int64_t total, int32_t num_tensors,
     return true;
 }
 
-template <typename T, int R, bool VEC>
-cudaError_t launch_fused_small(const OperandTable& ops, int operands, const SegmentTable& tab, float* partials,
-                               const FinishArgs& fin, void* out, const PassExtras& ex, int* status, cudaStream_t stream)
-{
-    const void* kernel = (const void*)fused_small_kernel<T, R, VEC, false>;
-    if constexpr (VEC) {
-        if (ex.start != nullptr)
-            kernel = (const void*)fused_small_kernel<T, R, true, true>;
-    }
-    if (!VEC && ex.start != nullptr)
-        return cudaErrorInvalidValue;
-    int operands_arg = operands;
-    const Segment* segments = tab.d_segments;
-    PassExtras ex_arg = ex;
-    void* args[] = {(void*)&ops, (void*)&operands_arg, (void*)&segments, (void*)&partials,
-                    (void*)&fin, (void*)&out,          (void*)&ex_arg,   (void*)&status};
-    return cudaLaunchCooperativeKernel(kernel, dim3((unsigned)tab.num_segments), dim3(kThreads), args, 0, stream);
-}
-
-template <typename T, bool VEC>
-cudaError_t launch_fused_small_radix(int radix, const OperandTable& ops, int operands, const SegmentTable& tab,
-                                     float* partials, const FinishArgs& fin, void* out, const PassExtras& ex,
-                                     int* status, cudaStream_t stream)
-{
-    switch (radix) {
-    case 2: return launch_fused_small<T, 2, VEC>(ops, operands, tab, partials, fin, out, ex, status, stream);
-    case 4: return launch_fused_small<T, 4, VEC>(ops, operands, tab, partials, fin, out, ex, status, stream);
-    case 8: return launch_fused_small<T, 8, VEC>(ops, operands, tab, partials, fin, out, ex, status, stream);
-    default: return cudaErrorInvalidValue;
-    }
-}
-
 // Blocks of fused_small_kernel that the current device keeps resident (0: no cooperative launch).
 int resident_small_blocks()
 {
@@ -602,141 +459,6 @@ int resident_small_blocks()
             cached[device] = sms * kSmallBlocksPerSm;
     }
     return cached[device] > 0 ? cached[device] : 0;
-}
-
-struct LevelArgs {
-    const void* const* operand_ptrs;   // host array, `operands` entries
-    int operands;
-    int groups;
-    GramKind kind;
-    const SegmentTable* gram_tab;
-    const SegmentTable* wsum_tab;
-    int32_t num_tensors;
-    float* partials;
-    int* counters;      // ticket counters for finishing inside pass 1, or nullptr
-    TreeOptions tree;
-    LevelPhase phase;
-    int* tc_status;     // status word for the tcgen05 kernel, or nullptr to keep to mma.sync
-    double* gram64;
-    float* weights;
-    void* dst;
-    int64_t dst_stride;
-    PassExtras extras;   // start: this level's operands are (operand - start); base / out_dtype: last level
-    bool vec;
-    cudaStream_t stream;
-    int level;
-    // fusion of this level's pass 2 with the next level's pass 1 (wsum_gram_kernel)
-    bool skip_gram;              // this level's Gram sums and weights were produced by the previous level's pass 2
-    int fuse_next_radix;         // 0: plain pass 2; 2 or 4: also pass 1 of the next level, which has this radix
-    const SegmentTable* fuse_tab;
-    int next_groups;
-    float* next_weights;
-    TreeOptions next_tree;
-};
-
-// Measured on a B200: fusing pays while this level's groups are narrow (literal tree 0.60 -> 0.54 ms on
-// the ResNet-50 list with 8 workers, 14.7 -> 13.0 ms on the BERT-Large list with 16); from radix 8 on
-// the plain second pass, which keeps three blocks per SM busy, is faster than the saving.
-bool fusable_radices(int radix, int next_radix) { return radix <= 4 && (next_radix == 2 || next_radix == 4); }
-
-template <typename T, int R1, int R2>
-adasum_status_t launch_wsum_gram(const LevelArgs& a)
-{
-    constexpr int kNextGroupsPerLaunch = kMaxOperandsPerLaunch / (R1 * R2);
-    const FinishArgs next_fin{a.fuse_tab->d_seg_first, a.counters, a.next_weights, a.next_tree};
-    for (int ng0 = 0; ng0 < a.next_groups; ng0 += kNextGroupsPerLaunch) {
-        const int next_here = a.next_groups - ng0 < kNextGroupsPerLaunch ? a.next_groups - ng0 : kNextGroupsPerLaunch;
-        const int g0 = ng0 * R2, op0 = g0 * R1;
-        const int ops_here = a.operands - op0 < kMaxOperandsPerLaunch ? a.operands - op0 : kMaxOperandsPerLaunch;
-        OperandTable table;
-        for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
-            table.ptr[i] = a.operand_ptrs[op0 + (i < ops_here ? i : 0)];
-        dim3 grid((unsigned)a.fuse_tab->num_segments, (unsigned)next_here);
-        wsum_gram_kernel<T, R1, R2, true><<<grid, kThreads, 0, a.stream>>>(
-            table, ops_here, a.fuse_tab->d_segments, a.weights, a.groups, g0, static_cast<float*>(a.dst), a.dst_stride,
-            a.partials, a.next_groups, ng0, next_fin);
-        profile_mark(a.stream, ADASUM_KERNEL_WSUM_GRAM, a.level, R1, false);
-    }
-    ADASUM_CUDA_CHECK(cudaGetLastError());
-    return ADASUM_OK;
-}
-
-template <typename T, int R>
-adasum_status_t run_level_typed(const LevelArgs& a)
-{
-    constexpr int kGroupsPerLaunch = kMaxOperandsPerLaunch / R;
-    // the last block of every (tensor, group) in pass 1 also derives the weights
-    const bool fused_finish = a.counters != nullptr && a.phase == PHASE_WHOLE;
-    const FinishArgs fin{a.gram_tab->d_seg_first, fused_finish ? a.counters : nullptr, a.weights, a.tree};
-    // pass 1
-    for (int g0 = 0; g0 < a.groups && a.phase != PHASE_APPLY && !a.skip_gram; g0 += kGroupsPerLaunch) {
-        const int groups_here = a.groups - g0 < kGroupsPerLaunch ? a.groups - g0 : kGroupsPerLaunch;
-        const int op0 = g0 * R;
-        const int ops_here = a.operands - op0 < kMaxOperandsPerLaunch ? a.operands - op0 : kMaxOperandsPerLaunch;
-        OperandTable table;
-        for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
-            table.ptr[i] = a.operand_ptrs[op0 + (i < ops_here ? i : 0)];
-        if (a.vec)
-            ADASUM_CUDA_CHECK((launch_gram<T, R, true>(a.kind, table, ops_here, groups_here, *a.gram_tab,
-                                                       a.partials, a.groups, g0, fin, a.stream, a.tc_status,
-                                                       a.extras.start)));
-        else
-            ADASUM_CUDA_CHECK((launch_gram<T, R, false>(a.kind, table, ops_here, groups_here, *a.gram_tab,
-                                                        a.partials, a.groups, g0, fin, a.stream)));
-        profile_mark(a.stream, ADASUM_KERNEL_GRAM_PARTIAL, a.level, R, false);
-    }
-    if (a.phase == PHASE_APPLY) {
-        launch_tree_from_sums<R>(a.gram64, a.num_tensors, a.operands, a.groups, a.weights, a.tree, a.stream);
-        profile_mark(a.stream, ADASUM_KERNEL_TREE_WEIGHTS, a.level, R, false);
-    } else if (!fused_finish && !a.skip_gram) {
-        int weight_launches = 0;
-        ADASUM_CUDA_CHECK(launch_weights<R>(a.partials, *a.gram_tab, a.num_tensors, a.operands, a.groups,
-                                            a.gram64, a.weights, a.tree, a.stream, &weight_launches,
-                                            a.phase == PHASE_GRAM_SUMS));
-        profile_mark(a.stream, ADASUM_KERNEL_TREE_WEIGHTS, a.level, R, false);
-    }
-    // pass 2, together with the next level's pass 1 where that is possible
-    if constexpr (R <= 4) {
-        if (a.fuse_next_radix == 2)
-            return launch_wsum_gram<T, R, 2>(a);
-        if (a.fuse_next_radix == 4)
-            return launch_wsum_gram<T, R, 4>(a);
-    }
-    for (int g0 = 0; g0 < a.groups && a.phase != PHASE_GRAM_SUMS; g0 += kGroupsPerLaunch) {
-        const int groups_here = a.groups - g0 < kGroupsPerLaunch ? a.groups - g0 : kGroupsPerLaunch;
-        const int op0 = g0 * R;
-        const int ops_here = a.operands - op0 < kMaxOperandsPerLaunch ? a.operands - op0 : kMaxOperandsPerLaunch;
-        OperandTable table;
-        for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
-            table.ptr[i] = a.operand_ptrs[op0 + (i < ops_here ? i : 0)];
-        if (a.vec)
-            launch_wsum<T, R, true>(table, ops_here, groups_here, *a.wsum_tab, a.weights, a.groups, g0, a.dst,
-                                    a.dst_stride, a.stream, a.extras);
-        else
-            launch_wsum<T, R, false>(table, ops_here, groups_here, *a.wsum_tab, a.weights, a.groups, g0, a.dst,
-                                     a.dst_stride, a.stream, a.extras);
-        profile_mark(a.stream, ADASUM_KERNEL_WEIGHTED_SUM, a.level, R, false);
-    }
-    ADASUM_CUDA_CHECK(cudaGetLastError());
-    return ADASUM_OK;
-}
-
-template <typename T>
-adasum_status_t run_level(int radix, const LevelArgs& a)
-{
-    switch (radix) {
-    case 2: return run_level_typed<T, 2>(a);
-    case 4: return run_level_typed<T, 4>(a);
-    case 8: return run_level_typed<T, 8>(a);
-    case 16: return run_level_typed<T, 16>(a);
-    case 32: return run_level_typed<T, 32>(a);
-    case 64:
-        if constexpr (sizeof(T) == 2)
-            return run_level_typed<T, 64>(a);
-        else
-            return fail(ADASUM_ERR_ARG, "radix 64 needs fp16 / bf16 operands");
-    default: return fail(ADASUM_ERR_ARG, "unsupported radix %d", radix);
-    }
 }
 
 int launches_of(const LevelPlan& plan, int n_workers, uint32_t flags, int64_t total, int32_t num_tensors,
@@ -866,7 +588,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     }
     if (start != nullptr && total > 0 && !vec)
         return fail(ADASUM_ERR_ARG, "the delta form needs every buffer 16-byte aligned");
-    const Layout lay = make_layout(plan, total, num_tensors);
+    const Layout lay = make_layout(plan, total, num_tensors, n_workers);
     if (n_workers > 1) {
         if (!workspace)
             return fail(ADASUM_ERR_WORKSPACE, "workspace is NULL");
@@ -887,17 +609,14 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
 
     profile_mark(stream, -1, 0, 0, true);
     if (n_workers == 1) {
-        const int64_t blocks = (total + kThreads - 1) / kThreads;
-        const unsigned grid = (unsigned)(blocks < 148 * 16 ? blocks : 148 * 16);
         PassExtras ex = last_extras;
         ex.start = start;
         if (dtype == ADASUM_F32)
-            convert_kernel<float><<<grid, kThreads, 0, stream>>>((const float*)grads[0], out, total, ex);
+            ADASUM_CUDA_CHECK(launch_convert<float>(grads[0], out, total, ex, stream));
         else if (dtype == ADASUM_F16)
-            convert_kernel<__half><<<grid, kThreads, 0, stream>>>((const __half*)grads[0], out, total, ex);
+            ADASUM_CUDA_CHECK(launch_convert<__half>(grads[0], out, total, ex, stream));
         else
-            convert_kernel<__nv_bfloat16><<<grid, kThreads, 0, stream>>>((const __nv_bfloat16*)grads[0], out, total, ex);
-        ADASUM_CUDA_CHECK(cudaGetLastError());
+            ADASUM_CUDA_CHECK(launch_convert<__nv_bfloat16>(grads[0], out, total, ex, stream));
         profile_mark(stream, ADASUM_KERNEL_CONVERT, 0, 1, false);
         return ADASUM_OK;
     }
@@ -934,11 +653,74 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     profile_mark(stream, -1, 0, 0, true);
     std::vector<const void*> operand_ptrs(grads, grads + n_workers);
 
+    // Tensors of at most kShortTensorElems elements are left out of the streaming kernels' segment
+    // tables and reduced in fp64 by a kernel of their own, launched last.  Not in the sharded calls:
+    // there a tensor's elements are spread over several GPUs and only its Gram sums travel.
+    const bool skip_short = !sharded;
+    TableRef short_ref;          // held for the whole call: every level's pass 2 uses this table too
+    if (skip_short) {
+        st = get_segment_table(offsets, num_tensors, wsum_segment_length(total), true, &short_ref);
+        if (st != ADASUM_OK)
+            return st;
+    }
+    auto run_short = [&]() -> adasum_status_t {
+        const int num_short = short_ref ? (int)short_ref->h_short.size() : 0;
+        if (num_short == 0)
+            return ADASUM_OK;
+        ShortArgs sa{};
+        sa.table = short_ref->d_short;
+        sa.order = tree_order(n_workers, flags);
+        sa.start = start;
+        sa.base_dtype = (int)dtype;
+        sa.out_dtype = (int)out_dtype;
+        OperandTable table;
+        if (n_workers <= kMaxOperandsPerLaunch) {
+            for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
+                table.ptr[i] = grads[i < n_workers ? i : 0];
+            sa.out = out;
+            sa.base = start;
+            sa.orthogonality = orthogonality;
+            ADASUM_CUDA_CHECK(launch_short_tensors((int)dtype, table, n_workers, num_short, sa, stream));
+            profile_mark(stream, ADASUM_KERNEL_SHORT_TENSORS, 0, 2, false);
+            return ADASUM_OK;
+        }
+        // more workers than one launch carries: every launch reduces the complete sub-tree of its
+        // kMaxOperandsPerLaunch workers to one fp64 vector, a last launch reduces those
+        double* vecs = reinterpret_cast<double*>(ws + lay.short_vecs);
+        double* sums = reinterpret_cast<double*>(ws + lay.short_sums);
+        const int launches = (n_workers + kMaxOperandsPerLaunch - 1) / kMaxOperandsPerLaunch;
+        for (int j = 0; j < launches; ++j) {
+            const int w0 = j * kMaxOperandsPerLaunch;
+            const int here = n_workers - w0 < kMaxOperandsPerLaunch ? n_workers - w0 : kMaxOperandsPerLaunch;
+            for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
+                table.ptr[i] = grads[w0 + (i < here ? i : 0)];
+            ShortArgs part = sa;
+            part.vec_out = vecs + (int64_t)j * lay.short_vec_stride;
+            part.leaf_sum_out = sums + (int64_t)j * lay.short_sum_stride;
+            ADASUM_CUDA_CHECK(launch_short_tensors((int)dtype, table, here, num_short, part, stream));
+            profile_mark(stream, ADASUM_KERNEL_SHORT_TENSORS, 0, 2, false);
+        }
+        for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
+            table.ptr[i] = vecs + (int64_t)(i < launches ? i : 0) * lay.short_vec_stride;
+        sa.start = nullptr;
+        sa.out = out;
+        sa.base = start;
+        sa.orthogonality = orthogonality;
+        sa.leaf_sum_in = sums;
+        sa.leaf_sum_launches = launches;
+        sa.leaf_sum_stride = lay.short_sum_stride;
+        ADASUM_CUDA_CHECK(launch_short_tensors(3, table, launches, num_short, sa, stream));
+        profile_mark(stream, ADASUM_KERNEL_SHORT_TENSORS, 1, 2, false);
+        return ADASUM_OK;
+    };
+    if (short_ref && short_ref->num_segments == 0)        // every tensor is short
+        return run_short();
+
     // Inputs that fit the L2: one cooperative launch does both passes and HBM sees the operands once.
     if (small_candidate) {
         int* dev_status = reinterpret_cast<int*>(ws + lay.counters + lay.counters_bytes - sizeof(int));
-        const SegmentTable* tab = nullptr;
-        st = get_segment_table(offsets, num_tensors, small_seg_len, &tab);
+        TableRef tab;
+        st = get_segment_table(offsets, num_tensors, small_seg_len, skip_short, &tab);
         if (st != ADASUM_OK)
             return st;
         if (tab->num_segments <= small_blocks) {
@@ -958,17 +740,14 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
             ex.start = start;
             cudaError_t err;
             if (dtype == ADASUM_F32)
-                err = vec ? launch_fused_small_radix<float, true>(radix, table, n_workers, *tab, partials, fin, out, ex, dev_status, stream)
-                          : launch_fused_small_radix<float, false>(radix, table, n_workers, *tab, partials, fin, out, ex, dev_status, stream);
+                err = launch_fused_small_any<float>(vec, radix, table, n_workers, *tab, partials, fin, out, ex, dev_status, stream);
             else if (dtype == ADASUM_F16)
-                err = vec ? launch_fused_small_radix<__half, true>(radix, table, n_workers, *tab, partials, fin, out, ex, dev_status, stream)
-                          : launch_fused_small_radix<__half, false>(radix, table, n_workers, *tab, partials, fin, out, ex, dev_status, stream);
+                err = launch_fused_small_any<__half>(vec, radix, table, n_workers, *tab, partials, fin, out, ex, dev_status, stream);
             else
-                err = vec ? launch_fused_small_radix<__nv_bfloat16, true>(radix, table, n_workers, *tab, partials, fin, out, ex, dev_status, stream)
-                          : launch_fused_small_radix<__nv_bfloat16, false>(radix, table, n_workers, *tab, partials, fin, out, ex, dev_status, stream);
+                err = launch_fused_small_any<__nv_bfloat16>(vec, radix, table, n_workers, *tab, partials, fin, out, ex, dev_status, stream);
             if (err == cudaSuccess) {
                 profile_mark(stream, ADASUM_KERNEL_FUSED_SMALL, 0, radix, false);
-                return ADASUM_OK;
+                return run_short();
             }
             if (err != cudaErrorCooperativeLaunchTooLarge)
                 return fail(ADASUM_ERR_CUDA, "cooperative launch: %s", cudaGetErrorString(err));
@@ -991,12 +770,11 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         }
         const bool simple_kernels = (flags & ADASUM_FLAG_SIMPLE_KERNELS) != 0;
         const GramKind kind = gram_kind(lv.radix, simple_kernels);
-        const SegmentTable* gram_tab = nullptr;
-        const SegmentTable* wsum_tab = nullptr;
-        st = get_segment_table(offsets, num_tensors, gram_segment_length(kind, total), &gram_tab);
+        TableRef gram_tab, wsum_tab, fuse_tab;     // held until this level's launches are enqueued
+        st = get_segment_table(offsets, num_tensors, gram_segment_length(kind, total), skip_short, &gram_tab);
         if (st != ADASUM_OK)
             return st;
-        st = get_segment_table(offsets, num_tensors, wsum_segment_length(total), &wsum_tab);
+        st = get_segment_table(offsets, num_tensors, wsum_segment_length(total), skip_short, &wsum_tab);
         if (st != ADASUM_OK)
             return st;
         const bool last = l + 1 == plan.num_levels;
@@ -1005,8 +783,8 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         a.operands = lv.operands;
         a.groups = lv.groups;
         a.kind = kind;
-        a.gram_tab = gram_tab;
-        a.wsum_tab = wsum_tab;
+        a.gram_tab = gram_tab.get();
+        a.wsum_tab = wsum_tab.get();
         a.num_tensors = num_tensors;
         a.partials = reinterpret_cast<float*>(ws + lay.partials);
         a.weights = reinterpret_cast<float*>(ws + ((l & 1) ? lay.weights_alt : lay.weights));
@@ -1040,9 +818,10 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         gram_done = false;
         if (!last && !sharded && !separate_finish && vec && !(flags & ADASUM_FLAG_NO_LEVEL_FUSION) &&
             a.extras.start == nullptr && fusable_radices(lv.radix, plan.level[l + 1].radix)) {
-            st = get_segment_table(offsets, num_tensors, gram_segment_length(GRAM_SIMPLE, total), &a.fuse_tab);
+            st = get_segment_table(offsets, num_tensors, gram_segment_length(GRAM_SIMPLE, total), skip_short, &fuse_tab);
             if (st != ADASUM_OK)
                 return st;
+            a.fuse_tab = fuse_tab.get();
             a.fuse_next_radix = plan.level[l + 1].radix;
             a.next_groups = plan.level[l + 1].groups;
             a.next_weights = reinterpret_cast<float*>(ws + (((l + 1) & 1) ? lay.weights_alt : lay.weights));
@@ -1068,7 +847,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
                 operand_ptrs[g] = static_cast<float*>(a.dst) + (int64_t)g * lay.padded_elems;
         }
     }
-    return ADASUM_OK;
+    return run_short();
 }
 
 // ---- fp64 gradients ------------------------------------------------------------------------------
@@ -1286,8 +1065,8 @@ adasum_status_t reduce_f64_impl(const void* const* grads, const int64_t* offsets
         ADASUM_CUDA_CHECK(cudaMemsetAsync(orthogonality, 0xff, sizeof(float) * (size_t)num_tensors, stream));
     if (num_tensors == 0)
         return ADASUM_OK;
-    const SegmentTable* tab = nullptr;
-    st = get_segment_table(offsets, num_tensors, segment_length_f64(total), &tab);
+    TableRef tab;
+    st = get_segment_table(offsets, num_tensors, segment_length_f64(total), false, &tab);
     if (st != ADASUM_OK)
         return st;
     // per-launch timing: the first kernel's interval starts here, after the clearing of counters above
@@ -1300,7 +1079,7 @@ adasum_status_t reduce_f64_impl(const void* const* grads, const int64_t* offsets
         a.operand_ptrs = operand_ptrs.data();
         a.operands = lv.operands;
         a.groups = lv.groups;
-        a.tab = tab;
+        a.tab = tab.get();
         a.partials = reinterpret_cast<double*>(ws + lay.partials);
         a.fin.seg_first = tab->d_seg_first;
         a.fin.counters = reinterpret_cast<int*>(ws + lay.counters);
@@ -1342,7 +1121,9 @@ constexpr size_t kNoallocSegBytes = ((size_t)kNoallocMaxSegments * sizeof(Segmen
 constexpr size_t kNoallocFirstBytes = ((size_t)(2 * kNoallocMaxTensors + 2) * sizeof(int32_t) + 255) / 256 * 256;
 constexpr size_t kNoallocPartialBytes = ((size_t)kNoallocMaxSegments * gram_entries(2) * sizeof(float) + 255) / 256 * 256;
 constexpr size_t kNoallocWeightBytes = ((size_t)kNoallocMaxTensors * 2 * sizeof(float) + 255) / 256 * 256;
-constexpr size_t kNoallocScratchBytes = kNoallocSegBytes + kNoallocFirstBytes + kNoallocPartialBytes + kNoallocWeightBytes;
+constexpr size_t kNoallocShortBytes = ((size_t)kNoallocMaxTensors * sizeof(ShortTensor) + 255) / 256 * 256;
+constexpr size_t kNoallocScratchBytes =
+    kNoallocSegBytes + kNoallocFirstBytes + kNoallocPartialBytes + kNoallocWeightBytes + kNoallocShortBytes;
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoallocScratchBytes];
 
@@ -1366,27 +1147,6 @@ adasum_status_t noalloc_scratch(unsigned char** ptr)
     }
     *ptr = g_noalloc_device_ptr[device];
     return ADASUM_OK;
-}
-
-template <typename T>
-cudaError_t noalloc_launch(bool vec, const OperandTable& ops, const SegmentTable& tab, int32_t num_tensors,
-                           float* partials, float* weights, float* out, cudaStream_t stream)
-{
-    const TreeOptions plain_tree{0, 1, 1, 1, nullptr, nullptr};
-    const FinishArgs no_fusion{nullptr, nullptr, nullptr, plain_tree};
-    cudaError_t err = vec ? launch_gram<T, 2, true>(GRAM_SIMPLE, ops, 2, 1, tab, partials, 1, 0, no_fusion, stream)
-                          : launch_gram<T, 2, false>(GRAM_SIMPLE, ops, 2, 1, tab, partials, 1, 0, no_fusion, stream);
-    if (err != cudaSuccess)
-        return err;
-    int weight_launches = 0;
-    err = launch_weights<2>(partials, tab, num_tensors, 2, 1, nullptr, weights, plain_tree, stream, &weight_launches);
-    if (err != cudaSuccess)
-        return err;
-    if (vec)
-        launch_wsum<T, 2, true>(ops, 2, 1, tab, weights, 1, 0, out, 0, stream);
-    else
-        launch_wsum<T, 2, false>(ops, 2, 1, tab, weights, 1, 0, out, 0, stream);
-    return cudaSuccess;
 }
 
 adasum_status_t pair_noalloc_impl(const void* a, const void* b, const int64_t* offsets, int32_t num_tensors,
@@ -1425,33 +1185,56 @@ adasum_status_t pair_noalloc_impl(const void* a, const void* b, const int64_t* o
         vec = vec && aligned16(in[w]);
     }
 
+    // This call's segment table is copied from host vectors that die when the call returns.  A
+    // captured copy would read them at every replay, long after that, so a capturing stream is refused.
+    cudaStreamCaptureStatus capture = cudaStreamCaptureStatusNone;
+    ADASUM_CUDA_CHECK(cudaStreamIsCapturing(stream, &capture));
+    if (capture != cudaStreamCaptureStatusNone)
+        return fail(ADASUM_ERR_ARG, "adasum_pair_noalloc cannot be recorded into a CUDA graph: it uploads a "
+                                    "per-call table from temporary host memory");
     unsigned char* scratch = nullptr;
     st = noalloc_scratch(&scratch);
     if (st != ADASUM_OK)
         return st;
     SegmentTable tab;                       // host-side only; its device pointers aim into the scratch
-    build_segments(offsets, num_tensors, kNoallocSegLen, &tab);
+    build_segments(offsets, num_tensors, kNoallocSegLen, true, &tab);      // short tensors apart, as in adasum_pair
     if ((int64_t)tab.num_segments > kNoallocMaxSegments)
         return fail(ADASUM_ERR_ARG, "segment table does not fit the static scratch");
     tab.d_segments = reinterpret_cast<Segment*>(scratch);
     tab.d_seg_first = reinterpret_cast<int32_t*>(scratch + kNoallocSegBytes);
     float* partials = reinterpret_cast<float*>(scratch + kNoallocSegBytes + kNoallocFirstBytes);
     float* weights = reinterpret_cast<float*>(scratch + kNoallocSegBytes + kNoallocFirstBytes + kNoallocPartialBytes);
+    ShortTensor* short_table = reinterpret_cast<ShortTensor*>(scratch + kNoallocSegBytes + kNoallocFirstBytes +
+                                                              kNoallocPartialBytes + kNoallocWeightBytes);
     // The host vectors are pageable memory: cudaMemcpyAsync has read them completely when it
     // returns, and the copies are ordered before the kernels on `stream`.
-    ADASUM_CUDA_CHECK(cudaMemcpyAsync(tab.d_segments, tab.h_segments.data(), sizeof(Segment) * tab.h_segments.size(),
-                                      cudaMemcpyHostToDevice, stream));
+    if (!tab.h_segments.empty())
+        ADASUM_CUDA_CHECK(cudaMemcpyAsync(tab.d_segments, tab.h_segments.data(),
+                                          sizeof(Segment) * tab.h_segments.size(), cudaMemcpyHostToDevice, stream));
     ADASUM_CUDA_CHECK(cudaMemcpyAsync(tab.d_seg_first, tab.h_seg_first.data(),
                                       sizeof(int32_t) * tab.h_seg_first.size(), cudaMemcpyHostToDevice, stream));
+    if (!tab.h_short.empty())
+        ADASUM_CUDA_CHECK(cudaMemcpyAsync(short_table, tab.h_short.data(), sizeof(ShortTensor) * tab.h_short.size(),
+                                          cudaMemcpyHostToDevice, stream));
     OperandTable ops;
     for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
         ops.ptr[i] = in[i < 2 ? i : 0];
-    if (dtype == ADASUM_F32)
-        ADASUM_CUDA_CHECK(noalloc_launch<float>(vec, ops, tab, num_tensors, partials, weights, out, stream));
-    else if (dtype == ADASUM_F16)
-        ADASUM_CUDA_CHECK(noalloc_launch<__half>(vec, ops, tab, num_tensors, partials, weights, out, stream));
-    else
-        ADASUM_CUDA_CHECK(noalloc_launch<__nv_bfloat16>(vec, ops, tab, num_tensors, partials, weights, out, stream));
+    if (tab.num_segments > 0) {
+        if (dtype == ADASUM_F32)
+            ADASUM_CUDA_CHECK(noalloc_launch<float>(vec, ops, tab, num_tensors, partials, weights, out, stream));
+        else if (dtype == ADASUM_F16)
+            ADASUM_CUDA_CHECK(noalloc_launch<__half>(vec, ops, tab, num_tensors, partials, weights, out, stream));
+        else
+            ADASUM_CUDA_CHECK(noalloc_launch<__nv_bfloat16>(vec, ops, tab, num_tensors, partials, weights, out, stream));
+    }
+    if (!tab.h_short.empty()) {         // tensors of at most kShortTensorElems elements: the fp64 kernel
+        ShortArgs sa{};
+        sa.table = short_table;
+        sa.out = out;
+        sa.base_dtype = (int)dtype;
+        sa.out_dtype = (int)ADASUM_F32;
+        ADASUM_CUDA_CHECK(launch_short_tensors((int)dtype, ops, 2, (int)tab.h_short.size(), sa, stream));
+    }
     ADASUM_CUDA_CHECK(cudaGetLastError());
     return ADASUM_OK;
 }
@@ -1474,7 +1257,7 @@ size_t adasum_workspace_bytes(int64_t total_elems, int32_t num_tensors, int32_t 
         return plan_levels_f64(n_workers, flags, &plan) ? make_layout_f64(plan, total_elems, num_tensors).total : 0;
     if (!plan_levels(n_workers, dtype, flags, &plan))
         return 0;
-    return make_layout(plan, total_elems, num_tensors).total;
+    return make_layout(plan, total_elems, num_tensors, n_workers).total;
 }
 
 adasum_status_t adasum_plan_info(int64_t total_elems, int32_t num_tensors, int32_t n_workers,
@@ -1597,7 +1380,7 @@ adasum_status_t adasum_device_status(int64_t total_elems, int32_t num_tensors, i
     LevelPlan plan;
     if (!plan_levels(n_workers, dtype, flags, &plan))
         return fail(ADASUM_ERR_ARG, "invalid flags 0x%x", flags);
-    const Layout lay = make_layout(plan, total_elems, num_tensors);
+    const Layout lay = make_layout(plan, total_elems, num_tensors, n_workers);
     if (lay.counters_bytes < sizeof(int))
         return ADASUM_OK;
     int word = 0;
@@ -1699,24 +1482,16 @@ adasum_status_t adasum_shutdown(void)
         g_profiler.marks.clear();
         g_profiler.used = 0;
     }
-    std::lock_guard<std::mutex> lock(g_tables_mutex);
-    if (g_tables.empty())
-        return ADASUM_OK;
-    int current = 0;
-    cudaError_t err = cudaGetDevice(&current);
-    bool ok = err == cudaSuccess;
-    for (auto& tab : g_tables) {
-        if (ok && cudaSetDevice(tab->device) == cudaSuccess) {
-            if (cudaFree(tab->d_segments) != cudaSuccess || cudaFree(tab->d_seg_first) != cudaSuccess)
-                ok = false;
-        } else {
-            ok = false;
-        }
+    std::vector<std::shared_ptr<SegmentTable>> dropped;
+    {
+        std::lock_guard<std::mutex> lock(g_tables_mutex);
+        dropped.swap(g_tables);
     }
-    g_tables.clear();
-    if (err == cudaSuccess)
-        cudaSetDevice(current);
-    return ok ? ADASUM_OK : fail(ADASUM_ERR_CUDA, "adasum_shutdown: a CUDA call failed");
+    if (dropped.empty())
+        return ADASUM_OK;       // nothing to free: no CUDA call (the library may be loaded without a GPU)
+    dropped.clear();            // frees the device arrays (cudaFree waits for the kernels that read them)
+    const cudaError_t err = cudaGetLastError();
+    return err == cudaSuccess ? ADASUM_OK : fail(ADASUM_ERR_CUDA, "adasum_shutdown: %s", cudaGetErrorString(err));
 }
 
 }  // extern "C"

@@ -85,3 +85,41 @@ def test_element_shards_cover_every_tensor_once():
                 assert int(local_offsets[t + 1] - local_offsets[t]) == hi - lo
                 cursor = hi
             assert cursor == int(offsets[t + 1])
+
+
+def _sharded_rank_main(rank, world, port, results):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    spec = workloads.SPECS["c2"]
+    local = torch.tensor(bench.sharded_local_sizes(spec, world, rank), dtype=torch.int64)
+    summed = local.clone()
+    dist.all_reduce(summed, op=dist.ReduceOp.SUM)             # the ranks' slices add up to every tensor
+    # strong scaling: the job is the whole configuration, the step time the slowest rank's
+    ms, _ = bench.aggregate_over_ranks(3.0 + rank, 0.0, world, "cpu")
+    results[rank] = (summed.tolist(), int(local.sum()), ms)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_sharded_mode_slices_and_aggregates_over_two_ranks():
+    world = 2
+    with mp.Manager() as manager:
+        results = manager.dict()
+        mp.spawn(_sharded_rank_main, args=(world, 29655, results), nprocs=world, join=True)
+        sizes = workloads.SPECS["c2"].tensor_sizes()
+        assert results[0][0] == results[1][0] == sizes
+        assert results[0][1] + results[1][1] == sum(sizes)
+        assert results[0][1] >= results[1][1] > 0.4 * sum(sizes)      # balanced up to the 64-element grid
+        assert results[0][2] == results[1][2] == 4.0
+
+
+def test_allreduce_bytes_per_level():
+    levels = [{"radix": 16, "operands": 256, "groups": 16}, {"radix": 16, "operands": 16, "groups": 1}]
+    assert bench.allreduce_bytes_per_level(161, levels) == [161 * 16 * 136 * 8, 161 * 136 * 8]
+
+
+def test_whole_reduce_summary_gives_both_readings():
+    s = bench.whole_reduce_summary(64, 1000, 2, 1.0, 6000.0)
+    assert s["one_read_bytes"] == 64 * 1000 * 2 + 4000 and s["two_read_bytes"] == 2 * 64 * 1000 * 2 + 4000
+    assert abs(s["one_read_roofline_frac_measured_peak"] - s["one_read_bytes"] / 1e-3 / 1e9 / 6000.0) < 1e-12
+    assert s["two_read_roofline_frac_measured_peak"] > s["one_read_roofline_frac_measured_peak"]

@@ -44,13 +44,13 @@ def _case(n, total, dtype, step, seed):
     return start, currents
 
 
-def _check(got, ref, ref_start, offsets, dtype, out_dtype, min_len=32):
+def _check(got, ref, ref_start, offsets, dtype, out_dtype):
     got = got.double().cpu().numpy()
     assert np.all(np.isfinite(got))
     for t in range(len(offsets) - 1):
         lo, hi = int(offsets[t]), int(offsets[t + 1])
-        if hi - lo < min_len:
-            continue            # very short tensors: covered by the condition-aware check of the main suite
+        if hi == lo:
+            continue
         r = ref[lo:hi] - ref_start[lo:hi]
         bound = TOL[dtype] * np.linalg.norm(r) + EPS_OUT[out_dtype] * np.linalg.norm(ref[lo:hi])
         assert np.linalg.norm(got[lo:hi] - ref[lo:hi]) <= bound, (t, np.linalg.norm(got[lo:hi] - ref[lo:hi]), bound)
@@ -127,8 +127,8 @@ def test_orthogonality_is_that_of_the_effective_gradients(lib):
     _, ref = oracle.adasum_reduce_delta([_np(c, "f32") for c in currents], _np(start, "f32"), offsets=OFFSETS,
                                         dtype="f32", return_orthogonality=True, threads=0)
     for t in range(len(OFFSETS) - 1):
-        if OFFSETS[t + 1] - OFFSETS[t] >= 32:
-            assert abs(float(ortho[t]) - ref[t]) <= 1e-4 * ref[t]
+        if OFFSETS[t + 1] > OFFSETS[t]:
+            assert abs(float(ortho[t]) - ref[t]) <= 1e-4 * ref[t], (t, float(ortho[t]), ref[t])
 
 
 def test_arguments_are_checked(lib):
@@ -160,4 +160,4 @@ def test_c2_full_size_every_tensor(lib):
     torch.cuda.synchronize()
     ref = oracle.adasum_reduce_delta([_np(c, "f32") for c in currents], _np(start, "f32"), offsets=wl.offsets,
                                      dtype="f32", threads=0)
-    _check(out, ref, start.double().cpu().numpy(), wl.offsets, "f32", "f32", min_len=65)
+    _check(out, ref, start.double().cpu().numpy(), wl.offsets, "f32", "f32")

@@ -56,7 +56,8 @@ def _kernels(lib, fn):
     lib.adasum_profile_enable(256)
     out = fn()
     torch.cuda.synchronize()
-    return out, [r["kernel"] for r in lib.adasum_profile_collect(256)]
+    # the tensors of at most 64 elements have a kernel of their own, launched last; it is not what these tests count
+    return out, [r["kernel"] for r in lib.adasum_profile_collect(256) if r["kernel"] != "short_tensors"]
 
 
 @pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])

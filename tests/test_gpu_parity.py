@@ -10,7 +10,6 @@ import torch
 
 from oracle import adasum_oracle as oracle
 from paper_2006_02924_b200 import workloads
-from tree_algebra import leaf_weights_from_gram
 
 pytestmark = pytest.mark.gpu
 
@@ -35,14 +34,9 @@ def _oracle(grads, offsets, dtype):
                                 threads=0)
 
 
-def _compare(out: np.ndarray, ref: np.ndarray, offsets, tol: float, grads=None):
-    """Returns (global rel-L2, worst per-tensor rel-L2); asserts both against tol.
-
-    With `grads` given, SHORT tensors (<= 64 elements) that miss tol are re-judged against
-    tol * kappa, kappa = sum_w |c_w| |g_w| / |ref| with c_w the exact fp64 leaf weights of the
-    tree: the result is the weighted sum of the leaves, so that is its condition number, and it is
-    large only when leaves cancel (one-element tensors of opposite sign).  Longer tensors and the
-    full-size benchmark configurations are always held to tol itself."""
+def _compare(out: np.ndarray, ref: np.ndarray, offsets, tol: float):
+    """Returns (global rel-L2, worst per-tensor rel-L2); asserts both against tol, for every tensor
+    whatever its length."""
     out = out.astype(np.float64)
     assert np.all(np.isfinite(out))
     worst = 0.0
@@ -56,29 +50,22 @@ def _compare(out: np.ndarray, ref: np.ndarray, offsets, tol: float, grads=None):
             assert not np.any(o), f"tensor {t}: reference is exactly zero, output is not"
             continue
         err = np.linalg.norm(o - r) / nr
-        bound = tol
-        if err > tol and grads is not None and hi - lo <= 64:
-            leaves = np.stack([g[lo:hi].double().cpu().numpy() for g in grads])
-            c = leaf_weights_from_gram(leaves @ leaves.T)
-            kappa = float(np.sum(np.abs(c) * np.linalg.norm(leaves, axis=1))) / nr
-            bound = tol * max(1.0, kappa)
-        assert err <= bound, f"tensor {t} (len {hi - lo}): rel-L2 {err:.3e} > {bound:.3e}"
-        if bound == tol:
-            worst = max(worst, err)
+        assert err <= tol, f"tensor {t} (len {hi - lo}): rel-L2 {err:.3e} > {tol:.3e}"
+        worst = max(worst, err)
     nr = np.linalg.norm(ref)
     glob = np.linalg.norm(out - ref) / nr if nr > 0 else 0.0
     assert glob <= tol, f"global rel-L2 {glob:.3e} > {tol}"
     return glob, worst
 
 
-def _run_and_check(lib, grads, offsets, dtype, flags=0, strict=False):
+def _run_and_check(lib, grads, offsets, dtype, flags=0):
     out = lib.adasum_reduce(grads, offsets, flags=flags)
     torch.cuda.synchronize()
     ref = _oracle(grads, offsets, dtype)
-    return _compare(out.cpu().numpy(), ref, offsets, TOL[dtype], grads=None if strict else grads)
+    return _compare(out.cpu().numpy(), ref, offsets, TOL[dtype])
 
 
-def _correlated(n, total, dtype, seed, rho=0.5, scale=1.0, device="cuda"):
+def _correlated(n, total, dtype, seed, rho=0.3, scale=1.0, device="cuda"):
     gen = torch.Generator(device=device)
     gen.manual_seed(seed)
     shared = torch.randn(total, generator=gen, device=device)
@@ -91,7 +78,7 @@ def _correlated(n, total, dtype, seed, rho=0.5, scale=1.0, device="cuda"):
 def test_c1_pair_one_million_fp32(lib):
     wl = workloads.generate("c1", device="cuda")
     assert wl.n_workers == 2 and wl.total_elems == 1_000_000
-    _run_and_check(lib, wl.grads, wl.offsets, "f32", strict=True)
+    _run_and_check(lib, wl.grads, wl.offsets, "f32")
     out = lib.adasum_pair(wl.grads[0], wl.grads[1])
     ref = _oracle(wl.grads, wl.offsets, "f32")
     _compare(out.cpu().numpy(), ref, wl.offsets, 1e-5)
@@ -248,7 +235,7 @@ def test_guard_bands_are_untouched(lib):
     torch.cuda.synchronize()
     assert bool((store[:pad] == 12345.0).all()) and bool((store[pad + total:] == 12345.0).all())
     assert bool((ws[:4096] == 0x5A).all()) and bool((ws[4096 + need:] == 0x5A).all())
-    _compare(out.cpu().numpy(), _oracle(grads, offsets, "f32"), offsets, 1e-5, grads=grads)
+    _compare(out.cpu().numpy(), _oracle(grads, offsets, "f32"), offsets, 1e-5)
 
 
 def test_too_small_workspace_is_rejected(lib):
@@ -275,7 +262,7 @@ def test_reduced_configurations(lib, name, divisor, n):
 def test_c2_full_size_every_tensor(lib):
     wl = workloads.generate("c2", device="cuda")
     assert wl.num_tensors == 161 and wl.total_elems == 25_557_032
-    glob, worst = _run_and_check(lib, wl.grads, wl.offsets, "f32", strict=True)
+    glob, worst = _run_and_check(lib, wl.grads, wl.offsets, "f32")
     print(f"c2 full: global {glob:.2e} worst tensor {worst:.2e}")
 
 
@@ -284,13 +271,14 @@ def test_c2_full_size_literal_tree(lib):
     level's combine is fused with the next level's dot products; and the same with separate kernels."""
     wl = workloads.generate("c2", device="cuda")
     for flags in (lib.flags_radix(2, 2), lib.flags_radix(2, 2) | lib.ADASUM_FLAG_NO_LEVEL_FUSION):
-        glob, worst = _run_and_check(lib, wl.grads, wl.offsets, "f32", flags=flags, strict=True)
+        glob, worst = _run_and_check(lib, wl.grads, wl.offsets, "f32", flags=flags)
         print(f"c2 full, literal tree (flags {flags:#x}): global {glob:.2e} worst tensor {worst:.2e}")
 
 
-def _sampled_tensor_check(lib, name, sample_count, max_len):
+def _sampled_tensor_check(lib, name, sample_count, max_len, also=()):
     """Full-size run in the launch configuration the benchmark uses; a sample of tensors (every
-    size class up to max_len elements, seeded choice) is reduced by the oracle and compared."""
+    size class up to max_len elements, seeded choice) and the tensors listed in `also` (the largest
+    ones: the embedding table and feed-forward matrices) are reduced by the oracle and compared."""
     spec = workloads.SPECS[name]
     wl = workloads.generate(spec, device="cuda")
     out = lib.adasum_reduce(wl.grads, wl.offsets)
@@ -303,21 +291,28 @@ def _sampled_tensor_check(lib, name, sample_count, max_len):
     chosen.add(int(eligible[np.argmax(sizes[eligible])]))      # the largest eligible tensor
     chosen.add(int(np.argmin(sizes)))                          # and the smallest
     chosen.update(int(t) for t in wl.zeroed if sizes[t] <= max_len)
-    worst = 0.0
-    for t in sorted(chosen):
-        lo, hi = int(wl.offsets[t]), int(wl.offsets[t + 1])
-        ref = _oracle([g[lo:hi] for g in wl.grads], [0, hi - lo], spec.dtype)
-        _, w = _compare(out[lo:hi].cpu().numpy(), ref, [0, hi - lo], TOL[spec.dtype])
-        worst = max(worst, w)
-    print(f"{name} full size: {len(chosen)} tensors checked, worst rel-L2 {worst:.2e}")
+    chosen.update(int(t) for t in also)
+    chosen = sorted(chosen, key=lambda t: -int(sizes[t]))      # longest first: the oracle's threads take whole tensors
+    # one oracle call over the chosen tensors packed side by side (its threads run across tensors)
+    packed_offsets = workloads.offsets_from_sizes([int(sizes[t]) for t in chosen])
+    packed = [torch.cat([g[int(wl.offsets[t]):int(wl.offsets[t + 1])] for t in chosen]) for g in wl.grads]
+    got = torch.cat([out[int(wl.offsets[t]):int(wl.offsets[t + 1])] for t in chosen]).cpu().numpy()
+    ref = _oracle(packed, packed_offsets, spec.dtype)
+    del packed
+    _, worst = _compare(got, ref, packed_offsets, TOL[spec.dtype])
+    share = float(sum(int(sizes[t]) for t in chosen)) / float(wl.total_elems)
+    print(f"{name} full size: {len(chosen)} tensors checked ({100 * share:.0f} % of the elements, largest "
+          f"{int(sizes[chosen[0]])}), worst rel-L2 {worst:.2e}")
 
 
+# BERT-Large list: tensor 0 is the word-embedding table (31,254,528 elements), 15 + 16 k / 17 + 16 k are
+# layer k's feed-forward matrices (4,194,304 elements each)
 def test_c3_full_size_sampled_tensors(lib):
-    _sampled_tensor_check(lib, "c3", sample_count=24, max_len=4_200_000)
+    _sampled_tensor_check(lib, "c3", sample_count=24, max_len=4_200_000, also=(0, 15, 17 + 16 * 23))
 
 
 def test_c4_full_size_sampled_tensors(lib):
-    _sampled_tensor_check(lib, "c4", sample_count=20, max_len=1_100_000)
+    _sampled_tensor_check(lib, "c4", sample_count=20, max_len=1_100_000, also=(0, 15, 17 + 16 * 11, 17 + 16 * 23))
 
 
 def test_c5_full_size_sampled_tensors(lib):

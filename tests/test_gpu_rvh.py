@@ -46,8 +46,8 @@ def test_emulated_ranks_match_the_oracle(dtype, size, tol):
         assert np.all(np.isfinite(got))
         for t in range(len(offsets) - 1):
             lo, hi = int(offsets[t]), int(offsets[t + 1])
-            if hi - lo < 32:
-                continue        # very short tensors: covered by the condition-aware check of the main suite
+            if hi == lo:
+                continue
             err = np.linalg.norm(got[lo:hi] - ref[lo:hi]) / np.linalg.norm(ref[lo:hi])
             assert err <= tol, (r, t, err)
         assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= tol

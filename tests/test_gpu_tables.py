@@ -1,0 +1,64 @@
+"""The cache of per-offset-table segment tables: a call keeps the tables it has looked up alive
+until its launches are enqueued, whatever else is dropped from the cache meanwhile."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import adasum_oracle as oracle
+from paper_2006_02924_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+SIMPLE = 1 << 16
+CACHE_TABLES = 256        # the library keeps at most this many tables
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2006_02924_b200 import binding
+
+    return binding
+
+
+def _inputs(n, total, seed):
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(seed)
+    shared = torch.randn(total, generator=gen, device="cuda")
+    return [0.55 * shared + 0.84 * torch.randn(total, generator=gen, device="cuda") for _ in range(n)]
+
+
+def test_a_call_survives_the_eviction_of_its_own_table(lib):
+    """Order that used to free a table in use: a call with the fp32-pipe kernels caches the short
+    segment length for X; a default call adds X's other lengths; other offset tables push the first
+    one to the front of the cache; the next call on X finds one of its tables and misses another,
+    which evicts the least recently used entry while the call is still holding tables."""
+    lib.adasum_shutdown()                                   # start from an empty cache
+    sizes_x = [70_000, 300, 9000, 129]
+    x_off = workloads.offsets_from_sizes(sizes_x)
+    grads = _inputs(16, int(x_off[-1]), seed=6000)
+    ref = oracle.adasum_reduce([g.cpu().numpy() for g in grads], offsets=x_off, dtype="f32", threads=0)
+
+    def check(out):
+        torch.cuda.synchronize()
+        got = out.double().cpu().numpy()
+        for t in range(len(sizes_x)):
+            lo, hi = int(x_off[t]), int(x_off[t + 1])
+            assert np.linalg.norm(got[lo:hi] - ref[lo:hi]) <= 1e-5 * np.linalg.norm(ref[lo:hi]), t
+
+    check(lib.adasum_reduce(grads, x_off, flags=SIMPLE))
+    check(lib.adasum_reduce(grads, x_off))
+    small = _inputs(2, 4096, seed=6001)
+    filler_ref = None
+    for k in range(CACHE_TABLES + 40):                      # each call adds at least one table
+        off = np.array([0, 100 + k, 4096], dtype=np.int64)
+        out = lib.adasum_reduce(small, off, flags=SIMPLE | (1 << 17))
+        if k == 0:
+            torch.cuda.synchronize()
+            filler_ref = oracle.adasum_reduce([g.cpu().numpy() for g in small], offsets=off, dtype="f32", threads=0)
+            assert np.linalg.norm(out.double().cpu().numpy() - filler_ref) <= 1e-5 * np.linalg.norm(filler_ref)
+        if k % 64 == 0:
+            check(lib.adasum_reduce(grads, x_off))          # hits and misses interleaved with the evictions
+    check(lib.adasum_reduce(grads, x_off))
+    check(lib.adasum_reduce(grads, x_off, flags=SIMPLE))
+    check(lib.adasum_reduce(grads, x_off, flags=2 | (2 << 8)))
+    lib.adasum_shutdown()
+    check(lib.adasum_reduce(grads, x_off))                  # and everything is rebuilt after a shutdown
