@@ -162,6 +162,11 @@ def generate(spec: WorkloadSpec | str, device="cpu", tensor_sizes=None, n_worker
     shared.mul_(shared_scale)
     del shared_scale
 
+    # The N worker buffers are the rows of one [N, pitch] allocation, pitch = the buffer length rounded
+    # up to 64 elements (what stacking the workers' fused buffers gives); each is handed out as a
+    # separate one-dimensional view.
+    pitch = (total + 63) // 64 * 64
+    store = torch.zeros((spec.n_workers, max(pitch, 1)), dtype=TORCH_DTYPES[spec.dtype], device=device)
     grads = []
     for w in range(spec.n_workers):
         gen.manual_seed(seed + 1 + w)
@@ -170,7 +175,8 @@ def generate(spec: WorkloadSpec | str, device="cpu", tensor_sizes=None, n_worker
         for t, workers in zeroed.items():
             if w in workers:
                 g[int(offsets[t]):int(offsets[t + 1])] = 0.0
-        grads.append(g.to(TORCH_DTYPES[spec.dtype]))
+        store[w, :total].copy_(g)
+        grads.append(store[w, :total])
         del g
     return Workload(spec, grads, offsets, rho, sigma, zeroed)
 

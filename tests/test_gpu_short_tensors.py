@@ -93,8 +93,8 @@ def test_cancelling_short_tensors(lib, dtype, n):
     ref = oracle.adasum_reduce([_np(g, dtype) for g in grads], offsets=offsets, dtype=dtype, threads=0)
     # the inputs do cancel: some short tensor's result is far smaller than its leaves
     lo, hi = int(offsets[0]), int(offsets[1])
-    if n & (n - 1) == 0:
-        assert np.linalg.norm(ref[lo:hi]) < 0.2 * float(grads[0][lo:hi].double().norm())
+    if dtype == "f32" and n & (n - 1) == 0:
+        assert np.linalg.norm(ref[lo:hi]) < 0.05 * float(grads[0][lo:hi].double().norm())
     out = lib.adasum_reduce(grads, offsets)
     torch.cuda.synchronize()
     _check(out, ref, offsets, TOL[dtype])
