@@ -129,14 +129,7 @@ typedef enum {
  *                (Algorithm 1's "apply" of one level and its dot products of the next), so the
  *                intermediate vectors are read once less.  Same results up to rounding; for
  *                comparison and debugging.
- *   bit 22       ADASUM_FLAG_NO_BULK_COPIES: when the workers' fp16 / bf16 buffers are rows of one
- *                allocation (grads[w] = grads[0] + w * pitch bytes, pitch a multiple of 16), the
- *                radix-64 tensor-memory kernel reads them through a two-dimensional tensor map with
- *                bulk tensor copies (one instruction per 64 rows x 128 bytes) instead of 16-byte
- *                asynchronous copies.  The flag keeps the 16-byte copies.  Same results bit for bit;
- *                for comparison and debugging.
  */
-#define ADASUM_FLAG_NO_BULK_COPIES (1u << 22)
 #define ADASUM_FLAG_NO_LEVEL_FUSION (1u << 21)
 #define ADASUM_FLAG_NO_TCGEN05 (1u << 19)
 #define ADASUM_FLAG_TOP_DOWN_HALVES (1u << 20)

