@@ -129,7 +129,15 @@ typedef enum {
  *                (Algorithm 1's "apply" of one level and its dot products of the next), so the
  *                intermediate vectors are read once less.  Same results up to rounding; for
  *                comparison and debugging.
+ *   bit 22       ADASUM_FLAG_SELFTEST_TIMEOUT: a self-test of the device status path, not a way to
+ *                reduce.  The radix-64 tensor-memory kernel leaves every segment's last tile
+ *                unmultiplied, so nothing ever releases that tile's stage, and waits for the release
+ *                with a limit of microseconds instead of the usual tenth of a second.  The wait runs
+ *                out, the kernel records it, frees its tensor memory and returns; the output is
+ *                wrong by construction and adasum_device_status reports ADASUM_ERR_TIMEOUT.  No other
+ *                kernel looks at the flag.
  */
+#define ADASUM_FLAG_SELFTEST_TIMEOUT (1u << 22)
 #define ADASUM_FLAG_NO_LEVEL_FUSION (1u << 21)
 #define ADASUM_FLAG_NO_TCGEN05 (1u << 19)
 #define ADASUM_FLAG_TOP_DOWN_HALVES (1u << 20)

@@ -27,6 +27,7 @@ ADASUM_FLAG_SIMPLE_KERNELS, ADASUM_FLAG_SEPARATE_FINISH, ADASUM_FLAG_LINEAR_ORDE
 ADASUM_FLAG_NO_TCGEN05 = 1 << 19
 ADASUM_FLAG_TOP_DOWN_HALVES = 1 << 20
 ADASUM_FLAG_NO_LEVEL_FUSION = 1 << 21
+ADASUM_FLAG_SELFTEST_TIMEOUT = 1 << 22
 ADASUM_OK = 0
 ADASUM_MAX_WORKERS = 4096
 ADASUM_MAX_LEVELS = 12

@@ -139,7 +139,7 @@ int tree_order(int n_workers, uint32_t flags)
 bool plan_levels(int n_workers, adasum_dtype_t dtype, uint32_t flags, LevelPlan* plan)
 {
     const int first = (int)(flags & 0xffu), later_flag = (int)((flags >> 8) & 0xffu);
-    if ((flags >> 22) != 0)
+    if ((flags >> 23) != 0)
         return false;
     if ((flags & ADASUM_FLAG_LINEAR_ORDER) && (flags & ADASUM_FLAG_TOP_DOWN_HALVES))
         return false;
@@ -731,6 +731,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
             fin.seg_first = tab->d_seg_first;
             fin.counters = nullptr;
             fin.weights = nullptr;
+            fin.selftest_timeout = 0;
             fin.tree = TreeOptions{tree_order(n_workers, flags), 1, 1, 1,
                                    orthogonality ? reinterpret_cast<double*>(ws + lay.leaf_sums) : nullptr,
                                    orthogonality};
@@ -795,6 +796,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         a.tc_status = (flags & ADASUM_FLAG_NO_TCGEN05)
                           ? nullptr
                           : reinterpret_cast<int*>(ws + lay.counters + lay.counters_bytes - sizeof(int));
+        a.selftest_timeout = (flags & ADASUM_FLAG_SELFTEST_TIMEOUT) != 0;
         a.tree.linear = tree_order(n_workers, flags);
         a.tree.level_is_first = l == 0;
         a.tree.level_is_last = l + 1 == plan.num_levels;
@@ -860,7 +862,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
 bool plan_levels_f64(int n_workers, uint32_t flags, LevelPlan* plan)
 {
     const int first = (int)(flags & 0xffu), later_flag = (int)((flags >> 8) & 0xffu);
-    if ((flags >> 22) != 0)
+    if ((flags >> 23) != 0)
         return false;
     if (flags & (ADASUM_FLAG_LINEAR_ORDER | ADASUM_FLAG_TOP_DOWN_HALVES | ADASUM_FLAG_SEPARATE_FINISH |
                  ADASUM_FLAG_SIMPLE_KERNELS))

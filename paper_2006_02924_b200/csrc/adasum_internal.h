@@ -140,6 +140,7 @@ struct LevelArgs {
     TreeOptions tree;
     LevelPhase phase;
     int* tc_status;     // status word for the tcgen05 kernel, or nullptr to keep to mma.sync
+    bool selftest_timeout;   // ADASUM_FLAG_SELFTEST_TIMEOUT
     double* gram64;
     float* weights;
     void* dst;

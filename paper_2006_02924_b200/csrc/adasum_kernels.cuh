@@ -350,6 +350,8 @@ struct FinishArgs {
     int* counters;              // [tensor][group], zero on entry
     float* weights;             // [tensor][group][R]
     TreeOptions tree;
+    int selftest_timeout;       // gram_partial_tc64_kernel only: leave the last tile unmultiplied and wait briefly,
+                                // so that the epilogue's bounded wait runs out (test of the status path)
 };
 
 template <int R>
@@ -973,6 +975,7 @@ constexpr int kTcTileBytes = kTcKBlocks * 8192;
 constexpr int kTcPadBytes = 8 * 1024;         // slack after the last stage
 constexpr size_t kTcSmemBytes = (size_t)kTcStages * kTcTileBytes + kTcPadBytes + 1024;   // + room to align to 1024
 constexpr uint32_t kTcSpinLimit = 1u << 22;   // about a tenth of a second; a real wait is microseconds
+constexpr uint32_t kTcSelftestSpinLimit = 1u << 14;   // the self-test's wait: long after every issued multiplication is done
 
 __device__ __forceinline__ uint32_t mbarrier_try_wait_parity(uint32_t bar, uint32_t parity)
 {
@@ -985,9 +988,9 @@ __device__ __forceinline__ uint32_t mbarrier_try_wait_parity(uint32_t bar, uint3
 }
 
 // Returns false if the barrier did not complete the phase within the spin limit.
-__device__ __forceinline__ bool mbarrier_wait_bounded(uint32_t bar, uint32_t parity)
+__device__ __forceinline__ bool mbarrier_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit = kTcSpinLimit)
 {
-    for (uint32_t spin = 0; spin < kTcSpinLimit; ++spin)
+    for (uint32_t spin = 0; spin < limit; ++spin)
         if (mbarrier_try_wait_parity(bar, parity))
             return true;
     return false;
@@ -1117,6 +1120,8 @@ gram_partial_tc64_kernel(const __grid_constant__ OperandTable ops, int operands,
         constexpr uint32_t kInstr =
             (1u << 4) | (kFormat << 7) | (kFormat << 10) | ((64u >> 3) << 17) | ((64u >> 4) << 24);
         for (int tile = 0; tile < ntiles; ++tile) {
+            if (fin.selftest_timeout && tile == ntiles - 1)
+                break;          // self-test: nothing arrives on this tile's `empty` barrier
             const int stage = tile % kTcStages;
             if (!timed_out && !mbarrier_wait_bounded(full0 + 8 * stage, (uint32_t)((tile / kTcStages) & 1)))
                 timed_out = true;
@@ -1146,7 +1151,8 @@ gram_partial_tc64_kernel(const __grid_constant__ OperandTable ops, int operands,
     {
         const int last = ntiles - 1;
         if (!timed_out &&
-            !mbarrier_wait_bounded(empty0 + 8 * (last % kTcStages), (uint32_t)((last / kTcStages) & 1)))
+            !mbarrier_wait_bounded(empty0 + 8 * (last % kTcStages), (uint32_t)((last / kTcStages) & 1),
+                                   fin.selftest_timeout ? kTcSelftestSpinLimit : kTcSpinLimit))
             timed_out = true;
     }
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");

@@ -201,7 +201,8 @@ adasum_status_t run_level_typed(const LevelArgs& a)
     constexpr int kGroupsPerLaunch = kMaxOperandsPerLaunch / R;
     // the last block of every (tensor, group) in pass 1 also derives the weights
     const bool fused_finish = a.counters != nullptr && a.phase == PHASE_WHOLE;
-    const FinishArgs fin{a.gram_tab->d_seg_first, fused_finish ? a.counters : nullptr, a.weights, a.tree};
+    const FinishArgs fin{a.gram_tab->d_seg_first, fused_finish ? a.counters : nullptr, a.weights, a.tree,
+                         a.selftest_timeout ? 1 : 0};
     // pass 1
     for (int g0 = 0; g0 < a.groups && a.phase != PHASE_APPLY && !a.skip_gram; g0 += kGroupsPerLaunch) {
         const int groups_here = a.groups - g0 < kGroupsPerLaunch ? a.groups - g0 : kGroupsPerLaunch;

@@ -117,7 +117,7 @@ def test_argument_errors_are_caught_on_the_host(binding):
     assert s(_call_reduce(binding, good, [1, 8], 2)) == "ADASUM_ERR_OFFSETS"
     assert s(_call_reduce(binding, good, [0, 8, 4], 2)) == "ADASUM_ERR_OFFSETS"
     assert s(_call_reduce(binding, good, [0, 8], 2, flags=3)) == "ADASUM_ERR_ARG"
-    assert s(_call_reduce(binding, good, [0, 8], 2, flags=1 << 22)) == "ADASUM_ERR_ARG"
+    assert s(_call_reduce(binding, good, [0, 8], 2, flags=1 << 23)) == "ADASUM_ERR_ARG"
     assert s(_call_reduce(binding, good, [0, 8], 2, flags=64)) == "ADASUM_ERR_ARG"        # radix 64 needs 16-bit inputs
     assert s(_call_reduce(binding, [0x30000000, 0], [0, 8], 2)) == "ADASUM_ERR_NULL"
     assert s(_call_reduce(binding, good, [0, 8], 2, out=0)) == "ADASUM_ERR_NULL"

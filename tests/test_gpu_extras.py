@@ -199,6 +199,30 @@ def test_radix_64_tensor_memory_kernel(lib, dtype, n):
     assert float(torch.linalg.norm(out - other) / torch.linalg.norm(other)) <= 1e-4
 
 
+def test_a_bounded_wait_that_runs_out_is_reported_and_leaves_the_gpu_usable(lib):
+    """The radix-64 tensor-memory kernel bounds every wait on the tensor core.  With the self-test flag
+    it leaves each segment's last tile unmultiplied, so the epilogue's wait for that tile (limit:
+    microseconds) runs out with no multiplication outstanding; the kernel records it, frees its tensor
+    memory and returns.  The host reads ADASUM_ERR_TIMEOUT, and the next ordinary reduce on the same
+    workspace is correct and reads status 0."""
+    offsets = workloads.offsets_from_sizes([20_000, 513, 6000])
+    total = int(offsets[-1])
+    grads = _correlated(64, total, "f16", seed=1800)
+    flags = lib.flags_radix(64, 0)
+    ws = torch.empty(lib.adasum_workspace_bytes(total, 3, 64, "f16", flags), dtype=torch.uint8, device="cuda")
+    good = lib.adasum_reduce(grads, offsets, workspace=ws, flags=flags).clone()
+    assert lib.adasum_device_status(total, 3, 64, "f16", ws, flags=flags) == 0
+    lib.adasum_reduce(grads, offsets, workspace=ws, flags=flags | lib.ADASUM_FLAG_SELFTEST_TIMEOUT)
+    assert lib.adasum_device_status(total, 3, 64, "f16", ws, flags=flags | lib.ADASUM_FLAG_SELFTEST_TIMEOUT) == 7
+    assert "bounded wait" in lib.adasum_last_error()
+    again = lib.adasum_reduce(grads, offsets, workspace=ws, flags=flags)
+    assert lib.adasum_device_status(total, 3, 64, "f16", ws, flags=flags) == 0
+    torch.cuda.synchronize()
+    assert torch.equal(again, good)
+    ref = oracle.adasum_reduce([_np(g, "f16") for g in grads], offsets=offsets, dtype="f16", threads=0)
+    assert np.linalg.norm(again.cpu().numpy() - ref) <= 2e-3 * np.linalg.norm(ref)
+
+
 def _stacked(n, total, dtype, seed, pad=0, rho=0.4):
     """Worker buffers that are rows of one [n, total + pad] allocation (a uniform pitch between them)."""
     gen = torch.Generator(device="cuda")
