@@ -295,18 +295,27 @@ constexpr size_t kMaxCachedTableBytes = size_t(256) << 20;
 size_t table_device_bytes(const SegmentTable& tab)
 {
     return sizeof(Segment) * (tab.h_segments.size() + 1) + sizeof(int32_t) * tab.h_seg_first.size() +
-           sizeof(ShortTensor) * (tab.h_short.size() + 1);
+           sizeof(ShortTensor) * (tab.h_short.size() + 1) + sizeof(WarpTensor) * (tab.h_warp.size() + 1);
 }
 
 // Segments are listed tensor by tensor, LARGEST tensor first (ties in index order): the blocks of
 // pass 1 that run last then belong to small tensors, whose per-tensor finish (adding the partial
 // matrices, tree weights) is short, instead of leaving one SM busy with a long tensor's finish
 // while the rest of the GPU idles.  Each tensor's segments stay contiguous, in element order.
-void build_segments(const int64_t* offsets, int32_t num_tensors, int seg_len, bool skip_short, SegmentTable* tab)
+void build_segments(const int64_t* offsets, int32_t num_tensors, int seg_len, bool skip_short, int warp_limit,
+                    SegmentTable* tab)
 {
     tab->skip_short = skip_short;
+    tab->warp_limit = warp_limit;
     tab->h_short.clear();
+    tab->h_warp.clear();
     tab->short_elems = 0;
+    const int64_t short_limit = skip_short ? kShortTensorElems : 0;
+    for (int32_t t = 0; t < num_tensors && warp_limit > 0; ++t) {
+        const int64_t len = offsets[t + 1] - offsets[t];
+        if (len > short_limit && len <= warp_limit)
+            tab->h_warp.push_back(WarpTensor{offsets[t], (int32_t)len, t});
+    }
     if (skip_short) {
         for (int32_t t = 0; t < num_tensors; ++t) {
             const int64_t len = offsets[t + 1] - offsets[t];
@@ -330,7 +339,7 @@ void build_segments(const int64_t* offsets, int32_t num_tensors, int seg_len, bo
         tab->h_seg_first[2 * (size_t)t] = (int32_t)tab->h_segments.size();
         int64_t b = offsets[t];
         const int64_t e = offsets[t + 1];
-        if (skip_short && e - b <= kShortTensorElems)
+        if ((skip_short && e - b <= kShortTensorElems) || e - b <= warp_limit)
             b = e;
         while (b < e) {
             // cut on a 64-element grid of the fused buffer so that interior cuts keep 16-byte
@@ -352,7 +361,7 @@ void build_segments(const int64_t* offsets, int32_t num_tensors, int seg_len, bo
 // The table for (current device, offsets, seg_len), built and uploaded on first use.  The caller
 // keeps the returned reference until it has enqueued its last launch that reads the table.
 adasum_status_t get_segment_table(const int64_t* offsets, int32_t num_tensors, int seg_len, bool skip_short,
-                                  TableRef* out)
+                                  TableRef* out, int warp_limit = 0)
 {
     int device = 0;
     ADASUM_CUDA_CHECK(cudaGetDevice(&device));
@@ -361,6 +370,7 @@ adasum_status_t get_segment_table(const int64_t* offsets, int32_t num_tensors, i
     for (size_t i = 0; i < g_tables.size(); ++i) {
         const SegmentTable& tab = *g_tables[i];
         if (tab.device == device && tab.seg_len == seg_len && tab.skip_short == skip_short &&
+            tab.warp_limit == warp_limit &&
             tab.offsets.size() == (size_t)num_tensors + 1 &&
             std::memcmp(tab.offsets.data(), offsets, sizeof(int64_t) * tab.offsets.size()) == 0) {
             // most recently used last
@@ -373,10 +383,11 @@ adasum_status_t get_segment_table(const int64_t* offsets, int32_t num_tensors, i
     tab->device = device;
     tab->seg_len = seg_len;
     tab->offsets.assign(offsets, offsets + num_tensors + 1);
-    build_segments(offsets, num_tensors, seg_len, skip_short, tab.get());
+    build_segments(offsets, num_tensors, seg_len, skip_short, warp_limit, tab.get());
     const size_t seg_bytes = sizeof(Segment) * (tab->h_segments.size() + 1);
     const size_t first_bytes = sizeof(int32_t) * tab->h_seg_first.size();
-    const size_t short_bytes = sizeof(ShortTensor) * (tab->h_short.size() + 1);
+    const size_t short_bytes = sizeof(ShortTensor) * (tab->h_short.size() + 1) +
+                               sizeof(WarpTensor) * (tab->h_warp.size() + 1);
     // Make room: least recently used tables leave the cache.  One that a call in flight still holds
     // lives on until that call lets go of it.
     size_t held = 0;
@@ -399,6 +410,12 @@ adasum_status_t get_segment_table(const int64_t* offsets, int32_t num_tensors, i
                          sizeof(Segment) * tab->h_segments.size(), cudaMemcpyHostToDevice);
     if (err == cudaSuccess)
         err = cudaMemcpy(tab->d_seg_first, tab->h_seg_first.data(), first_bytes, cudaMemcpyHostToDevice);
+    if (err == cudaSuccess && !tab->h_warp.empty()) {
+        err = cudaMalloc(&tab->d_warp, sizeof(WarpTensor) * tab->h_warp.size());
+        if (err == cudaSuccess)
+            err = cudaMemcpy(tab->d_warp, tab->h_warp.data(), sizeof(WarpTensor) * tab->h_warp.size(),
+                             cudaMemcpyHostToDevice);
+    }
     if (err == cudaSuccess && !tab->h_short.empty()) {
         err = cudaMalloc(&tab->d_short, short_bytes);
         if (err == cudaSuccess)
@@ -419,9 +436,11 @@ constexpr int kSmallBlocksPerSm = 2;                       // blocks per SM the 
 constexpr int kSmallSegmentGrain = 1024;
 
 // Host-only rule (no device query): is this reduce served by fused_small_kernel, and with which
-// segment length?  `blocks` is the number of blocks that can be resident at once.
-bool small_input_plan(const LevelPlan& plan, int64_t total, int32_t num_tensors, int n_workers, int elem_bytes,
-                      uint32_t flags, int blocks, int* seg_len)
+// segment length?  `blocks` is the number of blocks that can be resident at once; only the
+// `big_tensors` tensors of more than kWarpTensorElems elements (`big_elems` elements in all) are cut
+// into segments, one block each.
+bool small_input_plan(const LevelPlan& plan, int64_t total, int64_t big_tensors, int64_t big_elems, int n_workers,
+                      int elem_bytes, uint32_t flags, int blocks, int* seg_len)
 {
     if (plan.num_levels != 1 || plan.level[0].radix > 8 || plan.level[0].groups != 1)
         return false;
@@ -429,11 +448,11 @@ bool small_input_plan(const LevelPlan& plan, int64_t total, int32_t num_tensors,
         return false;
     if (total <= 0 || (int64_t)n_workers * total * elem_bytes > kSmallInputBytes)
         return false;
-    // every tensor ends with one ragged segment: budget for those first
-    const int64_t room = (int64_t)blocks - 2 * (int64_t)num_tensors;
+    // a tensor's first and last segments may be ragged: budget for those first
+    const int64_t room = (int64_t)blocks - 2 * big_tensors;
     if (room < 8)
         return false;
-    int64_t len = (total + room - 1) / room;
+    int64_t len = (big_elems + room - 1) / room;
     len = (len + kSmallSegmentGrain - 1) / kSmallSegmentGrain * kSmallSegmentGrain;
     if (len < 2048)
         len = 2048;
@@ -467,7 +486,8 @@ int launches_of(const LevelPlan& plan, int n_workers, uint32_t flags, int64_t to
     if (n_workers == 1)
         return 1;
     int seg_len = 0;        // on a B200: 148 SMs
-    if (small_input_plan(plan, total, num_tensors, n_workers, elem_bytes, flags, 148 * kSmallBlocksPerSm, &seg_len))
+    // without the offsets every tensor has to be taken for a long one
+    if (small_input_plan(plan, total, num_tensors, total, n_workers, elem_bytes, flags, 148 * kSmallBlocksPerSm, &seg_len))
         return 1;
     int n = 0;
     bool gram_done = false;      // by the previous level's pass 2 (16-byte aligned buffers assumed)
@@ -626,8 +646,16 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     // Inputs that fit the L2 are served by one cooperative launch that needs no ticket counters.
     int small_seg_len = 0;
     const int small_blocks = (sharded || total == 0 || num_tensors == 0) ? 0 : resident_small_blocks();
-    const bool small_candidate =
-        small_blocks > 0 && small_input_plan(plan, total, num_tensors, n_workers, eb, flags, small_blocks, &small_seg_len);
+    int64_t big_tensors = 0, big_elems = 0;       // tensors that the single-launch kernel would cut into segments
+    for (int32_t t = 0; t < num_tensors; ++t) {
+        const int64_t len = offsets[t + 1] - offsets[t];
+        if (len > kWarpTensorElems) {
+            ++big_tensors;
+            big_elems += len;
+        }
+    }
+    const bool small_candidate = small_blocks > 0 && small_input_plan(plan, total, big_tensors, big_elems, n_workers, eb,
+                                                                      flags, small_blocks, &small_seg_len);
     // the workspace arrives with unknown contents
     auto clear_counters = [&]() { return cudaMemsetAsync(ws + lay.counters, 0, lay.counters_bytes, stream); };
     if (lay.counters_bytes > 0 && phase != PHASE_APPLY && !small_candidate)
@@ -720,7 +748,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     if (small_candidate) {
         int* dev_status = reinterpret_cast<int*>(ws + lay.counters + lay.counters_bytes - sizeof(int));
         TableRef tab;
-        st = get_segment_table(offsets, num_tensors, small_seg_len, skip_short, &tab);
+        st = get_segment_table(offsets, num_tensors, small_seg_len, skip_short, &tab, kWarpTensorElems);
         if (st != ADASUM_OK)
             return st;
         if (tab->num_segments <= small_blocks) {
@@ -741,11 +769,11 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
             ex.start = start;
             cudaError_t err;
             if (dtype == ADASUM_F32)
-                err = launch_fused_small_any<float>(vec, radix, table, n_workers, *tab, partials, fin, out, ex, dev_status, stream);
+                err = launch_fused_small_any<float>(vec, radix, table, n_workers, *tab, small_blocks, partials, fin, out, ex, dev_status, stream);
             else if (dtype == ADASUM_F16)
-                err = launch_fused_small_any<__half>(vec, radix, table, n_workers, *tab, partials, fin, out, ex, dev_status, stream);
+                err = launch_fused_small_any<__half>(vec, radix, table, n_workers, *tab, small_blocks, partials, fin, out, ex, dev_status, stream);
             else
-                err = launch_fused_small_any<__nv_bfloat16>(vec, radix, table, n_workers, *tab, partials, fin, out, ex, dev_status, stream);
+                err = launch_fused_small_any<__nv_bfloat16>(vec, radix, table, n_workers, *tab, small_blocks, partials, fin, out, ex, dev_status, stream);
             if (err == cudaSuccess) {
                 profile_mark(stream, ADASUM_KERNEL_FUSED_SMALL, 0, radix, false);
                 return run_short();
@@ -1199,7 +1227,7 @@ adasum_status_t pair_noalloc_impl(const void* a, const void* b, const int64_t* o
     if (st != ADASUM_OK)
         return st;
     SegmentTable tab;                       // host-side only; its device pointers aim into the scratch
-    build_segments(offsets, num_tensors, kNoallocSegLen, true, &tab);      // short tensors apart, as in adasum_pair
+    build_segments(offsets, num_tensors, kNoallocSegLen, true, 0, &tab);      // short tensors apart, as in adasum_pair
     if ((int64_t)tab.num_segments > kNoallocMaxSegments)
         return fail(ADASUM_ERR_ARG, "segment table does not fit the static scratch");
     tab.d_segments = reinterpret_cast<Segment*>(scratch);

@@ -99,13 +99,18 @@ struct SegmentTable {
     ShortTensor* d_short = nullptr;
     int64_t short_elems = 0;
     std::vector<ShortTensor> h_short;
+    // Tensors of at most warp_limit elements (beyond the short ones), when the single-launch kernel
+    // gives each of them to one warp: no segments either.
+    int warp_limit = 0;
+    WarpTensor* d_warp = nullptr;
+    std::vector<WarpTensor> h_warp;
 
     SegmentTable() = default;
     SegmentTable(const SegmentTable&) = delete;
     SegmentTable& operator=(const SegmentTable&) = delete;
     ~SegmentTable()
     {
-        if (!owns_device_arrays || (!d_segments && !d_seg_first && !d_short))
+        if (!owns_device_arrays || (!d_segments && !d_seg_first && !d_short && !d_warp))
             return;
         int current = 0;
         const bool have_current = cudaGetDevice(&current) == cudaSuccess;
@@ -114,6 +119,7 @@ struct SegmentTable {
         cudaFree(d_segments);
         cudaFree(d_seg_first);
         cudaFree(d_short);
+        cudaFree(d_warp);
         if (have_current && current != device)
             cudaSetDevice(current);
     }
@@ -172,8 +178,9 @@ adasum_status_t run_level(int radix, const LevelArgs& a);
 // Both passes of a one-level reduce in one cooperative launch (fused_small_kernel), radix 2, 4 or 8.
 template <typename T>
 cudaError_t launch_fused_small_any(bool vec, int radix, const OperandTable& ops, int operands,
-                                   const SegmentTable& tab, float* partials, const FinishArgs& fin, void* out,
-                                   const PassExtras& ex, int* status, cudaStream_t stream);
+                                   const SegmentTable& tab, int resident_blocks, float* partials,
+                                   const FinishArgs& fin, void* out, const PassExtras& ex, int* status,
+                                   cudaStream_t stream);
 
 // The three launches of adasum_pair_noalloc (pass 1, coefficients, pass 2), nothing fused.
 template <typename T>

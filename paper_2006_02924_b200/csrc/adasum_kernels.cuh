@@ -1745,32 +1745,357 @@ wsum_gram_kernel(const __grid_constant__ OperandTable ops, int operands,
 
 // ---- both passes in one launch, for inputs that fit the L2 -------------------------------------
 //
-// One level, one group (n_workers <= 8), few enough segments that every block of the grid is
-// resident at the same time (cooperative launch).  Each block forms the Gram matrix of its
-// segment, the grid synchronises, each block adds up its tensor's partial matrices and derives
-// the weights for itself (the same numbers in every block of a tensor: fixed summation order),
-// and then writes the weighted sum of the segment it has just read, which the 126 MB L2 still
-// holds.  HBM sees the operands once.
-// grid = segments; block = kThreads; partials[segment * E + entry].
-template <typename T, int R, bool VEC, bool DELTA = false>
-__global__ void __launch_bounds__(kThreads, (sizeof(T) == 2 && R == 8) ? 2 : 3)
-fused_small_kernel(const __grid_constant__ OperandTable ops, int operands,
-                   const Segment* __restrict__ segments, float* __restrict__ partials, FinishArgs fin,
-                   void* out, PassExtras ex, int* __restrict__ status)
+// One level, one group (n_workers <= 8), one cooperative launch whose blocks are all resident.
+// HBM sees the operands once.  Work is dealt in two sizes:
+//
+//   - tensors of more than kWarpTensorElems elements are cut into segments, one per block.  A block
+//     forms the Gram matrix of its segment, the grid synchronises, each block adds up its tensor's
+//     partial matrices and derives the weights for itself (the same numbers in every block of a
+//     tensor: fixed summation order), and writes the weighted sum of its segment.  When the segment
+//     is short enough (a few 16-byte vectors per thread and row) the operands stay in registers
+//     across the grid barrier and the second pass loads nothing; otherwise it reads them again,
+//     out of the L2;
+//   - tensors of at most kWarpTensorElems elements (beyond the short ones that the fp64 kernel
+//     takes) are handled by one warp each, from the loads to the store, before the barrier: a fused
+//     buffer with hundreds of small tensors (biases, normalisation parameters) then needs neither a
+//     block nor a barrier per tensor.
+//
+// grid >= segments; block = kThreads; partials[segment * E + entry].
+
+constexpr int kWarpTensorElems = 2048;
+
+// A small tensor that one warp reduces: `begin`, `len` in the fused buffers; `tensor` its index.
+struct WarpTensor {
+    int64_t begin;
+    int32_t len;
+    int32_t tensor;
+};
+
+// The binary tree (or the other two orders of Section 3.4) evaluated on a packed R x R Gram matrix
+// by ONE thread, R <= 8: leaf weights w[0 .. members) and the squared norm of the result.  Same
+// recursion as tree_weights_from_gram.
+template <int R>
+__device__ void tree_weights_serial(const double* gram, int members, int order, double* w, double& root_norm)
+{
+    double norm[R];
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+        w[i] = 1.0;
+        norm[i] = i < members ? gram[gram_index(R, i, i)] : 0.0;
+    }
+    // a <- Adasum(a, b) for the nodes over leaves [lo, mid) and [mid, hi); norms kept at lo / mid
+    auto combine = [&](int lo, int mid, int hi) {
+        double dot = 0.0;
+        for (int i = lo; i < mid; ++i) {
+            double row = 0.0;
+            for (int k = mid; k < hi; ++k)
+                row += w[k] * gram[gram_index(R, i, k)];
+            dot += w[i] * row;
+        }
+        double ca, cb;
+        pair_coefficients(dot, norm[lo], norm[mid], ca, cb);
+        for (int i = lo; i < mid; ++i)
+            w[i] *= ca;
+        for (int k = mid; k < hi; ++k)
+            w[k] *= cb;
+        norm[lo] = ca * ca * norm[lo] + cb * cb * norm[mid] + 2.0 * ca * cb * dot;
+    };
+    if (order == 1) {
+        for (int k = 1; k < members; ++k)
+            combine(0, k, k + 1);
+    } else if (order == 2) {
+        int max_depth = 0;
+        while ((1 << max_depth) < members)
+            ++max_depth;
+        for (int depth = max_depth - 1; depth >= 0; --depth) {
+            for (int j = 0; j < (1 << depth); ++j) {
+                int lo = 0, hi = members;
+                bool alive = true;
+                for (int t = 0; t < depth && alive; ++t) {
+                    if (hi - lo < 2) {
+                        alive = false;
+                    } else {
+                        const int m = lo + (hi - lo) / 2;
+                        if ((j >> (depth - 1 - t)) & 1)
+                            lo = m;
+                        else
+                            hi = m;
+                    }
+                }
+                if (alive && hi - lo >= 2)
+                    combine(lo, lo + (hi - lo) / 2, hi);
+            }
+        }
+    } else {
+        for (int width = 1; width < members; width *= 2)
+            for (int left = 0; left + width < members; left += 2 * width)
+                combine(left, left + width, min(left + 2 * width, members));
+    }
+    root_norm = norm[0];
+}
+
+// Block reduction of per-thread Gram accumulators: warp shuffles, then the warps' sums in warp
+// order; entry k of the result goes to dst[k].  Ends without a barrier after the stores.
+template <int E>
+__device__ __forceinline__ void block_reduce_gram(const float (&acc)[E], float* __restrict__ dst)
+{
+    __shared__ float warp_sums[kWarps][E];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int k = 0; k < E; ++k) {
+        float s = acc[k];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1)
+            s += __shfl_xor_sync(0xffffffffu, s, d);
+        if (lane == 0)
+            warp_sums[warp][k] = s;
+    }
+    __syncthreads();
+    for (int k = threadIdx.x; k < E; k += kThreads) {
+        float s = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w)
+            s += warp_sums[w][k];
+        dst[k] = s;
+    }
+}
+
+// One small tensor, both passes, by one warp.  Element e of row i: ops.ptr[i][begin + e].
+template <typename T, int R, bool DELTA>
+__device__ void reduce_warp_tensor(const OperandTable& ops, int members, const WarpTensor& wt, const TreeOptions& opt,
+                                   void* out, const PassExtras& ex)
 {
     constexpr int E = gram_entries(R);
+    const int lane = threadIdx.x & 31;
+    const T* src[R];
+#pragma unroll
+    for (int i = 0; i < R; ++i)
+        src[i] = static_cast<const T*>(ops.ptr[i < members ? i : 0]) + wt.begin;
+    const T* start = static_cast<const T*>(ex.start) + wt.begin;
+    auto element = [&](int i, int e) -> float {
+        if constexpr (DELTA)
+            return delta_one(src[i], start, e);
+        else
+            return Element<T>::one(src[i] + e);
+    };
+    float acc[E];
+#pragma unroll
+    for (int k = 0; k < E; ++k)
+        acc[k] = 0.0f;
+#pragma unroll 2
+    for (int e = lane; e < wt.len; e += 32) {
+        float col[R];
+#pragma unroll
+        for (int i = 0; i < R; ++i)
+            col[i] = i < members ? element(i, e) : 0.0f;
+        gram_accumulate<R>(col, acc);
+    }
+    // the lanes' sums (at most 64 products each) are added in fp64; every lane ends with the same bits
+    double gram[E];
+#pragma unroll
+    for (int k = 0; k < E; ++k) {
+        double s = (double)acc[k];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1)
+            s += __shfl_xor_sync(0xffffffffu, s, d);
+        gram[k] = s;
+    }
+    double w64[R], root = 0.0;
+    tree_weights_serial<R>(gram, members, opt.linear, w64, root);
+    if (lane == 0 && opt.orthogonality != nullptr) {
+        double leaf_sum = 0.0;
+        for (int i = 0; i < members; ++i)
+            leaf_sum += gram[gram_index(R, i, i)];
+        opt.orthogonality[wt.tensor] = leaf_sum == 0.0 ? __int_as_float(0x7fc00000) : (float)(root / leaf_sum);
+    }
+    float w[R];
+#pragma unroll
+    for (int i = 0; i < R; ++i)
+        w[i] = i < members ? (float)w64[i] : 0.0f;
+#pragma unroll 2
+    for (int e = lane; e < wt.len; e += 32) {
+        float y = 0.0f;
+#pragma unroll
+        for (int i = 0; i < R; ++i)
+            if (i < members)
+                y = fmaf(w[i], element(i, e), y);
+        if (ex.base != nullptr)
+            y += load_as_float(ex.base, ex.base_dtype, wt.begin + e);
+        store_from_float(out, ex.out_dtype, wt.begin + e, y);
+    }
+}
+
+// The partial matrices of segments [seg_begin, seg_end) added in fp64 in a fixed order by the whole
+// block, then the tree: leaf weights to weights_dst (shared memory), by-products as opt says.
+// Thread (q, kk) adds the partials of segments q, q + Q, ... for entry kk; a warp then adds the Q
+// slice sums of an entry (lane-strided, then a butterfly).
+template <int R>
+__device__ void finish_small(const float* partials, int seg_begin, int seg_end, int tensor, int members,
+                             float* weights_dst, const TreeOptions& opt)
+{
+    constexpr int E = gram_entries(R);
+    constexpr int Q = kThreads / E;
+    static_assert(E <= kThreads, "one thread per entry at least");
+    __shared__ double slice_sum[E * Q];
+    __shared__ double gram[E];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int q = threadIdx.x / E, kk = threadIdx.x - q * E;
+    if (q < Q) {
+        double s = 0.0;
+#pragma unroll 4
+        for (int seg = seg_begin + q; seg < seg_end; seg += Q)
+            s += (double)__ldcg(partials + (int64_t)seg * E + kk);
+        slice_sum[kk * Q + q] = s;
+    }
+    __syncthreads();
+    for (int k = warp; k < E; k += kWarps) {
+        double s = 0.0;
+        for (int qq = lane; qq < Q; qq += 32)
+            s += slice_sum[k * Q + qq];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1)
+            s += __shfl_xor_sync(0xffffffffu, s, d);
+        if (lane == 0)
+            gram[k] = s;
+    }
+    __syncthreads();
+    if constexpr (R <= 4) {
+        if (threadIdx.x == 0) {
+            double w64[R], root = 0.0;
+            tree_weights_serial<R>(gram, members, opt.linear, w64, root);
+            for (int i = 0; i < R; ++i)
+                weights_dst[i] = i < members ? (float)w64[i] : 0.0f;
+            if (opt.orthogonality != nullptr) {
+                double leaf_sum = 0.0;
+                for (int i = 0; i < members; ++i)
+                    leaf_sum += gram[gram_index(R, i, i)];
+                opt.orthogonality[tensor] = leaf_sum == 0.0 ? __int_as_float(0x7fc00000) : (float)(root / leaf_sum);
+            }
+        }
+    } else {
+        tree_weights_from_gram<R>(gram, members, weights_dst, opt, tensor, 0);
+    }
+    __syncthreads();
+}
+
+// 16-byte vectors per thread and row that stay in registers between the passes.
+template <int R>
+__host__ __device__ constexpr int small_keep_vectors() { return R <= 2 ? 4 : (R <= 4 ? 2 : 0); }
+
+template <typename T, int R, bool VEC, bool DELTA = false>
+__global__ void __launch_bounds__(kThreads, 2)
+fused_small_kernel(const __grid_constant__ OperandTable ops, int operands,
+                   const Segment* __restrict__ segments, int num_segments,
+                   const WarpTensor* __restrict__ warp_tensors, int num_warp_tensors,
+                   float* __restrict__ partials, FinishArgs fin, void* out, PassExtras ex, int* __restrict__ status)
+{
+    constexpr int E = gram_entries(R);
+    constexpr int V = Element<T>::kVec;
+    constexpr int K = small_keep_vectors<R>();
     // This path uses no ticket counters, so the host does not clear them (one operation less in
     // front of a reduce that takes microseconds); the device status word, which lives beside
     // them and which adasum_device_status reads, is cleared here instead.
     if (blockIdx.x == 0 && threadIdx.x == 0)
         *status = 0;
-    const Segment seg = segments[blockIdx.x];
     const int members = min(R, operands);
-    gram_of_segment<T, R, VEC, DELTA>(ops, 0, members, seg, partials + (int64_t)blockIdx.x * E,
-                                      static_cast<const T*>(ex.start));
+    const bool has_segment = (int)blockIdx.x < num_segments;
+    const Segment seg = has_segment ? segments[blockIdx.x] : Segment{0, 0, 0};
+    const int64_t begin = seg.begin, end = seg.begin + seg.len;
+    int64_t body_begin, body_end;
+    split_segment<V, VEC>(begin, end, body_begin, body_end);
+    const bool keep = K > 0 && VEC && has_segment && (body_end - body_begin) <= (int64_t)K * kThreads * V;
+
+    // ---- pass 1 of this block's segment
+    uint4 raw[R][K > 0 ? K : 1];
+    if (keep) {
+        const T* src[R];
+#pragma unroll
+        for (int i = 0; i < R; ++i)
+            src[i] = static_cast<const T*>(ops.ptr[i < members ? i : 0]);
+        // every load of the segment is issued before the first use
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            const int64_t v = body_begin + ((int64_t)threadIdx.x + (int64_t)k * kThreads) * V;
+            if (v < body_end) {
+#pragma unroll
+                for (int i = 0; i < R; ++i)
+                    raw[i][k] = i < members ? load_keep_16B(src[i] + v) : make_uint4(0u, 0u, 0u, 0u);
+            } else {
+#pragma unroll
+                for (int i = 0; i < R; ++i)
+                    raw[i][k] = make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
+        if constexpr (DELTA) {
+#pragma unroll
+            for (int k = 0; k < K; ++k) {
+                const int64_t v = body_begin + ((int64_t)threadIdx.x + (int64_t)k * kThreads) * V;
+                if (v < body_end) {
+                    const uint4 sraw = load_plain_16B(static_cast<const T*>(ex.start) + v);
+#pragma unroll
+                    for (int i = 0; i < R; ++i)
+                        if (i < members)
+                            raw[i][k] = delta_words<T>(raw[i][k], sraw);
+                }
+            }
+        }
+        float acc[E];
+#pragma unroll
+        for (int e = 0; e < E; ++e)
+            acc[e] = 0.0f;
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            float x[R][V];
+#pragma unroll
+            for (int i = 0; i < R; ++i)
+                decode_vector<T>(raw[i][k], x[i]);         // zero vectors beyond the segment add nothing
+#pragma unroll
+            for (int j = 0; j < V; ++j) {
+                float col[R];
+#pragma unroll
+                for (int i = 0; i < R; ++i)
+                    col[i] = x[i][j];
+                gram_accumulate<R>(col, acc);
+            }
+        }
+        // scalar head [begin, body_begin) and tail [body_end, end)
+        for (int pass = 0; pass < 2; ++pass) {
+            const int64_t lo = pass == 0 ? begin : body_end;
+            const int64_t hi = pass == 0 ? body_begin : end;
+            for (int64_t e = lo + threadIdx.x; e < hi; e += kThreads) {
+                float col[R];
+#pragma unroll
+                for (int i = 0; i < R; ++i) {
+                    if constexpr (DELTA)
+                        col[i] = i < members ? delta_one(src[i], static_cast<const T*>(ex.start), e) : 0.0f;
+                    else
+                        col[i] = i < members ? Element<T>::one(src[i] + e) : 0.0f;
+                }
+                gram_accumulate<R>(col, acc);
+            }
+        }
+        block_reduce_gram<E>(acc, partials + (int64_t)blockIdx.x * E);
+    } else if (has_segment) {
+        gram_of_segment<T, R, VEC, DELTA>(ops, 0, members, seg, partials + (int64_t)blockIdx.x * E,
+                                          static_cast<const T*>(ex.start));
+    }
+
+    // ---- the small tensors, one warp each, while the segments' loads and stores drain
+    {
+        TreeOptions opt = fin.tree;
+        const int warps_total = (int)gridDim.x * kWarps;
+        // dealt from the last block backwards: the first blocks are the ones whose segments are longest
+        const int first = ((int)gridDim.x - 1 - (int)blockIdx.x) * kWarps + (threadIdx.x >> 5);
+        for (int s = first; s < num_warp_tensors; s += warps_total)
+            reduce_warp_tensor<T, R, DELTA>(ops, members, warp_tensors[s], opt, out, ex);
+    }
+
     __threadfence();
     cooperative_groups::this_grid().sync();
+    if (!has_segment)
+        return;
 
+    // ---- coefficients of this block's tensor, then pass 2 of its segment
     __shared__ float leaf_weights[R];
     const int s0 = fin.seg_first[2 * seg.tensor], s1 = fin.seg_first[2 * seg.tensor + 1];
     TreeOptions opt = fin.tree;
@@ -1778,9 +2103,55 @@ fused_small_kernel(const __grid_constant__ OperandTable ops, int operands,
         opt.leaf_norm_sums = nullptr;
         opt.orthogonality = nullptr;
     }
-    finish_group_in_block<R>(partials, s0, s1, seg.tensor, 0, 1, members, leaf_weights, opt);
-    __syncthreads();
-    weighted_sum_of_segment<T, R, VEC, DELTA>(ops, 0, members, seg, leaf_weights, out, ex);
+    finish_small<R>(partials, s0, s1, seg.tensor, members, leaf_weights, opt);
+    if (keep) {
+        float w[R];
+#pragma unroll
+        for (int i = 0; i < R; ++i)
+            w[i] = leaf_weights[i];
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            const int64_t v = body_begin + ((int64_t)threadIdx.x + (int64_t)k * kThreads) * V;
+            if (v < body_end) {
+                float y[V];
+#pragma unroll
+                for (int j = 0; j < V; ++j)
+                    y[j] = 0.0f;
+#pragma unroll
+                for (int i = 0; i < R; ++i) {
+                    float x[V];
+                    decode_vector<T>(raw[i][k], x);
+#pragma unroll
+                    for (int j = 0; j < V; ++j)
+                        y[j] = fmaf(w[i], x[j], y[j]);
+                }
+                if (ex.base != nullptr)
+                    add_vector_as_float<V>(ex.base, ex.base_dtype, v, y);
+                store_vector_from_float<V>(out, ex.out_dtype, v, y);
+            }
+        }
+        for (int pass = 0; pass < 2; ++pass) {
+            const int64_t lo = pass == 0 ? begin : body_end;
+            const int64_t hi = pass == 0 ? body_begin : end;
+            for (int64_t e = lo + threadIdx.x; e < hi; e += kThreads) {
+                float y = 0.0f;
+#pragma unroll
+                for (int i = 0; i < R; ++i) {
+                    if (i < members) {
+                        if constexpr (DELTA)
+                            y = fmaf(w[i], delta_one(static_cast<const T*>(ops.ptr[i]), static_cast<const T*>(ex.start), e), y);
+                        else
+                            y = fmaf(w[i], Element<T>::one(static_cast<const T*>(ops.ptr[i]) + e), y);
+                    }
+                }
+                if (ex.base != nullptr)
+                    y += load_as_float(ex.base, ex.base_dtype, e);
+                store_from_float(out, ex.out_dtype, e, y);
+            }
+        }
+    } else {
+        weighted_sum_of_segment<T, R, VEC, DELTA>(ops, 0, members, seg, leaf_weights, out, ex);
+    }
 }
 
 // n_workers = 1: the result is the input (with a start: start + (input - start), the difference

@@ -142,8 +142,9 @@ void launch_tree_from_sums(const double* gram64, int32_t num_tensors, int operan
 }
 
 template <typename T, int R, bool VEC>
-cudaError_t launch_fused_small(const OperandTable& ops, int operands, const SegmentTable& tab, float* partials,
-                               const FinishArgs& fin, void* out, const PassExtras& ex, int* status, cudaStream_t stream)
+cudaError_t launch_fused_small(const OperandTable& ops, int operands, const SegmentTable& tab, int resident_blocks,
+                               float* partials, const FinishArgs& fin, void* out, const PassExtras& ex, int* status,
+                               cudaStream_t stream)
 {
     const void* kernel = (const void*)fused_small_kernel<T, R, VEC, false>;
     if constexpr (VEC) {
@@ -154,21 +155,32 @@ cudaError_t launch_fused_small(const OperandTable& ops, int operands, const Segm
         return cudaErrorInvalidValue;
     int operands_arg = operands;
     const Segment* segments = tab.d_segments;
+    int num_segments = tab.num_segments;
+    const WarpTensor* warp_tensors = tab.d_warp;
+    int num_warp_tensors = (int)tab.h_warp.size();
     PassExtras ex_arg = ex;
-    void* args[] = {(void*)&ops, (void*)&operands_arg, (void*)&segments, (void*)&partials,
-                    (void*)&fin, (void*)&out,          (void*)&ex_arg,   (void*)&status};
-    return cudaLaunchCooperativeKernel(kernel, dim3((unsigned)tab.num_segments), dim3(kThreads), args, 0, stream);
+    // one block per segment, and enough blocks for the small tensors' warps (never more than are resident)
+    int for_warps = (num_warp_tensors + kWarps - 1) / kWarps;
+    if (for_warps > resident_blocks)
+        for_warps = resident_blocks;
+    int grid = num_segments > for_warps ? num_segments : for_warps;
+    if (grid < 1)
+        grid = 1;
+    void* args[] = {(void*)&ops,          (void*)&operands_arg,     (void*)&segments, (void*)&num_segments,
+                    (void*)&warp_tensors, (void*)&num_warp_tensors, (void*)&partials, (void*)&fin,
+                    (void*)&out,          (void*)&ex_arg,           (void*)&status};
+    return cudaLaunchCooperativeKernel(kernel, dim3((unsigned)grid), dim3(kThreads), args, 0, stream);
 }
 
 template <typename T, bool VEC>
 cudaError_t launch_fused_small_radix(int radix, const OperandTable& ops, int operands, const SegmentTable& tab,
-                                     float* partials, const FinishArgs& fin, void* out, const PassExtras& ex,
-                                     int* status, cudaStream_t stream)
+                                     int resident_blocks, float* partials, const FinishArgs& fin, void* out,
+                                     const PassExtras& ex, int* status, cudaStream_t stream)
 {
     switch (radix) {
-    case 2: return launch_fused_small<T, 2, VEC>(ops, operands, tab, partials, fin, out, ex, status, stream);
-    case 4: return launch_fused_small<T, 4, VEC>(ops, operands, tab, partials, fin, out, ex, status, stream);
-    case 8: return launch_fused_small<T, 8, VEC>(ops, operands, tab, partials, fin, out, ex, status, stream);
+    case 2: return launch_fused_small<T, 2, VEC>(ops, operands, tab, resident_blocks, partials, fin, out, ex, status, stream);
+    case 4: return launch_fused_small<T, 4, VEC>(ops, operands, tab, resident_blocks, partials, fin, out, ex, status, stream);
+    case 8: return launch_fused_small<T, 8, VEC>(ops, operands, tab, resident_blocks, partials, fin, out, ex, status, stream);
     default: return cudaErrorInvalidValue;
     }
 }
@@ -297,11 +309,14 @@ cudaError_t noalloc_launch(bool vec, const OperandTable& ops, const SegmentTable
 
 template <typename T>
 cudaError_t launch_fused_small_any(bool vec, int radix, const OperandTable& ops, int operands,
-                                   const SegmentTable& tab, float* partials, const FinishArgs& fin, void* out,
-                                   const PassExtras& ex, int* status, cudaStream_t stream)
+                                   const SegmentTable& tab, int resident_blocks, float* partials,
+                                   const FinishArgs& fin, void* out, const PassExtras& ex, int* status,
+                                   cudaStream_t stream)
 {
-    return vec ? launch_fused_small_radix<T, true>(radix, ops, operands, tab, partials, fin, out, ex, status, stream)
-               : launch_fused_small_radix<T, false>(radix, ops, operands, tab, partials, fin, out, ex, status, stream);
+    return vec ? launch_fused_small_radix<T, true>(radix, ops, operands, tab, resident_blocks, partials, fin, out, ex,
+                                                   status, stream)
+               : launch_fused_small_radix<T, false>(radix, ops, operands, tab, resident_blocks, partials, fin, out, ex,
+                                                    status, stream);
 }
 
 template <typename T>
@@ -315,7 +330,7 @@ cudaError_t launch_convert(const void* src, void* dst, int64_t n, const PassExtr
 
 #define ADASUM_INSTANTIATE_LEVELS(T)                                                                              \
     template adasum_status_t run_level<T>(int, const LevelArgs&);                                                 \
-    template cudaError_t launch_fused_small_any<T>(bool, int, const OperandTable&, int, const SegmentTable&,      \
+    template cudaError_t launch_fused_small_any<T>(bool, int, const OperandTable&, int, const SegmentTable&, int, \
                                                    float*, const FinishArgs&, void*, const PassExtras&, int*,     \
                                                    cudaStream_t);                                                 \
     template cudaError_t noalloc_launch<T>(bool, const OperandTable&, const SegmentTable&, int32_t, float*,       \
