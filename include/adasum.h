@@ -20,8 +20,10 @@
  * large terms (a one-element tensor whose workers disagree in sign), so adasum_reduce,
  * adasum_reduce_ex, adasum_reduce_delta and adasum_pair apply the operator to them literally, pair
  * by pair and level by level, in fp64 from the loads to the one rounding of the stored result (one
- * more small kernel launch when a buffer has such tensors; the sharded calls, whose tensors are
- * spread over several GPUs, keep to the general path).
+ * more small kernel when a buffer has such tensors, run beside the streaming passes on a stream of
+ * the library's own that is forked from `stream` and joined to it again with events before the call
+ * returns; the single-launch path does them inside its one kernel; the sharded calls, whose tensors
+ * are spread over several GPUs, keep to the general path).
  *
  * Conventions for every entry point:
  *   - plain C, no exceptions; every call returns a status, and on any status other than

@@ -429,6 +429,76 @@ adasum_status_t get_segment_table(const int64_t* offsets, int32_t num_tensors, i
     return ADASUM_OK;
 }
 
+// ---- side streams ---------------------------------------------------------------------------------
+//
+// The kernel for the tensors of at most 64 elements is independent of the streaming passes (other
+// elements of the output, its own part of the workspace), so it runs beside them: forked from the
+// caller's stream with an event, on a stream of the library's own, joined with a second event
+// before the call returns.  Both dependencies are ordinary stream operations (they are recorded
+// like any other when the caller's stream is being captured).  A lane is borrowed for the duration
+// of one call; lanes are created on demand and kept until adasum_shutdown().
+
+struct SideLane {
+    int device = -1;
+    cudaStream_t stream = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+};
+
+std::mutex g_lanes_mutex;
+std::vector<SideLane> g_lanes;
+
+bool borrow_lane(SideLane* lane)
+{
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess)
+        return false;
+    {
+        std::lock_guard<std::mutex> lock(g_lanes_mutex);
+        for (size_t i = 0; i < g_lanes.size(); ++i) {
+            if (g_lanes[i].device == device) {
+                *lane = g_lanes[i];
+                g_lanes.erase(g_lanes.begin() + (ptrdiff_t)i);
+                return true;
+            }
+        }
+    }
+    SideLane fresh;
+    fresh.device = device;
+    if (cudaStreamCreateWithFlags(&fresh.stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&fresh.fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&fresh.join, cudaEventDisableTiming) != cudaSuccess) {
+        if (fresh.stream)
+            cudaStreamDestroy(fresh.stream);
+        if (fresh.fork)
+            cudaEventDestroy(fresh.fork);
+        (void)cudaGetLastError();
+        return false;
+    }
+    *lane = fresh;
+    return true;
+}
+
+void return_lane(const SideLane& lane)
+{
+    std::lock_guard<std::mutex> lock(g_lanes_mutex);
+    g_lanes.push_back(lane);
+}
+
+// Joins a forked lane into `stream` when the call ends, however it ends.
+struct LaneJoin {
+    SideLane lane;
+    cudaStream_t stream = nullptr;
+    bool forked = false;
+    ~LaneJoin()
+    {
+        if (!forked)
+            return;
+        cudaEventRecord(lane.join, lane.stream);
+        cudaStreamWaitEvent(stream, lane.join, 0);
+        return_lane(lane);
+    }
+};
+
 // ---- single-launch path for inputs that fit the L2 ------------------------------------------------
 
 constexpr int64_t kSmallInputBytes = int64_t(96) << 20;    // operands that the 126 MB L2 holds with room to spare
@@ -691,10 +761,12 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         if (st != ADASUM_OK)
             return st;
     }
-    auto run_short = [&]() -> adasum_status_t {
+    bool short_done = false;
+    auto run_short = [&](cudaStream_t stream) -> adasum_status_t {       // launches on the stream it is given
         const int num_short = short_ref ? (int)short_ref->h_short.size() : 0;
-        if (num_short == 0)
+        if (num_short == 0 || short_done)
             return ADASUM_OK;
+        short_done = true;
         ShortArgs sa{};
         sa.table = short_ref->d_short;
         sa.order = tree_order(n_workers, flags);
@@ -742,7 +814,24 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         return ADASUM_OK;
     };
     if (short_ref && short_ref->num_segments == 0)        // every tensor is short
-        return run_short();
+        return run_short(stream);
+    // Beside the streaming passes, on a stream of the library's own (not while launches are being
+    // timed one by one, and not where the single-launch kernel takes these tensors itself).
+    LaneJoin lane_join;
+    if (short_ref && !short_ref->h_short.empty() && !small_candidate && !g_profiler.enabled &&
+        borrow_lane(&lane_join.lane)) {
+        lane_join.stream = stream;
+        if (cudaEventRecord(lane_join.lane.fork, stream) == cudaSuccess &&
+            cudaStreamWaitEvent(lane_join.lane.stream, lane_join.lane.fork, 0) == cudaSuccess) {
+            lane_join.forked = true;
+            st = run_short(lane_join.lane.stream);
+            if (st != ADASUM_OK)
+                return st;
+        } else {
+            (void)cudaGetLastError();
+            return_lane(lane_join.lane);
+        }
+    }
 
     // Inputs that fit the L2: one cooperative launch does both passes and HBM sees the operands once.
     if (small_candidate) {
@@ -776,7 +865,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
                 err = launch_fused_small_any<__nv_bfloat16>(vec, radix, table, n_workers, *tab, small_blocks, partials, fin, out, ex, dev_status, stream);
             if (err == cudaSuccess) {
                 profile_mark(stream, ADASUM_KERNEL_FUSED_SMALL, 0, radix, false);
-                return run_short();
+                return ADASUM_OK;          // the tensors of at most 64 elements included
             }
             if (err != cudaErrorCooperativeLaunchTooLarge)
                 return fail(ADASUM_ERR_CUDA, "cooperative launch: %s", cudaGetErrorString(err));
@@ -877,7 +966,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
                 operand_ptrs[g] = static_cast<float*>(a.dst) + (int64_t)g * lay.padded_elems;
         }
     }
-    return run_short();
+    return run_short(stream);       // unless they already run on the side stream
 }
 
 // ---- fp64 gradients ------------------------------------------------------------------------------
@@ -1511,6 +1600,21 @@ adasum_status_t adasum_shutdown(void)
         g_profiler.events.clear();
         g_profiler.marks.clear();
         g_profiler.used = 0;
+    }
+    {
+        std::lock_guard<std::mutex> lock(g_lanes_mutex);
+        for (const SideLane& lane : g_lanes) {
+            int current = 0;
+            const bool have = cudaGetDevice(&current) == cudaSuccess;
+            if (have && current != lane.device)
+                cudaSetDevice(lane.device);
+            cudaStreamDestroy(lane.stream);
+            cudaEventDestroy(lane.fork);
+            cudaEventDestroy(lane.join);
+            if (have && current != lane.device)
+                cudaSetDevice(current);
+        }
+        g_lanes.clear();
     }
     std::vector<std::shared_ptr<SegmentTable>> dropped;
     {

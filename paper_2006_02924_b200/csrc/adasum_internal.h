@@ -33,15 +33,6 @@ void profile_mark(cudaStream_t stream, int kernel, int level, int radix, bool st
 constexpr int kShortTensorElems = 64;            // tensors of at most this many elements take the fp64 path
 constexpr int kShortChunkLeaves = 64;            // leaves a block reduces per round in shared memory
 
-// One short tensor: where it starts in the fused buffers, and where in the packed numbering of
-// the short tensors' elements (used for the fp64 vectors that travel between launches).
-struct ShortTensor {
-    int64_t begin;
-    int32_t len;
-    int32_t tensor;
-    int64_t packed;
-};
-
 struct ShortArgs {
     const ShortTensor* table;     // device, one entry per short tensor (= per block)
     int order;                    // 0 bottom-up pairs with carry, 1 sequential, 2 top-down halves

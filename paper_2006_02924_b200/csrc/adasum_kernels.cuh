@@ -32,6 +32,8 @@
 #include <cuda_fp16.h>
 #include <stdint.h>
 
+#include "adasum_short.cuh"
+
 namespace adasum {
 
 constexpr int kThreads = 256;               // threads per block of the streaming kernels
@@ -1465,6 +1467,10 @@ gram_finish_kernel(const float* __restrict__ partials, const int32_t* __restrict
     }
     if (SINGLE && !sums_only) {      // sums_only is uniform over the grid
         __syncthreads();
+        if (s0 == s1) {              // no segments: an empty tensor, or one that another kernel reduces
+            opt.leaf_norm_sums = nullptr;
+            opt.orthogonality = nullptr;
+        }
         tree_weights_from_gram<R>(gram, min(R, operands - group * R),
                                   weights + ((int64_t)tensor * groups + group) * R, opt, tensor, group);
     }
@@ -1475,11 +1481,18 @@ gram_finish_kernel(const float* __restrict__ partials, const int32_t* __restrict
 // run the tree.
 template <int R>
 __global__ void __launch_bounds__(kThreads)
-tree_weights_kernel(const double* __restrict__ gram64, int operands, float* __restrict__ weights, TreeOptions opt)
+tree_weights_kernel(const double* __restrict__ gram64, int operands, float* __restrict__ weights, TreeOptions opt,
+                    const int32_t* __restrict__ seg_first)
 {
     constexpr int E = gram_entries(R);
     __shared__ double gram[E];
     const int tensor = blockIdx.x, group = blockIdx.y, groups = gridDim.y;
+    // a tensor without segments (seg_first given): empty, or reduced by another kernel, which then
+    // also reports its by-products
+    if (seg_first != nullptr && seg_first[2 * tensor] == seg_first[2 * tensor + 1]) {
+        opt.leaf_norm_sums = nullptr;
+        opt.orthogonality = nullptr;
+    }
     const double* src = gram64 + ((int64_t)tensor * groups + group) * E;
     for (int k = threadIdx.x; k < E; k += kThreads)
         gram[k] = src[k];
@@ -1764,6 +1777,16 @@ wsum_gram_kernel(const __grid_constant__ OperandTable ops, int operands,
 
 constexpr int kWarpTensorElems = 2048;
 
+// One tensor of at most kShortSlotElems elements: where it starts in the fused buffers, and where in
+// the packed numbering of the short tensors' elements (used for the fp64 vectors that travel
+// between the launches of adasum_short.cu).
+struct ShortTensor {
+    int64_t begin;
+    int32_t len;
+    int32_t tensor;
+    int64_t packed;
+};
+
 // A small tensor that one warp reduces: `begin`, `len` in the fused buffers; `tensor` its index.
 struct WarpTensor {
     int64_t begin;
@@ -1925,6 +1948,48 @@ __device__ void reduce_warp_tensor(const OperandTable& ops, int members, const W
     }
 }
 
+// One tensor of at most kShortSlotElems elements by one warp, in fp64 from the loads to the store and
+// with the operator applied literally (what adasum_short.cu does for the other paths): the leaves go
+// to `slot` (this warp's R x kShortSlotElems doubles of shared memory), the tree runs in place.
+template <typename T, int R, bool DELTA>
+__device__ void reduce_short_tensor_warp(const OperandTable& ops, int members, const ShortTensor& st,
+                                         const TreeOptions& opt, double* slot, void* out, const PassExtras& ex)
+{
+    const int lane = threadIdx.x & 31;
+    const int len = st.len;
+    double leaf_sum = 0.0;
+    for (int i = 0; i < members; ++i) {
+        const T* src = static_cast<const T*>(ops.ptr[i]);
+        double sq = 0.0;
+        for (int e = lane; e < len; e += 32) {
+            double x;
+            if constexpr (DELTA)
+                x = (double)delta_one(src, static_cast<const T*>(ex.start), st.begin + e);
+            else
+                x = (double)Element<T>::one(src + st.begin + e);
+            slot[i * kShortSlotElems + e] = x;
+            sq += x * x;
+        }
+        leaf_sum += warp_sum(sq);
+    }
+    __syncwarp();
+    warp_tree_in_place(slot, members, len, opt.linear);
+    __syncwarp();
+    if (opt.orthogonality != nullptr) {
+        const double r0 = lane < len ? slot[lane] : 0.0, r1 = lane + 32 < len ? slot[lane + 32] : 0.0;
+        const double norm = warp_sum(r0 * r0 + r1 * r1);
+        if (lane == 0)
+            opt.orthogonality[st.tensor] = leaf_sum == 0.0 ? __int_as_float(0x7fc00000) : (float)(norm / leaf_sum);
+    }
+    for (int e = lane; e < len; e += 32) {
+        double y = slot[e];
+        if (ex.base != nullptr)
+            y += (double)load_as_float(ex.base, ex.base_dtype, st.begin + e);
+        store_from_float(out, ex.out_dtype, st.begin + e, (float)y);
+    }
+    __syncwarp();
+}
+
 // The partial matrices of segments [seg_begin, seg_end) added in fp64 in a fixed order by the whole
 // block, then the tree: leaf weights to weights_dst (shared memory), by-products as opt says.
 // Thread (q, kk) adds the partials of segments q, q + Q, ... for entry kk; a warp then adds the Q
@@ -1987,11 +2052,13 @@ __global__ void __launch_bounds__(kThreads, 2)
 fused_small_kernel(const __grid_constant__ OperandTable ops, int operands,
                    const Segment* __restrict__ segments, int num_segments,
                    const WarpTensor* __restrict__ warp_tensors, int num_warp_tensors,
+                   const ShortTensor* __restrict__ short_tensors, int num_short_tensors,
                    float* __restrict__ partials, FinishArgs fin, void* out, PassExtras ex, int* __restrict__ status)
 {
     constexpr int E = gram_entries(R);
     constexpr int V = Element<T>::kVec;
     constexpr int K = small_keep_vectors<R>();
+    __shared__ double short_slots[kWarps][R * kShortSlotElems];
     // This path uses no ticket counters, so the host does not clear them (one operation less in
     // front of a reduce that takes microseconds); the device status word, which lives beside
     // them and which adasum_device_status reads, is cleared here instead.
@@ -2088,6 +2155,10 @@ fused_small_kernel(const __grid_constant__ OperandTable ops, int operands,
         const int first = ((int)gridDim.x - 1 - (int)blockIdx.x) * kWarps + (threadIdx.x >> 5);
         for (int s = first; s < num_warp_tensors; s += warps_total)
             reduce_warp_tensor<T, R, DELTA>(ops, members, warp_tensors[s], opt, out, ex);
+        // ... and the tensors of at most 64 elements, in fp64
+        for (int s = first; s < num_short_tensors; s += warps_total)
+            reduce_short_tensor_warp<T, R, DELTA>(ops, members, short_tensors[s], opt, short_slots[threadIdx.x >> 5],
+                                                  out, ex);
     }
 
     __threadfence();

@@ -127,7 +127,7 @@ cudaError_t launch_weights(const float* partials, const SegmentTable& tab, int32
         return cudaSuccess;
     if constexpr (tree_entry_blocks(R) > 1) {
         dim3 grid2((unsigned)num_tensors, (unsigned)groups);
-        tree_weights_kernel<R><<<grid2, kThreads, 0, stream>>>(gram64, operands, weights, opt);
+        tree_weights_kernel<R><<<grid2, kThreads, 0, stream>>>(gram64, operands, weights, opt, tab.d_seg_first);
         *launches = 2;
     }
     return cudaSuccess;
@@ -138,7 +138,7 @@ void launch_tree_from_sums(const double* gram64, int32_t num_tensors, int operan
                            const TreeOptions& opt, cudaStream_t stream)
 {
     dim3 grid((unsigned)num_tensors, (unsigned)groups);
-    tree_weights_kernel<R><<<grid, kThreads, 0, stream>>>(gram64, operands, weights, opt);
+    tree_weights_kernel<R><<<grid, kThreads, 0, stream>>>(gram64, operands, weights, opt, nullptr);
 }
 
 template <typename T, int R, bool VEC>
@@ -158,17 +158,21 @@ cudaError_t launch_fused_small(const OperandTable& ops, int operands, const Segm
     int num_segments = tab.num_segments;
     const WarpTensor* warp_tensors = tab.d_warp;
     int num_warp_tensors = (int)tab.h_warp.size();
+    const ShortTensor* short_tensors = tab.d_short;
+    int num_short_tensors = (int)tab.h_short.size();
     PassExtras ex_arg = ex;
     // one block per segment, and enough blocks for the small tensors' warps (never more than are resident)
-    int for_warps = (num_warp_tensors + kWarps - 1) / kWarps;
+    const int small = num_warp_tensors > num_short_tensors ? num_warp_tensors : num_short_tensors;
+    int for_warps = (small + kWarps - 1) / kWarps;
     if (for_warps > resident_blocks)
         for_warps = resident_blocks;
     int grid = num_segments > for_warps ? num_segments : for_warps;
     if (grid < 1)
         grid = 1;
     void* args[] = {(void*)&ops,          (void*)&operands_arg,     (void*)&segments, (void*)&num_segments,
-                    (void*)&warp_tensors, (void*)&num_warp_tensors, (void*)&partials, (void*)&fin,
-                    (void*)&out,          (void*)&ex_arg,           (void*)&status};
+                    (void*)&warp_tensors, (void*)&num_warp_tensors, (void*)&short_tensors, (void*)&num_short_tensors,
+                    (void*)&partials,     (void*)&fin,              (void*)&out,      (void*)&ex_arg,
+                    (void*)&status};
     return cudaLaunchCooperativeKernel(kernel, dim3((unsigned)grid), dim3(kThreads), args, 0, stream);
 }
 

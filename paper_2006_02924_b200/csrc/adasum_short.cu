@@ -20,6 +20,7 @@
 namespace adasum {
 namespace {
 
+static_assert(kShortTensorElems == kShortSlotElems, "a leaf slot holds the longest short tensor");
 constexpr int kShortThreads = 256;
 constexpr int kShortWarps = kShortThreads / 32;
 constexpr int kShortMaxChunks = kMaxOperandsPerLaunch / kShortChunkLeaves;
@@ -36,31 +37,6 @@ template <>
 __device__ __forceinline__ double short_load<double>(const void* p, const void*, int64_t e)
 {
     return static_cast<const double*>(p)[e];
-}
-
-__device__ __forceinline__ double warp_sum(double v)
-{
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1)
-        v += __shfl_xor_sync(0xffffffffu, v, d);
-    return v;
-}
-
-// a <- Adasum(a, b) for vectors of len <= 64 doubles in shared memory, by one warp.
-__device__ __forceinline__ void pair_in_place(double* a, const double* b, int len, int lane)
-{
-    const double a0 = lane < len ? a[lane] : 0.0, a1 = lane + 32 < len ? a[lane + 32] : 0.0;
-    const double b0 = lane < len ? b[lane] : 0.0, b1 = lane + 32 < len ? b[lane + 32] : 0.0;
-    const double dot = warp_sum(a0 * b0 + a1 * b1);
-    const double na = warp_sum(a0 * a0 + a1 * a1);
-    const double nb = warp_sum(b0 * b0 + b1 * b1);
-    // Algorithm 1, "Apply Adasum"; an operand with zero squared norm keeps coefficient 1
-    const double ca = na == 0.0 ? 1.0 : 1.0 - dot / (2.0 * na);
-    const double cb = nb == 0.0 ? 1.0 : 1.0 - dot / (2.0 * nb);
-    if (lane < len)
-        a[lane] = ca * a0 + cb * b0;
-    if (lane + 32 < len)
-        a[lane + 32] = ca * a1 + cb * b1;
 }
 
 // The tree over slot[0 .. n) (each kShortTensorElems doubles); the result ends in slot[0].

@@ -213,3 +213,42 @@ def test_unaligned_buffers_and_zero_leaves(lib):
     ref = oracle.adasum_reduce([_np(g, "f16") for g in grads], offsets=offsets, dtype="f16", threads=0)
     _check(out, ref, offsets, 2e-3)
     assert not out[lo1:hi1].any()
+
+
+def test_side_stream_under_graph_capture_and_back_to_back_calls(lib):
+    """Outside the per-launch timing mode the fp64 kernel runs on a stream of the library's own, forked
+    from the caller's stream and joined to it with events.  Back-to-back calls on one workspace and a
+    captured, replayed call must order it correctly against everything else."""
+    offsets = workloads.offsets_from_sizes(SIZES)
+    total = int(offsets[-1])
+    n = 24
+    grads = _cancelling(n, offsets, "f32", seed=5700)
+    ref = oracle.adasum_reduce([_np(g, "f32") for g in grads], offsets=offsets, dtype="f32", threads=0)
+    out = torch.empty(total, device="cuda")
+    ws = torch.empty(lib.adasum_workspace_bytes(total, len(SIZES), n, "f32"), dtype=torch.uint8, device="cuda")
+    for _ in range(5):                          # no synchronisation in between
+        out.fill_(float("nan"))
+        lib.adasum_reduce(grads, offsets, out=out, workspace=ws)
+    torch.cuda.synchronize()
+    _check(out, ref, offsets, 1e-5)
+    side = torch.cuda.Stream()                  # a caller's stream other than the default one
+    with torch.cuda.stream(side):
+        out.fill_(float("nan"))
+        lib.adasum_reduce(grads, offsets, out=out, workspace=ws, stream=side)
+        first = out.clone()
+    side.synchronize()
+    _check(first, ref, offsets, 1e-5)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        lib.adasum_reduce(grads, offsets, out=out, workspace=ws)
+    out.fill_(float("nan"))
+    graph.replay()
+    torch.cuda.synchronize()
+    _check(out, ref, offsets, 1e-5)
+    fresh = _cancelling(n, offsets, "f32", seed=5701)
+    for dst, src in zip(grads, fresh):
+        dst.copy_(src)
+    graph.replay()
+    torch.cuda.synchronize()
+    _check(out, oracle.adasum_reduce([_np(g, "f32") for g in grads], offsets=offsets, dtype="f32", threads=0), offsets,
+           1e-5)
