@@ -564,7 +564,7 @@ def measure_config(lib, name, spec, steps, warmup, flags, peak, peak_kind, *, wo
                    sampler=None, e2e_steps=3, cpu_seconds=10.0, tensor_sizes=None, traffic_key=None):
     """One configuration end to end: the timed steps, the per-launch breakdown with the roofline of
     the dominant kernel, the end-to-end leg and (one GPU only) the CPU oracle beside it."""
-    sharded = mode == "sharded" and world > 1
+    sharded = mode == "sharded"
     wl = workloads.generate(spec, device="cuda", tensor_sizes=tensor_sizes, replica=rank)
     reducer = Reducer(lib, wl, flags, sharded=sharded)
     ms_local = time_steps(reducer, steps, warmup, world=world, sampler=sampler)
@@ -593,11 +593,13 @@ def measure_config(lib, name, spec, steps, warmup, flags, peak, peak_kind, *, wo
         "whole_reduce": whole_reduce_summary(spec.n_workers, job_elems if sharded else wl.total_elems, eb,
                                              ms if sharded else ms_local, peak),
     }
-    e2e_ms_local, h2d, d2h, _ = time_e2e(reducer, e2e_steps, world=world)
-    e2e_ms, _ = aggregate_over_ranks(e2e_ms_local, 0.0, world, "cuda")
-    e2e = {"value": job_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
-           "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps,
-           "bytes_are": "per rank" if world > 1 else "whole job"}
+    e2e = None
+    if e2e_steps > 0:
+        e2e_ms_local, h2d, d2h, _ = time_e2e(reducer, e2e_steps, world=world)
+        e2e_ms, _ = aggregate_over_ranks(e2e_ms_local, 0.0, world, "cuda")
+        e2e = {"value": job_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps,
+               "bytes_are": "per rank" if world > 1 else "whole job"}
     cpu_baseline = None
     if rank == 0 and world == 1 and cpu_seconds > 0:
         cpu_baseline = cpu_baseline_of(wl, name, cpu_seconds)
@@ -624,6 +626,9 @@ def cuda_arm(args):
     torch.cuda.set_device(local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    elif args.force_multi:          # the multi-GPU code path on a group of one rank
+        dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29687", rank=0, world_size=1,
+                                device_id=torch.device("cuda", local_rank))
     from paper_2006_02924_b200 import binding as lib
 
     flags = lib.flags_radix(args.radix_first, args.radix_later)
@@ -634,7 +639,7 @@ def cuda_arm(args):
     peak, peak_kind = measured_peak()
     sampler = ClockSampler(local_rank)
     steps, warmup = max(args.steps, 1), max(args.warmup, 3)
-    mode = "single" if world == 1 else args.multi
+    mode = "single" if world == 1 and not args.force_multi else args.multi
     single = rank == 0 and world == 1
 
     main_spec = resolve_spec(args.workload, args.n_workers, args.tensor_list)
@@ -695,7 +700,7 @@ def cuda_arm(args):
         if "allreduce_bytes_per_level" in head:
             line["config"]["allreduce_bytes_per_level"] = head["allreduce_bytes_per_level"]
         print(json.dumps(line))
-    if world > 1:
+    if dist.is_initialized():
         dist.barrier()
         dist.destroy_process_group()
 
@@ -710,6 +715,8 @@ def main():
     ap.add_argument("--multi", default="sharded", choices=["sharded", "replicas"],
                     help="with several GPUs: every rank holds a slice of every tensor and the Gram sums are "
                          "all-reduced (sharded), or every rank reduces an independent copy of the workload (replicas)")
+    ap.add_argument("--force-multi", action="store_true",
+                    help="with one GPU: run the --multi code path all the same, on a process group of one rank")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-seconds", type=float, default=12.0,
                     help="about how long the CPU oracle runs on its sample of the headline workload")
