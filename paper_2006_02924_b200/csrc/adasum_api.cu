@@ -505,11 +505,28 @@ constexpr int64_t kSmallInputBytes = int64_t(96) << 20;    // operands that the 
 constexpr int kSmallBlocksPerSm = 2;                       // blocks per SM the grid is sized for (all variants keep >= 2 resident)
 constexpr int kSmallSegmentGrain = 1024;
 
+// Segments that build_segments makes of the tensors of more than kWarpTensorElems elements at this
+// segment length (cuts on the 64-element grid of the fused buffer).
+int64_t count_long_segments(const int64_t* offsets, int32_t num_tensors, int64_t seg_len)
+{
+    int64_t n = 0;
+    for (int32_t t = 0; t < num_tensors; ++t) {
+        const int64_t b = offsets[t], e = offsets[t + 1];
+        if (e - b <= kWarpTensorElems)
+            continue;
+        const int64_t first_cut = b / 64 * 64 + seg_len;
+        n += first_cut >= e ? 1 : 1 + (e - first_cut + seg_len - 1) / seg_len;
+    }
+    return n;
+}
+
 // Host-only rule (no device query): is this reduce served by fused_small_kernel, and with which
-// segment length?  `blocks` is the number of blocks that can be resident at once; only the
-// `big_tensors` tensors of more than kWarpTensorElems elements (`big_elems` elements in all) are cut
-// into segments, one block each.
-bool small_input_plan(const LevelPlan& plan, int64_t total, int64_t big_tensors, int64_t big_elems, int n_workers,
+// segment length?  `blocks` is the number of blocks that can be resident at once; only the tensors
+// of more than kWarpTensorElems elements are cut into segments, one block each.  With the offsets
+// the shortest segment length (a multiple of kSmallSegmentGrain) whose segments fit the blocks is
+// found exactly; without them (offsets == nullptr, adasum_plan_info) every tensor is taken for a
+// long one with two ragged ends.
+bool small_input_plan(const LevelPlan& plan, int64_t total, int32_t num_tensors, const int64_t* offsets, int n_workers,
                       int elem_bytes, uint32_t flags, int blocks, int* seg_len)
 {
     if (plan.num_levels != 1 || plan.level[0].radix > 8 || plan.level[0].groups != 1)
@@ -518,15 +535,29 @@ bool small_input_plan(const LevelPlan& plan, int64_t total, int64_t big_tensors,
         return false;
     if (total <= 0 || (int64_t)n_workers * total * elem_bytes > kSmallInputBytes)
         return false;
-    // a tensor's first and last segments may be ragged: budget for those first
-    const int64_t room = (int64_t)blocks - 2 * big_tensors;
-    if (room < 8)
-        return false;
-    int64_t len = (big_elems + room - 1) / room;
-    len = (len + kSmallSegmentGrain - 1) / kSmallSegmentGrain * kSmallSegmentGrain;
-    if (len < 2048)
-        len = 2048;
-    if (len > (int64_t(1) << 20))
+    constexpr int64_t kLongest = int64_t(1) << 20;
+    auto round_up = [](int64_t len) {
+        len = (len + kSmallSegmentGrain - 1) / kSmallSegmentGrain * kSmallSegmentGrain;
+        return len < 2048 ? int64_t(2048) : len;
+    };
+    if (offsets == nullptr) {
+        const int64_t room = (int64_t)blocks - 2 * (int64_t)num_tensors;
+        if (room < 8)
+            return false;
+        const int64_t len = round_up((total + room - 1) / room);
+        if (len > kLongest)
+            return false;
+        *seg_len = (int)len;
+        return true;
+    }
+    int64_t long_elems = 0;
+    for (int32_t t = 0; t < num_tensors; ++t)
+        if (offsets[t + 1] - offsets[t] > kWarpTensorElems)
+            long_elems += offsets[t + 1] - offsets[t];
+    int64_t len = round_up((long_elems + blocks - 1) / blocks);
+    while (len <= kLongest && count_long_segments(offsets, num_tensors, len) > blocks)
+        len += len < 16 * kSmallSegmentGrain ? kSmallSegmentGrain : len / 16 / kSmallSegmentGrain * kSmallSegmentGrain;
+    if (len > kLongest)
         return false;
     *seg_len = (int)len;
     return true;
@@ -556,8 +587,7 @@ int launches_of(const LevelPlan& plan, int n_workers, uint32_t flags, int64_t to
     if (n_workers == 1)
         return 1;
     int seg_len = 0;        // on a B200: 148 SMs
-    // without the offsets every tensor has to be taken for a long one
-    if (small_input_plan(plan, total, num_tensors, total, n_workers, elem_bytes, flags, 148 * kSmallBlocksPerSm, &seg_len))
+    if (small_input_plan(plan, total, num_tensors, nullptr, n_workers, elem_bytes, flags, 148 * kSmallBlocksPerSm, &seg_len))
         return 1;
     int n = 0;
     bool gram_done = false;      // by the previous level's pass 2 (16-byte aligned buffers assumed)
@@ -716,15 +746,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     // Inputs that fit the L2 are served by one cooperative launch that needs no ticket counters.
     int small_seg_len = 0;
     const int small_blocks = (sharded || total == 0 || num_tensors == 0) ? 0 : resident_small_blocks();
-    int64_t big_tensors = 0, big_elems = 0;       // tensors that the single-launch kernel would cut into segments
-    for (int32_t t = 0; t < num_tensors; ++t) {
-        const int64_t len = offsets[t + 1] - offsets[t];
-        if (len > kWarpTensorElems) {
-            ++big_tensors;
-            big_elems += len;
-        }
-    }
-    const bool small_candidate = small_blocks > 0 && small_input_plan(plan, total, big_tensors, big_elems, n_workers, eb,
+    const bool small_candidate = small_blocks > 0 && small_input_plan(plan, total, num_tensors, offsets, n_workers, eb,
                                                                       flags, small_blocks, &small_seg_len);
     // the workspace arrives with unknown contents
     auto clear_counters = [&]() { return cudaMemsetAsync(ws + lay.counters, 0, lay.counters_bytes, stream); };

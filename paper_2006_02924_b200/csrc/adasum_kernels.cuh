@@ -405,7 +405,7 @@ __device__ __forceinline__ void gram_accumulate(const float (&x)[R], float (&acc
 // The Gram matrix of one segment of the group whose first operand is ops.ptr[first], computed by
 // the whole block on the fp32 pipes and written to dst[0 .. E).
 // With DELTA the rows are (operand - start), rounded to T.
-template <typename T, int R, bool VEC, bool DELTA = false>
+template <typename T, int R, bool VEC, bool DELTA = false, int UNROLL = 1>
 __device__ __forceinline__ void gram_of_segment(const OperandTable& ops, int first, int members,
                                                 const Segment& seg, float* __restrict__ dst,
                                                 const T* start = nullptr)
@@ -427,6 +427,9 @@ __device__ __forceinline__ void gram_of_segment(const OperandTable& ops, int fir
     int64_t body_begin, body_end;
     split_segment<V, VEC>(begin, end, body_begin, body_end);
 
+    // UNROLL > 1 (the single-launch kernel, whose blocks are few and bound by latency): that many
+    // independent vectors per thread in flight
+#pragma unroll(UNROLL)
     for (int64_t v = body_begin + (int64_t)threadIdx.x * V; v < body_end; v += (int64_t)kThreads * V) {
         float x[R][V];
         uint4 sraw = make_uint4(0u, 0u, 0u, 0u);
@@ -685,12 +688,9 @@ __host__ __device__ constexpr size_t mma_smem_bytes()
 // with the same columns of `start`; a lane subtracts its 16 bytes of it from every fragment it
 // loads.  Rows beyond the group's members are copies of `start`, so that they come out as zero.
 template <typename T, int R, bool VEC, bool DELTA = false>
-__global__ void __launch_bounds__(kThreads, mma_min_blocks<T, R>())
-gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
-                        const Segment* __restrict__ segments, float* __restrict__ partials,
-                        int groups_total, int group_base, FinishArgs fin, const void* start_ptr)
+__device__ __forceinline__ void gram_segment_mma(const OperandTable& ops, int first, int members, const Segment& seg,
+                                                 float* __restrict__ dst, const void* start_ptr)
 {
-    constexpr int E = gram_entries(R);
     constexpr int V = Element<T>::kVec;          // elements per 16-byte vector
     constexpr int RB = R / 8;                    // blocks of 8 rows
     constexpr int MB = (R + 15) / 16;            // blocks of 16 rows (R = 8: the upper half is zero)
@@ -710,9 +710,6 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
     static_assert(PIECES_PER_ROW % 32 == 0 && kThreads % PIECES_PER_ROW == 0, "a warp copies within one row");
     extern __shared__ __align__(128) unsigned char stage_mem[];
 
-    const Segment seg = segments[blockIdx.x];
-    const int first = blockIdx.y * R;
-    const int members = min(R, operands - first);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
 
@@ -926,7 +923,6 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
         __syncthreads();
     }
     // entries (i <= j) of the packed upper triangle from the accumulator fragments
-    float* dst = partials + ((int64_t)blockIdx.x * groups_total + group_base + blockIdx.y) * E;
     for (int idx = threadIdx.x; idx < R * R; idx += kThreads) {
         const int i = idx / R, j = idx % R;
         if (i > j)
@@ -938,6 +934,23 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
         }
         dst[gram_index(R, i, j)] = v;
     }
+}
+
+// grid = (segments, groups in this launch); block = kThreads; dynamic shared memory =
+// mma_smem_bytes<T, R>().
+template <typename T, int R, bool VEC, bool DELTA = false>
+__global__ void __launch_bounds__(kThreads, mma_min_blocks<T, R>())
+gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
+                        const Segment* __restrict__ segments, float* __restrict__ partials,
+                        int groups_total, int group_base, FinishArgs fin, const void* start_ptr)
+{
+    constexpr int E = gram_entries(R);
+    const Segment seg = segments[blockIdx.x];
+    const int first = blockIdx.y * R;
+    const int members = min(R, operands - first);
+    gram_segment_mma<T, R, VEC, DELTA>(ops, first, members, seg,
+                                       partials + ((int64_t)blockIdx.x * groups_total + group_base + blockIdx.y) * E,
+                                       start_ptr);
     finish_if_last<R>(fin, partials, seg.tensor, group_base + blockIdx.y, groups_total, members);
 }
 
@@ -1511,7 +1524,7 @@ tree_weights_kernel(const double* __restrict__ gram64, int operands, float* __re
 // DELTA: the rows are (operand - ex.start), rounded to T.  ex.base (if any) is added to the sum
 // and the result is stored in ex.out_dtype; dst may be the same buffer as ex.start / ex.base
 // (every element is read by the thread that writes it, before it writes).
-template <typename T, int R, bool VEC, bool DELTA = false>
+template <typename T, int R, bool VEC, bool DELTA = false, int UNROLL = 1>
 __device__ __forceinline__ void weighted_sum_of_segment(const OperandTable& ops, int first, int members,
                                                         const Segment& seg, const float* wsrc,
                                                         void* dst, const PassExtras& ex)
@@ -1542,6 +1555,7 @@ __device__ __forceinline__ void weighted_sum_of_segment(const OperandTable& ops,
     int64_t body_begin, body_end;
     split_segment<V, VEC>(begin, end, body_begin, body_end);
 
+#pragma unroll(UNROLL)
     for (int64_t v = body_begin + (int64_t)threadIdx.x * V; v < body_end; v += (int64_t)kThreads * V) {
         float y[V];
 #pragma unroll
@@ -1775,7 +1789,7 @@ wsum_gram_kernel(const __grid_constant__ OperandTable ops, int operands,
 //
 // grid >= segments; block = kThreads; partials[segment * E + entry].
 
-constexpr int kWarpTensorElems = 2048;
+constexpr int kWarpTensorElems = 512;
 
 // One tensor of at most kShortSlotElems elements: where it starts in the fused buffers, and where in
 // the packed numbering of the short tensors' elements (used for the fp64 vectors that travel
@@ -1883,37 +1897,73 @@ __device__ __forceinline__ void block_reduce_gram(const float (&acc)[E], float* 
     }
 }
 
-// One small tensor, both passes, by one warp.  Element e of row i: ops.ptr[i][begin + e].
-template <typename T, int R, bool DELTA>
+// One small tensor, both passes, by one warp: 16-byte vectors over the aligned body (several
+// independent vectors per lane in flight), scalars for the ragged ends.
+template <typename T, int R, bool VEC, bool DELTA>
 __device__ void reduce_warp_tensor(const OperandTable& ops, int members, const WarpTensor& wt, const TreeOptions& opt,
                                    void* out, const PassExtras& ex)
 {
     constexpr int E = gram_entries(R);
+    constexpr int V = Element<T>::kVec;
+    constexpr int UNROLL = R <= 2 ? 4 : (R <= 4 ? 2 : 1);
     const int lane = threadIdx.x & 31;
     const T* src[R];
 #pragma unroll
     for (int i = 0; i < R; ++i)
-        src[i] = static_cast<const T*>(ops.ptr[i < members ? i : 0]) + wt.begin;
-    const T* start = static_cast<const T*>(ex.start) + wt.begin;
-    auto element = [&](int i, int e) -> float {
+        src[i] = static_cast<const T*>(ops.ptr[i < members ? i : 0]);
+    const T* start = static_cast<const T*>(ex.start);
+    const int64_t begin = wt.begin, end = wt.begin + wt.len;
+    int64_t body_begin, body_end;
+    split_segment<V, VEC>(begin, end, body_begin, body_end);
+    auto element = [&](int i, int64_t e) -> float {
         if constexpr (DELTA)
             return delta_one(src[i], start, e);
         else
             return Element<T>::one(src[i] + e);
     };
+    auto vector = [&](int i, int64_t v, float (&x)[V]) {
+        if constexpr (DELTA)
+            decode_vector<T>(delta_words<T>(load_keep_16B(src[i] + v), load_plain_16B(start + v)), x);
+        else
+            Element<T>::vec(src[i] + v, x);
+    };
     float acc[E];
 #pragma unroll
     for (int k = 0; k < E; ++k)
         acc[k] = 0.0f;
-#pragma unroll 2
-    for (int e = lane; e < wt.len; e += 32) {
-        float col[R];
+#pragma unroll(UNROLL)
+    for (int64_t v = body_begin + (int64_t)lane * V; v < body_end; v += 32 * V) {
+        float x[R][V];
 #pragma unroll
-        for (int i = 0; i < R; ++i)
-            col[i] = i < members ? element(i, e) : 0.0f;
-        gram_accumulate<R>(col, acc);
+        for (int i = 0; i < R; ++i) {
+            if (i < members) {
+                vector(i, v, x[i]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < V; ++j)
+                    x[i][j] = 0.0f;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+            float col[R];
+#pragma unroll
+            for (int i = 0; i < R; ++i)
+                col[i] = x[i][j];
+            gram_accumulate<R>(col, acc);
+        }
     }
-    // the lanes' sums (at most 64 products each) are added in fp64; every lane ends with the same bits
+    for (int pass = 0; pass < 2; ++pass) {
+        const int64_t lo = pass == 0 ? begin : body_end, hi = pass == 0 ? body_begin : end;
+        for (int64_t e = lo + lane; e < hi; e += 32) {
+            float col[R];
+#pragma unroll
+            for (int i = 0; i < R; ++i)
+                col[i] = i < members ? element(i, e) : 0.0f;
+            gram_accumulate<R>(col, acc);
+        }
+    }
+    // the lanes' sums (a few dozen products each) are added in fp64; every lane ends with the same bits
     double gram[E];
 #pragma unroll
     for (int k = 0; k < E; ++k) {
@@ -1935,16 +1985,38 @@ __device__ void reduce_warp_tensor(const OperandTable& ops, int members, const W
 #pragma unroll
     for (int i = 0; i < R; ++i)
         w[i] = i < members ? (float)w64[i] : 0.0f;
-#pragma unroll 2
-    for (int e = lane; e < wt.len; e += 32) {
-        float y = 0.0f;
+#pragma unroll(UNROLL)
+    for (int64_t v = body_begin + (int64_t)lane * V; v < body_end; v += 32 * V) {
+        float y[V];
 #pragma unroll
-        for (int i = 0; i < R; ++i)
-            if (i < members)
-                y = fmaf(w[i], element(i, e), y);
+        for (int j = 0; j < V; ++j)
+            y[j] = 0.0f;
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            if (i < members) {
+                float x[V];
+                vector(i, v, x);
+#pragma unroll
+                for (int j = 0; j < V; ++j)
+                    y[j] = fmaf(w[i], x[j], y[j]);
+            }
+        }
         if (ex.base != nullptr)
-            y += load_as_float(ex.base, ex.base_dtype, wt.begin + e);
-        store_from_float(out, ex.out_dtype, wt.begin + e, y);
+            add_vector_as_float<V>(ex.base, ex.base_dtype, v, y);
+        store_vector_from_float<V>(out, ex.out_dtype, v, y);
+    }
+    for (int pass = 0; pass < 2; ++pass) {
+        const int64_t lo = pass == 0 ? begin : body_end, hi = pass == 0 ? body_begin : end;
+        for (int64_t e = lo + lane; e < hi; e += 32) {
+            float y = 0.0f;
+#pragma unroll
+            for (int i = 0; i < R; ++i)
+                if (i < members)
+                    y = fmaf(w[i], element(i, e), y);
+            if (ex.base != nullptr)
+                y += load_as_float(ex.base, ex.base_dtype, e);
+            store_from_float(out, ex.out_dtype, e, y);
+        }
     }
 }
 
@@ -2058,6 +2130,7 @@ fused_small_kernel(const __grid_constant__ OperandTable ops, int operands,
     constexpr int E = gram_entries(R);
     constexpr int V = Element<T>::kVec;
     constexpr int K = small_keep_vectors<R>();
+    constexpr int kSmallUnroll = R <= 2 ? 4 : (R <= 4 ? 2 : 1);      // vectors per thread in flight where nothing is kept
     __shared__ double short_slots[kWarps][R * kShortSlotElems];
     // This path uses no ticket counters, so the host does not clear them (one operation less in
     // front of a reduce that takes microseconds); the device status word, which lives beside
@@ -2143,8 +2216,8 @@ fused_small_kernel(const __grid_constant__ OperandTable ops, int operands,
         }
         block_reduce_gram<E>(acc, partials + (int64_t)blockIdx.x * E);
     } else if (has_segment) {
-        gram_of_segment<T, R, VEC, DELTA>(ops, 0, members, seg, partials + (int64_t)blockIdx.x * E,
-                                          static_cast<const T*>(ex.start));
+        gram_of_segment<T, R, VEC, DELTA, kSmallUnroll>(ops, 0, members, seg, partials + (int64_t)blockIdx.x * E,
+                                                        static_cast<const T*>(ex.start));
     }
 
     // ---- the small tensors, one warp each, while the segments' loads and stores drain
@@ -2154,7 +2227,7 @@ fused_small_kernel(const __grid_constant__ OperandTable ops, int operands,
         // dealt from the last block backwards: the first blocks are the ones whose segments are longest
         const int first = ((int)gridDim.x - 1 - (int)blockIdx.x) * kWarps + (threadIdx.x >> 5);
         for (int s = first; s < num_warp_tensors; s += warps_total)
-            reduce_warp_tensor<T, R, DELTA>(ops, members, warp_tensors[s], opt, out, ex);
+            reduce_warp_tensor<T, R, VEC, DELTA>(ops, members, warp_tensors[s], opt, out, ex);
         // ... and the tensors of at most 64 elements, in fp64
         for (int s = first; s < num_short_tensors; s += warps_total)
             reduce_short_tensor_warp<T, R, DELTA>(ops, members, short_tensors[s], opt, short_slots[threadIdx.x >> 5],
@@ -2221,7 +2294,7 @@ fused_small_kernel(const __grid_constant__ OperandTable ops, int operands,
             }
         }
     } else {
-        weighted_sum_of_segment<T, R, VEC, DELTA>(ops, 0, members, seg, leaf_weights, out, ex);
+        weighted_sum_of_segment<T, R, VEC, DELTA, kSmallUnroll>(ops, 0, members, seg, leaf_weights, out, ex);
     }
 }
 

@@ -1,6 +1,6 @@
 """The single cooperative launch that serves one-level reduces of at most 8 workers whose operands fit
 the L2: long tensors are cut into one segment per block (operands kept in registers across the grid
-barrier when the segment is short enough), tensors of 65 to 2048 elements are reduced by one warp
+barrier when the segment is short enough), tensors of 65 to 512 elements are reduced by one warp
 each, and those of at most 64 elements by the fp64 kernel.  Against the fp64 oracle at the plain
 tolerance, every tensor."""
 import numpy as np
