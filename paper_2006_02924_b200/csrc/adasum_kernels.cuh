@@ -900,28 +900,33 @@ __device__ __forceinline__ void gram_segment_mma(const OperandTable& ops, int fi
     }
     cp_async_wait<0>();
 
-    // block reduction: the warps add their fragments into shared memory one after the other
-    __shared__ float total[(UBLK + CBLK) * 128];
-#pragma unroll 1
-    for (int w = 0; w < kWarps; ++w) {
-        if (warp == w) {
+    // block reduction: every warp parks its fragments in the (drained) stage memory, then each
+    // slot is added over the warps in warp order
+    constexpr int SLOTS = (UBLK + CBLK) * 128;
+    static_assert((size_t)kWarps * SLOTS * sizeof(float) <= (size_t)STAGES * STAGE_BYTES, "the stages hold the fragments");
+    __shared__ float total[SLOTS];
+    float* slab = reinterpret_cast<float*>(stage_mem) + warp * SLOTS;
+    __syncthreads();                     // every warp has finished reading the stages
 #pragma unroll
-            for (int b = 0; b < UBLK; ++b)
+    for (int b = 0; b < UBLK; ++b)
 #pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const int slot = (b * 4 + r) * 32 + lane;
-                    total[slot] = w == 0 ? acc[b][r] : total[slot] + acc[b][r];
-                }
+        for (int r = 0; r < 4; ++r)
+            slab[(b * 4 + r) * 32 + lane] = acc[b][r];
 #pragma unroll
-            for (int b = 0; b < CBLK; ++b)
+    for (int b = 0; b < CBLK; ++b)
 #pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const int slot = ((UBLK + b) * 4 + r) * 32 + lane;
-                    total[slot] = w == 0 ? acc_c[b][r] : total[slot] + acc_c[b][r];
-                }
-        }
-        __syncthreads();
+        for (int r = 0; r < 4; ++r)
+            slab[((UBLK + b) * 4 + r) * 32 + lane] = acc_c[b][r];
+    __syncthreads();
+    for (int slot = threadIdx.x; slot < SLOTS; slot += kThreads) {
+        const float* column = reinterpret_cast<const float*>(stage_mem) + slot;
+        float sum = column[0];
+#pragma unroll
+        for (int w = 1; w < kWarps; ++w)
+            sum = sum + column[w * SLOTS];
+        total[slot] = sum;
     }
+    __syncthreads();
     // entries (i <= j) of the packed upper triangle from the accumulator fragments
     for (int idx = threadIdx.x; idx < R * R; idx += kThreads) {
         const int i = idx / R, j = idx % R;
