@@ -20,6 +20,8 @@
 //
 // Two more kernels merge neighbouring steps: fused_small_kernel (both passes of a small input in
 // one cooperative launch) and wsum_gram_kernel (pass 2 of a level with pass 1 of the next).
+// Tensors of at most 64 elements are not streamed at all: they are reduced in fp64 with the
+// operator applied literally (adasum_short.cu; one warp each inside fused_small_kernel).
 //
 // No kernel waits on another kernel and none uses floating-point atomics, so results are
 // deterministic.  The only waits are inside a launch: the grid barrier of the cooperative
@@ -676,8 +678,9 @@ __host__ __device__ constexpr size_t mma_smem_bytes()
     return (size_t)mma_stages<T, R>() * (kMmaTileBytes + (DELTA ? kMmaTileBytes / R : 0));
 }
 
-// grid = (segments, groups in this launch); block = kThreads; dynamic shared memory =
-// mma_smem_bytes<T, R>().
+// The Gram matrix of one segment of the group whose first operand is ops.ptr[first], formed by the
+// whole block (kThreads threads, mma_smem_bytes<T, R>() of dynamic shared memory) on the tensor cores
+// and written to dst[0 .. E).
 //
 // Shared-memory layout of a tile: row-major, 64-byte chunk index XOR (row & 1), so that the
 // fragment reads of a quarter warp (two rows, four 16-byte pieces each) fall into distinct banks.

@@ -62,3 +62,40 @@ def test_a_call_survives_the_eviction_of_its_own_table(lib):
     check(lib.adasum_reduce(grads, x_off, flags=2 | (2 << 8)))
     lib.adasum_shutdown()
     check(lib.adasum_reduce(grads, x_off))                  # and everything is rebuilt after a shutdown
+
+
+def test_host_threads_share_the_library(lib):
+    """Several host threads reduce at the same time, each on a stream and a workspace of its own and
+    with tensor tables of its own: the table cache, the pool of side streams (the buffers have tensors
+    of at most 64 elements) and the per-thread error text are shared state."""
+    import threading
+
+    results, errors = {}, []
+
+    def worker(k):
+        try:
+            torch.cuda.set_device(0)
+            stream = torch.cuda.Stream()
+            with torch.cuda.stream(stream):
+                for rep in range(12):
+                    sizes = [30_000 + 64 * k + rep, 9 + k, 64, 5000 + rep, 1]
+                    offsets = workloads.offsets_from_sizes(sizes)
+                    grads = _inputs(12 + k, int(offsets[-1]), seed=6100 + 100 * k + rep)
+                    out = lib.adasum_reduce(grads, offsets, stream=stream)
+                    stream.synchronize()
+                    results[(k, rep)] = (out.double().cpu().numpy(), [g.cpu().numpy() for g in grads], offsets)
+        except Exception as exc:          # noqa: BLE001
+            errors.append((k, repr(exc)))
+
+    threads = [threading.Thread(target=worker, args=(k,)) for k in range(4)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    assert len(results) == 48
+    for (k, rep), (got, arrays, offsets) in results.items():
+        ref = oracle.adasum_reduce(arrays, offsets=offsets, dtype="f32", threads=0)
+        for t in range(len(offsets) - 1):
+            lo, hi = int(offsets[t]), int(offsets[t + 1])
+            assert np.linalg.norm(got[lo:hi] - ref[lo:hi]) <= 1e-5 * np.linalg.norm(ref[lo:hi]), (k, rep, t)
