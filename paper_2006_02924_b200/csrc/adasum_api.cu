@@ -197,9 +197,15 @@ bool plan_levels(int n_workers, adasum_dtype_t dtype, uint32_t flags, LevelPlan*
     return true;
 }
 
+// Blocks that a pass-1 table's tapering is laid out for: two blocks on each of a B200's 148 SMs.
+constexpr int kTaperSlots = 296;
+
+// Upper bound of the segments of a table with this nominal segment length (tapered or not: the
+// shorter segments at both ends of a tapered table add fewer than 4 per slot).
 int64_t segment_bound(int64_t total, int32_t num_tensors, int seg_len)
 {
-    return total / seg_len + 2 * (int64_t)num_tensors + 1;
+    const bool may_taper = total >= 3 * (int64_t)kTaperSlots * seg_len;
+    return total / seg_len + 2 * (int64_t)num_tensors + 1 + (may_taper ? 4 * kTaperSlots : 0);
 }
 
 struct Layout {
@@ -302,8 +308,15 @@ size_t table_device_bytes(const SegmentTable& tab)
 // pass 1 that run last then belong to small tensors, whose per-tensor finish (adding the partial
 // matrices, tree weights) is short, instead of leaving one SM busy with a long tensor's finish
 // while the rest of the GPU idles.  Each tensor's segments stay contiguous, in element order.
+//
+// taper_slots > 0 (pass-1 tables of long buffers): the blocks of a launch are handed out in table
+// order, `taper_slots` at a time.  Segments of one length would leave the machine half empty while
+// the last round of blocks drains, and would keep the two blocks of an SM starting and ending
+// together, pipelines empty at the same moments.  So the segments that the last one and a half
+// rounds would cover are cut at half the length, those of the last half round at a quarter, and
+// the first quarter round at half length, which staggers the blocks that share an SM.
 void build_segments(const int64_t* offsets, int32_t num_tensors, int seg_len, bool skip_short, int warp_limit,
-                    SegmentTable* tab)
+                    int taper_slots, SegmentTable* tab)
 {
     tab->skip_short = skip_short;
     tab->warp_limit = warp_limit;
@@ -335,19 +348,40 @@ void build_segments(const int64_t* offsets, int32_t num_tensors, int seg_len, bo
     // h_seg_first[2 t], h_seg_first[2 t + 1]: first and one-past-last segment of tensor t
     tab->h_seg_first.assign(2 * (size_t)num_tensors + 2, 0);
     tab->max_segments_per_tensor = 0;
+    const auto in_segments = [&](int32_t t) {
+        const int64_t len = offsets[t + 1] - offsets[t];
+        return !((skip_short && len <= kShortTensorElems) || len <= warp_limit);
+    };
+    int64_t left = 0;           // elements that the segments from here to the end of the table cover
+    for (int32_t t = 0; t < num_tensors; ++t)
+        left += in_segments(t) ? offsets[t + 1] - offsets[t] : 0;
+    const int64_t round = (int64_t)taper_slots * seg_len;
+    if (left < 3 * round || seg_len % 256 != 0)
+        taper_slots = 0;        // too short a launch to have a middle
+    tab->taper_slots = taper_slots;
+    int64_t done = 0;
     for (int32_t t : order) {
         tab->h_seg_first[2 * (size_t)t] = (int32_t)tab->h_segments.size();
         int64_t b = offsets[t];
         const int64_t e = offsets[t + 1];
-        if ((skip_short && e - b <= kShortTensorElems) || e - b <= warp_limit)
+        if (!in_segments(t))
             b = e;
         while (b < e) {
+            int64_t len = seg_len;
+            if (taper_slots > 0) {
+                if (left <= round / 2)
+                    len = seg_len / 4;
+                else if (left <= round + round / 2 || done < round / 4)
+                    len = seg_len / 2;
+            }
             // cut on a 64-element grid of the fused buffer so that interior cuts keep 16-byte
             // alignment whatever the tensor's own start
-            int64_t next = b / 64 * 64 + seg_len;
+            int64_t next = b / 64 * 64 + len;
             if (next > e)
                 next = e;
             tab->h_segments.push_back(Segment{b, (int32_t)(next - b), t});
+            done += next - b;
+            left -= next - b;
             b = next;
         }
         tab->h_seg_first[2 * (size_t)t + 1] = (int32_t)tab->h_segments.size();
@@ -361,7 +395,7 @@ void build_segments(const int64_t* offsets, int32_t num_tensors, int seg_len, bo
 // The table for (current device, offsets, seg_len), built and uploaded on first use.  The caller
 // keeps the returned reference until it has enqueued its last launch that reads the table.
 adasum_status_t get_segment_table(const int64_t* offsets, int32_t num_tensors, int seg_len, bool skip_short,
-                                  TableRef* out, int warp_limit = 0)
+                                  TableRef* out, int warp_limit = 0, int taper_slots = 0)
 {
     int device = 0;
     ADASUM_CUDA_CHECK(cudaGetDevice(&device));
@@ -370,7 +404,7 @@ adasum_status_t get_segment_table(const int64_t* offsets, int32_t num_tensors, i
     for (size_t i = 0; i < g_tables.size(); ++i) {
         const SegmentTable& tab = *g_tables[i];
         if (tab.device == device && tab.seg_len == seg_len && tab.skip_short == skip_short &&
-            tab.warp_limit == warp_limit &&
+            tab.warp_limit == warp_limit && tab.taper_request == taper_slots &&
             tab.offsets.size() == (size_t)num_tensors + 1 &&
             std::memcmp(tab.offsets.data(), offsets, sizeof(int64_t) * tab.offsets.size()) == 0) {
             // most recently used last
@@ -383,7 +417,8 @@ adasum_status_t get_segment_table(const int64_t* offsets, int32_t num_tensors, i
     tab->device = device;
     tab->seg_len = seg_len;
     tab->offsets.assign(offsets, offsets + num_tensors + 1);
-    build_segments(offsets, num_tensors, seg_len, skip_short, warp_limit, tab.get());
+    tab->taper_request = taper_slots;
+    build_segments(offsets, num_tensors, seg_len, skip_short, warp_limit, taper_slots, tab.get());
     const size_t seg_bytes = sizeof(Segment) * (tab->h_segments.size() + 1);
     const size_t first_bytes = sizeof(int32_t) * tab->h_seg_first.size();
     const size_t short_bytes = sizeof(ShortTensor) * (tab->h_short.size() + 1) +
@@ -911,7 +946,8 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         const bool simple_kernels = (flags & ADASUM_FLAG_SIMPLE_KERNELS) != 0;
         const GramKind kind = gram_kind(lv.radix, simple_kernels);
         TableRef gram_tab, wsum_tab, fuse_tab;     // held until this level's launches are enqueued
-        st = get_segment_table(offsets, num_tensors, gram_segment_length(kind, total), skip_short, &gram_tab);
+        st = get_segment_table(offsets, num_tensors, gram_segment_length(kind, total), skip_short, &gram_tab, 0,
+                               kTaperSlots);
         if (st != ADASUM_OK)
             return st;
         st = get_segment_table(offsets, num_tensors, wsum_segment_length(total), skip_short, &wsum_tab);
@@ -1338,7 +1374,7 @@ adasum_status_t pair_noalloc_impl(const void* a, const void* b, const int64_t* o
     if (st != ADASUM_OK)
         return st;
     SegmentTable tab;                       // host-side only; its device pointers aim into the scratch
-    build_segments(offsets, num_tensors, kNoallocSegLen, true, 0, &tab);      // short tensors apart, as in adasum_pair
+    build_segments(offsets, num_tensors, kNoallocSegLen, true, 0, 0, &tab);      // short tensors apart, as in adasum_pair
     if ((int64_t)tab.num_segments > kNoallocMaxSegments)
         return fail(ADASUM_ERR_ARG, "segment table does not fit the static scratch");
     tab.d_segments = reinterpret_cast<Segment*>(scratch);

@@ -93,6 +93,9 @@ struct SegmentTable {
     // Tensors of at most warp_limit elements (beyond the short ones), when the single-launch kernel
     // gives each of them to one warp: no segments either.
     int warp_limit = 0;
+    // Tapered cutting (shorter segments at both ends of the table): what the table was asked for
+    // (part of its identity in the cache) and what it was built with (0 if the buffer is too short).
+    int taper_request = 0, taper_slots = 0;
     WarpTensor* d_warp = nullptr;
     std::vector<WarpTensor> h_warp;
 

@@ -678,238 +678,245 @@ __host__ __device__ constexpr size_t mma_smem_bytes()
     return (size_t)mma_stages<T, R>() * (kMmaTileBytes + (DELTA ? kMmaTileBytes / R : 0));
 }
 
-// The Gram matrix of one segment of the group whose first operand is ops.ptr[first], formed by the
-// whole block (kThreads threads, mma_smem_bytes<T, R>() of dynamic shared memory) on the tensor cores
-// and written to dst[0 .. E).
+// Sizes of the tensor-core Gram pass that its pieces below share.
+template <typename T, int R, bool DELTA>
+struct MmaShape {
+    static constexpr int V = Element<T>::kVec;          // elements per 16-byte vector
+    static constexpr int RB = R / 8;                    // blocks of 8 rows
+    static constexpr int MB = (R + 15) / 16;            // blocks of 16 rows (R = 8: the upper half is zero)
+    static constexpr int RBP = 2 * MB;                  // row blocks the fragments are indexed with
+    static constexpr int UBLK = mma_upper_blocks<R>();
+    static constexpr bool SPLIT = sizeof(T) == 4;
+    static constexpr int CBLK = SPLIT ? mma_all_blocks<R>() : 0;
+    static constexpr int CDIM = SPLIT ? CBLK : 1;
+    static constexpr int DEPTH = mma_depth<T, R>();
+    static constexpr int STAGES = mma_stages<T, R>();
+    static constexpr int ROW_BYTES = kMmaTileBytes / R;
+    static constexpr int STAGE_BYTES = kMmaTileBytes + (DELTA ? ROW_BYTES : 0);
+    static constexpr int PIECES_PER_ROW = ROW_BYTES / 16;
+    static constexpr int TILE_ELEMS = PIECES_PER_ROW * V;               // elements of one row in a tile
+    static constexpr int PIECES = kMmaTileBytes / 16 / kThreads;        // 16-byte pieces a thread copies per tile
+    static constexpr int ROWS_PER_PASS = kThreads / PIECES_PER_ROW;     // piece i of a thread is in row row0 + i * this
+    static constexpr int SLOTS = (UBLK + CBLK) * 128;                   // accumulator words of a warp
+    static constexpr int SLAB_BYTES = kWarps * SLOTS * (int)sizeof(float);
+    static_assert(DEPTH * kWarps * 64 == ROW_BYTES, "a tile row is split evenly among the warps");
+    static_assert(PIECES_PER_ROW % 32 == 0 && kThreads % PIECES_PER_ROW == 0, "a warp copies within one row");
+    static_assert(SLAB_BYTES <= STAGES * STAGE_BYTES, "the stages hold the fragments");
+};
+
+// Copy side of the tensor-core Gram pass: piece i of this thread is (row0 + i * ROWS_PER_PASS, col0)
+// of every tile.
 //
 // Shared-memory layout of a tile: row-major, 64-byte chunk index XOR (row & 1), so that the
 // fragment reads of a quarter warp (two rows, four 16-byte pieces each) fall into distinct banks.
-// The pipeline is the usual multi-stage one: wait for the oldest copy group, one __syncthreads
-// per tile, refill the slot that was consumed in the previous iteration.
 //
 // DELTA: the rows are (operand - start), rounded to T.  The tile gets one more row, unswizzled,
 // with the same columns of `start`; a lane subtracts its 16 bytes of it from every fragment it
 // loads.  Rows beyond the group's members are copies of `start`, so that they come out as zero.
-template <typename T, int R, bool VEC, bool DELTA = false>
-__device__ __forceinline__ void gram_segment_mma(const OperandTable& ops, int first, int members, const Segment& seg,
-                                                 float* __restrict__ dst, const void* start_ptr)
-{
-    constexpr int V = Element<T>::kVec;          // elements per 16-byte vector
-    constexpr int RB = R / 8;                    // blocks of 8 rows
-    constexpr int MB = (R + 15) / 16;            // blocks of 16 rows (R = 8: the upper half is zero)
-    constexpr int RBP = 2 * MB;                  // row blocks the fragments are indexed with
-    constexpr int UBLK = mma_upper_blocks<R>();
-    constexpr bool SPLIT = sizeof(T) == 4;
-    constexpr int CBLK = SPLIT ? mma_all_blocks<R>() : 0;
-    constexpr int DEPTH = mma_depth<T, R>();
-    constexpr int STAGES = mma_stages<T, R>();
-    constexpr int ROW_BYTES = kMmaTileBytes / R;
-    constexpr int STAGE_BYTES = kMmaTileBytes + (DELTA ? ROW_BYTES : 0);
-    constexpr int PIECES_PER_ROW = ROW_BYTES / 16;
-    constexpr int TILE_ELEMS = PIECES_PER_ROW * V;               // elements of one row in a tile
-    constexpr int PIECES = kMmaTileBytes / 16 / kThreads;        // 16-byte pieces a thread copies per tile
-    constexpr int ROWS_PER_PASS = kThreads / PIECES_PER_ROW;     // piece i of a thread is in row row0 + i * this
-    static_assert(DEPTH * kWarps * 64 == ROW_BYTES, "a tile row is split evenly among the warps");
-    static_assert(PIECES_PER_ROW % 32 == 0 && kThreads % PIECES_PER_ROW == 0, "a warp copies within one row");
-    extern __shared__ __align__(128) unsigned char stage_mem[];
+template <typename T, int R, bool VEC, bool DELTA>
+struct MmaCopier {
+    using S = MmaShape<T, R, DELTA>;
+    const T* src[S::PIECES];     // row pointer + this thread's column; rows beyond the members alias row 0
+    const T* start_src;          // DELTA: threads of row0 == 0 copy it
+    uint32_t smem_base;
+    int row0, col0, members;
+    bool full_group;
 
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int g = lane >> 2, t = lane & 3;
-
-    const int64_t begin = seg.begin, end = seg.begin + seg.len;
-    const int64_t k0 = VEC ? begin / V * V : begin;
-    const int ntiles = (int)((end - k0 + TILE_ELEMS - 1) / TILE_ELEMS);
-
-    // ---- copy side: piece i of this thread is (row0 + i * ROWS_PER_PASS, col0) of the tile
-    const uint32_t smem_base = static_cast<uint32_t>(__cvta_generic_to_shared(stage_mem));
-    const int row0 = threadIdx.x / PIECES_PER_ROW, col0 = threadIdx.x % PIECES_PER_ROW;
-    // byte offset of piece i inside a tile (the swizzle depends on the row's parity)
-    auto copy_off = [&](int i) -> uint32_t {
-        const int row = row0 + i * ROWS_PER_PASS;
-        return row * ROW_BYTES + (((col0 >> 2) ^ (row & 1)) << 6) + ((col0 & 3) << 4);
-    };
-    const T* copy_src[PIECES];     // row pointer + this thread's column; rows beyond the members alias row 0
+    __device__ __forceinline__ void init(const OperandTable& ops, int first, int members_, const void* start_ptr,
+                                         uint32_t smem_base_)
+    {
+        smem_base = smem_base_;
+        members = members_;
+        row0 = threadIdx.x / S::PIECES_PER_ROW;
+        col0 = threadIdx.x % S::PIECES_PER_ROW;
 #pragma unroll
-    for (int i = 0; i < PIECES; ++i) {
-        const int row = row0 + i * ROWS_PER_PASS;
-        copy_src[i] = static_cast<const T*>(ops.ptr[first + (row < members ? row : 0)]) + col0 * V;
-        if (DELTA && row >= members)
-            copy_src[i] = static_cast<const T*>(start_ptr) + col0 * V;
+        for (int i = 0; i < S::PIECES; ++i) {
+            const int row = row0 + i * S::ROWS_PER_PASS;
+            src[i] = static_cast<const T*>(ops.ptr[first + (row < members ? row : 0)]) + col0 * S::V;
+            if (DELTA && row >= members)
+                src[i] = static_cast<const T*>(start_ptr) + col0 * S::V;
+        }
+        start_src = static_cast<const T*>(start_ptr) + col0 * S::V;
+        full_group = members == R || DELTA;
     }
-    const T* start_src = static_cast<const T*>(start_ptr) + col0 * V;      // DELTA: threads of row0 == 0 copy it
-    const bool full_group = members == R || DELTA;
-
-    auto issue = [&](int tile, int stage) {
-        if (tile < ntiles) {
-            const uint32_t dst = smem_base + stage * STAGE_BYTES;
-            const int64_t tile_elem0 = k0 + (int64_t)tile * TILE_ELEMS;
-            if (VEC && full_group && tile_elem0 >= begin && tile_elem0 + TILE_ELEMS <= end) {
+    // byte offset of piece i inside a tile (the swizzle depends on the row's parity)
+    __device__ __forceinline__ uint32_t piece_offset(int i) const
+    {
+        const int row = row0 + i * S::ROWS_PER_PASS;
+        return row * S::ROW_BYTES + (((col0 >> 2) ^ (row & 1)) << 6) + ((col0 & 3) << 4);
+    }
+    // Starts the copy of the tile whose first element is tile_elem0 into `stage` (elements outside
+    // [begin, end) become zero).  The caller commits the copy group.
+    __device__ __forceinline__ void issue(int64_t begin, int64_t end, int64_t tile_elem0, int stage) const
+    {
+        const uint32_t dst = smem_base + stage * S::STAGE_BYTES;
+        if (VEC && full_group && tile_elem0 >= begin && tile_elem0 + S::TILE_ELEMS <= end) {
 #pragma unroll
-                for (int i = 0; i < PIECES; ++i)
-                    cp_async_16B_shared(dst + copy_off(i), copy_src[i] + tile_elem0);
-                if (DELTA && row0 == 0)
+            for (int i = 0; i < S::PIECES; ++i)
+                cp_async_16B_shared(dst + piece_offset(i), src[i] + tile_elem0);
+            if (DELTA && row0 == 0)
+                cp_async_16B_shared(dst + kMmaTileBytes + (col0 << 4), start_src + tile_elem0);
+        } else {
+            // ragged tile, partial group or unaligned buffers: test every piece
+            const int64_t e0 = tile_elem0 + (int64_t)col0 * S::V;
+            const bool whole = VEC && e0 >= begin && e0 + S::V <= end;
+#pragma unroll
+            for (int i = 0; i < S::PIECES; ++i) {
+                const uint32_t slot = dst + piece_offset(i);
+                if (!DELTA && row0 + i * S::ROWS_PER_PASS >= members)
+                    store_shared_16B(slot, make_uint4(0u, 0u, 0u, 0u));
+                else if (whole)
+                    cp_async_16B_shared(slot, src[i] + tile_elem0);
+                else
+                    store_shared_16B(slot, load_masked_words<T>(src[i] - col0 * S::V, e0, begin, end));
+            }
+            if (DELTA && row0 == 0) {
+                if (whole)
                     cp_async_16B_shared(dst + kMmaTileBytes + (col0 << 4), start_src + tile_elem0);
-            } else {
-                // ragged tile, partial group or unaligned buffers: test every piece
-                const int64_t e0 = tile_elem0 + (int64_t)col0 * V;
-                const bool whole = VEC && e0 >= begin && e0 + V <= end;
-#pragma unroll
-                for (int i = 0; i < PIECES; ++i) {
-                    const uint32_t slot = dst + copy_off(i);
-                    if (!DELTA && row0 + i * ROWS_PER_PASS >= members)
-                        store_shared_16B(slot, make_uint4(0u, 0u, 0u, 0u));
-                    else if (whole)
-                        cp_async_16B_shared(slot, copy_src[i] + tile_elem0);
-                    else
-                        store_shared_16B(slot, load_masked_words<T>(copy_src[i] - col0 * V, e0, begin, end));
-                }
-                if (DELTA && row0 == 0) {
-                    if (whole)
-                        cp_async_16B_shared(dst + kMmaTileBytes + (col0 << 4), start_src + tile_elem0);
-                    else
-                        store_shared_16B(dst + kMmaTileBytes + (col0 << 4),
-                                         load_masked_words<T>(start_src - col0 * V, e0, begin, end));
-                }
+                else
+                    store_shared_16B(dst + kMmaTileBytes + (col0 << 4),
+                                     load_masked_words<T>(start_src - col0 * S::V, e0, begin, end));
             }
         }
-        cp_async_commit();
-    };
+    }
+};
 
-    // ---- multiply side
-    const uint32_t frag_off = g * ROW_BYTES + (t << 4);
+// Multiply side: adds the products of the tile in `stage` to the warp's accumulators.  `acc` are
+// the accumulators themselves for 16-bit inputs and the rounded sums of H for fp32, `acc_c` the
+// rounded sums of C (fp32 only).
+template <typename T, int R, bool DELTA>
+__device__ __forceinline__ void mma_multiply_tile(uint32_t stage_addr, int warp, int g, int t,
+                                                  float (&acc)[MmaShape<T, R, DELTA>::UBLK][4],
+                                                  float (&acc_c)[MmaShape<T, R, DELTA>::CDIM][4])
+{
+    using S = MmaShape<T, R, DELTA>;
+    constexpr int RB = S::RB, MB = S::MB, RBP = S::RBP, UBLK = S::UBLK, CBLK = S::CBLK, DEPTH = S::DEPTH;
+    constexpr int ROW_BYTES = S::ROW_BYTES;
+    const uint32_t src_stage = stage_addr + g * ROW_BYTES + (t << 4);
+    const uint32_t start_stage = stage_addr + kMmaTileBytes + (t << 4);
     uint32_t chunk_off[DEPTH];
 #pragma unroll
     for (int d = 0; d < DEPTH; ++d)
         chunk_off[d] = ((warp * DEPTH + d) ^ (g & 1)) << 6;
 
-    float acc[UBLK][4];                            // 16-bit inputs: the accumulators; fp32: rounded sums of H
-    float acc_c[SPLIT ? CBLK : 1][4];              // fp32: rounded sums of C
+    if constexpr (!S::SPLIT) {
 #pragma unroll
-    for (int b = 0; b < UBLK; ++b)
+        for (int d = 0; d < DEPTH; ++d) {
+            uint32_t w[RBP][4];
+            uint4 sv = make_uint4(0u, 0u, 0u, 0u);
+            if constexpr (DELTA)
+                sv = load_shared_16B(start_stage + ((warp * DEPTH + d) << 6));
+#pragma unroll
+            for (int rb = 0; rb < RBP; ++rb) {
+                uint4 v = rb < RB ? load_shared_16B(src_stage + chunk_off[d] + rb * 8 * ROW_BYTES)
+                                  : make_uint4(0u, 0u, 0u, 0u);
+                if (DELTA && rb < RB)
+                    v = delta_words<T>(v, sv);
+                w[rb][0] = v.x; w[rb][1] = v.y; w[rb][2] = v.z; w[rb][3] = v.w;
+            }
+#pragma unroll
+            for (int step = 0; step < 2; ++step) {
+#pragma unroll
+                for (int mb = 0; mb < MB; ++mb)
+#pragma unroll
+                    for (int nb = 2 * mb; nb < RB; ++nb)
+                        mma_step<T>(acc[mma_upper_index<R>(mb, nb)], w[2 * mb][2 * step], w[2 * mb + 1][2 * step],
+                                    w[2 * mb][2 * step + 1], w[2 * mb + 1][2 * step + 1], w[nb][2 * step],
+                                    w[nb][2 * step + 1]);
+            }
+        }
+    } else {
+        float tile_h[UBLK][4], tile_c[S::CDIM][4];
+#pragma unroll
+        for (int b = 0; b < UBLK; ++b)
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+                tile_h[b][r] = 0.0f;
+#pragma unroll
+        for (int b = 0; b < CBLK; ++b)
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+                tile_c[b][r] = 0.0f;
+#pragma unroll
+        for (int d = 0; d < DEPTH; ++d) {
+            uint32_t hi[RBP][4], lo[RBP][4];
+            uint4 sv = make_uint4(0u, 0u, 0u, 0u);
+            if constexpr (DELTA)
+                sv = load_shared_16B(start_stage + ((warp * DEPTH + d) << 6));
+#pragma unroll
+            for (int rb = 0; rb < RBP; ++rb) {
+                uint4 v = rb < RB ? load_shared_16B(src_stage + chunk_off[d] + rb * 8 * ROW_BYTES)
+                                  : make_uint4(0u, 0u, 0u, 0u);
+                if (DELTA && rb < RB)
+                    v = delta_words<T>(v, sv);
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    // nearest tf32 by integer arithmetic (the conversion instruction runs on
+                    // the slow special-function pipe): add half a tf32 ulp, drop 13 bits
+                    hi[rb][j] = (w[j] + 0x1000u) & 0xffffe000u;
+                    lo[rb][j] = __float_as_uint(__uint_as_float(w[j]) - __uint_as_float(hi[rb][j]));
+                }
+            }
+#pragma unroll
+            for (int step = 0; step < 2; ++step) {
+#pragma unroll
+                for (int mb = 0; mb < MB; ++mb) {
+#pragma unroll
+                    for (int nb = 0; nb < RB; ++nb) {
+                        if (nb >= 2 * mb)
+                            mma_step<T>(tile_h[mma_upper_index<R>(mb, nb)], hi[2 * mb][2 * step],
+                                        hi[2 * mb + 1][2 * step], hi[2 * mb][2 * step + 1],
+                                        hi[2 * mb + 1][2 * step + 1], hi[nb][2 * step], hi[nb][2 * step + 1]);
+                        mma_step<T>(tile_c[mb * RB + nb], hi[2 * mb][2 * step], hi[2 * mb + 1][2 * step],
+                                    hi[2 * mb][2 * step + 1], hi[2 * mb + 1][2 * step + 1], lo[nb][2 * step],
+                                    lo[nb][2 * step + 1]);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int b = 0; b < UBLK; ++b)
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+                acc[b][r] += tile_h[b][r];
+#pragma unroll
+        for (int b = 0; b < CBLK; ++b)
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+                acc_c[b][r] += tile_c[b][r];
+    }
+}
+
+template <typename T, int R, bool DELTA>
+__device__ __forceinline__ void mma_clear(float (&acc)[MmaShape<T, R, DELTA>::UBLK][4],
+                                          float (&acc_c)[MmaShape<T, R, DELTA>::CDIM][4])
+{
+    using S = MmaShape<T, R, DELTA>;
+#pragma unroll
+    for (int b = 0; b < S::UBLK; ++b)
 #pragma unroll
         for (int r = 0; r < 4; ++r)
             acc[b][r] = 0.0f;
 #pragma unroll
-    for (int b = 0; b < (SPLIT ? CBLK : 1); ++b)
+    for (int b = 0; b < S::CDIM; ++b)
 #pragma unroll
         for (int r = 0; r < 4; ++r)
             acc_c[b][r] = 0.0f;
+}
 
-#pragma unroll
-    for (int st = 0; st < STAGES - 1; ++st)
-        issue(st, st);
-
-    int stage = 0;
-    for (int tile = 0; tile < ntiles; ++tile) {
-        cp_async_wait<STAGES - 2>();     // this thread's copies for `tile` have landed
-        __syncthreads();                 // ... and everybody's; the previous tile's slot is free
-        int refill = stage + STAGES - 1;
-        if (refill >= STAGES)
-            refill -= STAGES;
-        issue(tile + STAGES - 1, refill);
-
-        const uint32_t src_stage = smem_base + stage * STAGE_BYTES + frag_off;
-        const uint32_t start_stage = smem_base + stage * STAGE_BYTES + kMmaTileBytes + (t << 4);
-        if (++stage == STAGES)
-            stage = 0;
-
-        if constexpr (!SPLIT) {
-#pragma unroll
-            for (int d = 0; d < DEPTH; ++d) {
-                uint32_t w[RBP][4];
-                uint4 sv = make_uint4(0u, 0u, 0u, 0u);
-                if constexpr (DELTA)
-                    sv = load_shared_16B(start_stage + ((warp * DEPTH + d) << 6));
-#pragma unroll
-                for (int rb = 0; rb < RBP; ++rb) {
-                    uint4 v = rb < RB ? load_shared_16B(src_stage + chunk_off[d] + rb * 8 * ROW_BYTES)
-                                      : make_uint4(0u, 0u, 0u, 0u);
-                    if (DELTA && rb < RB)
-                        v = delta_words<T>(v, sv);
-                    w[rb][0] = v.x; w[rb][1] = v.y; w[rb][2] = v.z; w[rb][3] = v.w;
-                }
-#pragma unroll
-                for (int step = 0; step < 2; ++step) {
-#pragma unroll
-                    for (int mb = 0; mb < MB; ++mb)
-#pragma unroll
-                        for (int nb = 2 * mb; nb < RB; ++nb)
-                            mma_step<T>(acc[mma_upper_index<R>(mb, nb)], w[2 * mb][2 * step], w[2 * mb + 1][2 * step],
-                                        w[2 * mb][2 * step + 1], w[2 * mb + 1][2 * step + 1], w[nb][2 * step],
-                                        w[nb][2 * step + 1]);
-                }
-            }
-        } else {
-            float tile_h[UBLK][4], tile_c[SPLIT ? CBLK : 1][4];
-#pragma unroll
-            for (int b = 0; b < UBLK; ++b)
-#pragma unroll
-                for (int r = 0; r < 4; ++r)
-                    tile_h[b][r] = 0.0f;
-#pragma unroll
-            for (int b = 0; b < CBLK; ++b)
-#pragma unroll
-                for (int r = 0; r < 4; ++r)
-                    tile_c[b][r] = 0.0f;
-#pragma unroll
-            for (int d = 0; d < DEPTH; ++d) {
-                uint32_t hi[RBP][4], lo[RBP][4];
-                uint4 sv = make_uint4(0u, 0u, 0u, 0u);
-                if constexpr (DELTA)
-                    sv = load_shared_16B(start_stage + ((warp * DEPTH + d) << 6));
-#pragma unroll
-                for (int rb = 0; rb < RBP; ++rb) {
-                    uint4 v = rb < RB ? load_shared_16B(src_stage + chunk_off[d] + rb * 8 * ROW_BYTES)
-                                      : make_uint4(0u, 0u, 0u, 0u);
-                    if (DELTA && rb < RB)
-                        v = delta_words<T>(v, sv);
-                    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        // nearest tf32 by integer arithmetic (the conversion instruction runs on
-                        // the slow special-function pipe): add half a tf32 ulp, drop 13 bits
-                        hi[rb][j] = (w[j] + 0x1000u) & 0xffffe000u;
-                        lo[rb][j] = __float_as_uint(__uint_as_float(w[j]) - __uint_as_float(hi[rb][j]));
-                    }
-                }
-#pragma unroll
-                for (int step = 0; step < 2; ++step) {
-#pragma unroll
-                    for (int mb = 0; mb < MB; ++mb) {
-#pragma unroll
-                        for (int nb = 0; nb < RB; ++nb) {
-                            if (nb >= 2 * mb)
-                                mma_step<T>(tile_h[mma_upper_index<R>(mb, nb)], hi[2 * mb][2 * step],
-                                            hi[2 * mb + 1][2 * step], hi[2 * mb][2 * step + 1],
-                                            hi[2 * mb + 1][2 * step + 1], hi[nb][2 * step], hi[nb][2 * step + 1]);
-                            mma_step<T>(tile_c[mb * RB + nb], hi[2 * mb][2 * step], hi[2 * mb + 1][2 * step],
-                                        hi[2 * mb][2 * step + 1], hi[2 * mb + 1][2 * step + 1], lo[nb][2 * step],
-                                        lo[nb][2 * step + 1]);
-                        }
-                    }
-                }
-            }
-#pragma unroll
-            for (int b = 0; b < UBLK; ++b)
-#pragma unroll
-                for (int r = 0; r < 4; ++r)
-                    acc[b][r] += tile_h[b][r];
-#pragma unroll
-            for (int b = 0; b < CBLK; ++b)
-#pragma unroll
-                for (int r = 0; r < 4; ++r)
-                    acc_c[b][r] += tile_c[b][r];
-        }
-    }
-    cp_async_wait<0>();
-
-    // block reduction: every warp parks its fragments in the (drained) stage memory, then each
-    // slot is added over the warps in warp order
-    constexpr int SLOTS = (UBLK + CBLK) * 128;
-    static_assert((size_t)kWarps * SLOTS * sizeof(float) <= (size_t)STAGES * STAGE_BYTES, "the stages hold the fragments");
-    __shared__ float total[SLOTS];
-    float* slab = reinterpret_cast<float*>(stage_mem) + warp * SLOTS;
-    __syncthreads();                     // every warp has finished reading the stages
+// Block reduction, first half: every warp parks its fragments in `slab_base` (SLAB_BYTES of shared
+// memory that nobody else is using: stage memory whose tile has been consumed).  Begins with a
+// barrier (every warp has finished reading the stage that becomes the slab).
+template <typename T, int R, bool DELTA>
+__device__ __forceinline__ void mma_park(float* slab_base, int warp, int lane,
+                                         const float (&acc)[MmaShape<T, R, DELTA>::UBLK][4],
+                                         const float (&acc_c)[MmaShape<T, R, DELTA>::CDIM][4])
+{
+    using S = MmaShape<T, R, DELTA>;
+    constexpr int UBLK = S::UBLK, CBLK = S::CBLK, SLOTS = S::SLOTS;
+    float* slab = slab_base + warp * SLOTS;
+    __syncthreads();
 #pragma unroll
     for (int b = 0; b < UBLK; ++b)
 #pragma unroll
@@ -920,9 +927,20 @@ __device__ __forceinline__ void gram_segment_mma(const OperandTable& ops, int fi
 #pragma unroll
         for (int r = 0; r < 4; ++r)
             slab[((UBLK + b) * 4 + r) * 32 + lane] = acc_c[b][r];
+}
+
+// Second half: each slot is added over the warps in warp order and the packed upper triangle is
+// written to dst[0 .. E).  The slab is free again once every thread has passed this function's
+// last barrier, i.e. on return.
+template <typename T, int R, bool DELTA>
+__device__ __forceinline__ void mma_sum_store(const float* slab_base, float* __restrict__ dst)
+{
+    using S = MmaShape<T, R, DELTA>;
+    constexpr int UBLK = S::UBLK, SLOTS = S::SLOTS, RB = S::RB;
+    __shared__ float total[SLOTS];
     __syncthreads();
     for (int slot = threadIdx.x; slot < SLOTS; slot += kThreads) {
-        const float* column = reinterpret_cast<const float*>(stage_mem) + slot;
+        const float* column = slab_base + slot;
         float sum = column[0];
 #pragma unroll
         for (int w = 1; w < kWarps; ++w)
@@ -936,12 +954,66 @@ __device__ __forceinline__ void gram_segment_mma(const OperandTable& ops, int fi
         if (i > j)
             continue;
         float v = total[mma_upper_index<R>(i / 16, j / 8) * 128 + mma_fragment_slot(i % 16, j % 8)];
-        if (SPLIT) {
+        if (S::SPLIT) {
             v += total[(UBLK + (i / 16) * RB + j / 8) * 128 + mma_fragment_slot(i % 16, j % 8)];   // C_ij
             v += total[(UBLK + (j / 16) * RB + i / 8) * 128 + mma_fragment_slot(j % 16, i % 8)];   // C_ji
         }
         dst[gram_index(R, i, j)] = v;
     }
+}
+
+// The Gram matrix of one segment of the group whose first operand is ops.ptr[first], formed by the
+// whole block (kThreads threads, mma_smem_bytes<T, R>() of dynamic shared memory) on the tensor cores
+// and written to dst[0 .. E).
+//
+// The pipeline is the usual multi-stage one: wait for the oldest copy group, one __syncthreads
+// per tile, refill the slot that was consumed in the previous iteration.
+template <typename T, int R, bool VEC, bool DELTA = false>
+__device__ __forceinline__ void gram_segment_mma(const OperandTable& ops, int first, int members, const Segment& seg,
+                                                 float* __restrict__ dst, const void* start_ptr)
+{
+    using S = MmaShape<T, R, DELTA>;
+    constexpr int STAGES = S::STAGES;
+    extern __shared__ __align__(128) unsigned char stage_mem[];
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, t = lane & 3;
+
+    const int64_t begin = seg.begin, end = seg.begin + seg.len;
+    const int64_t k0 = VEC ? begin / S::V * S::V : begin;
+    const int ntiles = (int)((end - k0 + S::TILE_ELEMS - 1) / S::TILE_ELEMS);
+
+    const uint32_t smem_base = static_cast<uint32_t>(__cvta_generic_to_shared(stage_mem));
+    MmaCopier<T, R, VEC, DELTA> copier;
+    copier.init(ops, first, members, start_ptr, smem_base);
+    auto issue = [&](int tile, int stage) {
+        if (tile < ntiles)
+            copier.issue(begin, end, k0 + (int64_t)tile * S::TILE_ELEMS, stage);
+        cp_async_commit();
+    };
+
+    float acc[S::UBLK][4], acc_c[S::CDIM][4];
+    mma_clear<T, R, DELTA>(acc, acc_c);
+
+#pragma unroll
+    for (int st = 0; st < STAGES - 1; ++st)
+        issue(st, st);
+
+    int stage = 0;
+    for (int tile = 0; tile < ntiles; ++tile) {
+        cp_async_wait<STAGES - 2>();     // this thread's copies for `tile` have landed
+        __syncthreads();                 // ... and everybody's; the previous tile's slot is free
+        int refill = stage + STAGES - 1;
+        if (refill >= STAGES)
+            refill -= STAGES;
+        issue(tile + STAGES - 1, refill);
+        mma_multiply_tile<T, R, DELTA>(smem_base + stage * S::STAGE_BYTES, warp, g, t, acc, acc_c);
+        if (++stage == STAGES)
+            stage = 0;
+    }
+    cp_async_wait<0>();
+    mma_park<T, R, DELTA>(reinterpret_cast<float*>(stage_mem), warp, lane, acc, acc_c);
+    mma_sum_store<T, R, DELTA>(reinterpret_cast<const float*>(stage_mem), dst);
 }
 
 // grid = (segments, groups in this launch); block = kThreads; dynamic shared memory =
