@@ -99,3 +99,31 @@ def test_host_threads_share_the_library(lib):
         for t in range(len(offsets) - 1):
             lo, hi = int(offsets[t]), int(offsets[t + 1])
             assert np.linalg.norm(got[lo:hi] - ref[lo:hi]) <= 1e-5 * np.linalg.norm(ref[lo:hi]), (k, rep, t)
+
+
+@pytest.mark.parametrize("n,flags,total_target,lead", [
+    (4, SIMPLE | (1 << 17), 2_600_000, 700_000),      # fp32 pipes, segments of 2048: tapered from 1.82 M elements
+    (2, 1 << 17, 2_400_000, 1_500_000),               # the pair, separate finish (no single launch)
+    (16, 0, 7_900_000, 3_000_000),                    # tensor cores, segments of 8192: tapered from 7.27 M elements
+])
+def test_tapered_tables_cover_every_element_once(lib, n, flags, total_target, lead):
+    """Pass-1 tables of buffers that fill the GPU at least three times over are cut with shorter
+    segments at both ends.  Tensor boundaries are placed inside every zone (the half-length start,
+    the full-length middle, the half- and quarter-length end), with odd sizes so that cuts fall off
+    the 64-element grid, and every tensor is compared with the oracle."""
+    rng = np.random.default_rng(77 + n)
+    sizes = [lead, 65, 1031]
+    while sum(sizes) < total_target:
+        sizes.append(int(rng.choice([97, 513, 2049, 8191, 16385, 40_001, 150_003, 333_337])))
+    order = rng.permutation(len(sizes))
+    sizes = [sizes[i] for i in order]
+    off = workloads.offsets_from_sizes(sizes)
+    grads = _inputs(n, int(off[-1]), seed=6100 + n)
+    out = lib.adasum_reduce(grads, off, flags=flags)
+    torch.cuda.synchronize()
+    ref = oracle.adasum_reduce([g.cpu().numpy() for g in grads], offsets=off, dtype="f32", threads=0)
+    got = out.double().cpu().numpy()
+    assert np.all(np.isfinite(got))
+    for t in range(len(sizes)):
+        lo, hi = int(off[t]), int(off[t + 1])
+        assert np.linalg.norm(got[lo:hi] - ref[lo:hi]) <= 1e-5 * np.linalg.norm(ref[lo:hi]), (t, sizes[t])
