@@ -263,8 +263,9 @@ def time_steps(call, steps, warmup, world=1, sampler=None, flush=True, device="c
 
 
 def time_variants(lib, wl, steps, warmup, flags):
-    """The same workload through adasum_reduce_delta: with a start buffer (the optimizer-delta form,
-    result written over the start buffer) and with bf16 output.  Per-step events, L2 flushed."""
+    """The same workload through adasum_reduce_delta (with a start buffer: the optimizer-delta form,
+    result written over the start buffer; and with bf16 output) and through adasum_reduce_scaled.
+    Per-step events, L2 flushed."""
     dev = wl.grads[0].device
     dt = wl.grads[0].dtype
     need = lib.adasum_workspace_bytes(wl.total_elems, wl.num_tensors, wl.n_workers, wl.spec.dtype, flags)
@@ -285,6 +286,14 @@ def time_variants(lib, wl, steps, warmup, flags):
                                          stream=stream),
          2 * wl.n_workers * wl.total_elems * b + 2 * wl.total_elems),
     ]
+    if wl.n_workers >= 2:
+        # the same buffers read as scale x gradient (dynamic scaling): one scale per worker and tensor
+        scales = torch.exp2(torch.randint(-4, 5, (wl.n_workers, wl.num_tensors), generator=gen, device=dev).float())
+        out32 = torch.empty(wl.total_elems, dtype=torch.float32, device=dev)
+        cases.append(("scaled reduce, one scale per worker and tensor",
+                      lambda: lib.adasum_reduce_scaled(wl.grads, scales, wl.offsets, out=out32, workspace=ws,
+                                                       flags=flags, stream=stream),
+                      2 * wl.n_workers * wl.total_elems * b + 4 * wl.total_elems))
     if wl.spec.dtype == "f32" and wl.input_bytes <= 4e9:
         # the same values as fp64 buffers: the fp64 kernels (levels of radix 4 / 2, doubles throughout)
         grads64 = [g.double() for g in wl.grads]

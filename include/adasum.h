@@ -215,6 +215,40 @@ adasum_status_t adasum_reduce_ex(const void* const* grads, const int64_t* tensor
                                  size_t workspace_bytes, uint32_t flags, void* stream);
 
 /*
+ * The reduce of gradients that are stored with a scale ("dynamic scaling", Section 4.4.1: in a
+ * low-precision type every tensor is kept multiplied by a scale that holds its values inside the
+ * type's range, and the scale is adjusted as training goes).  Worker w's buffer holds, for tensor t,
+ *
+ *     grads[w][e] = scales[w * num_tensors + t] * g_w[e]        (e in tensor t),
+ *
+ * and the call returns the combination of the gradients themselves, in fp32:
+ *
+ *     out = Adasum_w(g_w) = Adasum_w(grads[w] / scales[w][t])           per tensor.
+ *
+ * The operator is not linear, so workers with different scales cannot be combined as stored and
+ * rescaled afterwards.  Nothing is rescaled in memory either: the dot products are formed of the
+ * stored values as in adasum_reduce, and the fp64 coefficient step divides entry (i, k) of a
+ * tensor's Gram matrix by scales[i][t] * scales[k][t] and the weight of worker i's stored values by
+ * scales[i][t] (tensors of at most 64 elements: every loaded value is divided, in fp64).  Same
+ * traffic and launches as adasum_reduce_ex, except that inputs small enough for the single
+ * cooperative launch take the two-pass path.
+ *
+ *   scales          device, n_workers * num_tensors floats (worker-major), 4-byte aligned; every
+ *                   entry finite and > 0 (not checked: anything else gives Inf or NaN in that
+ *                   tensor's output); read during the call's kernels, so it must stay unchanged
+ *                   until they have run
+ *   dtype           ADASUM_F32, ADASUM_F16 or ADASUM_BF16 (ADASUM_ERR_DTYPE for ADASUM_F64)
+ *   n_workers       2 .. ADASUM_MAX_WORKERS (ADASUM_ERR_ARG for 1)
+ *   orthogonality   as for adasum_reduce_ex (of the gradients themselves), or NULL
+ *   everything else as for adasum_reduce_ex, including the workspace size and the flags.
+ */
+adasum_status_t adasum_reduce_scaled(const void* const* grads, const float* scales,
+                                     const int64_t* tensor_offsets, int32_t num_tensors,
+                                     int32_t n_workers, adasum_dtype_t dtype, float* out,
+                                     float* orthogonality, void* workspace, size_t workspace_bytes,
+                                     uint32_t flags, void* stream);
+
+/*
  * The reduce wrapped around a local optimizer step (Section 4.1, the figure that applies the
  * operator after optimizer.step(); also "Low Precision Support" in Section 4.4.1 and the
  * delta-from-the-last-allreduce of Section 5.2).  Every worker has taken its own optimizer step

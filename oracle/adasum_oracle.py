@@ -7,8 +7,8 @@ module imports nothing from them.
 The arithmetic lives in ``adasum_oracle.c`` (plain C, fp64, left-to-right sums); this file only
 compiles it with gcc on first use and marshals numpy arrays.  Paper passages followed: the Adasum
 pair operator (Section 3), its recursive binary-tree extension (Section 3.4, Algorithm 1's
-bottom-up pairing), per-layer application (Sections 3.6 and 4.4.3), double accumulation
-(Section 4.4.1) and the orthogonality measure (Section 3.6).
+bottom-up pairing), per-layer application (Sections 3.6 and 4.4.3), double accumulation and
+gradients stored with a scale (Section 4.4.1) and the orthogonality measure (Section 3.6).
 """
 from __future__ import annotations
 
@@ -182,3 +182,26 @@ def adasum_reduce_delta(currents, start, offsets=None, dtype: str | None = None,
     if return_orthogonality:
         return s + res[0], res[1]
     return s + res
+
+
+# ---- gradients stored with a scale -------------------------------------------------------------
+
+def adasum_reduce_scaled(grads, scales, offsets=None, dtype: str | None = None, linear_order: bool = False,
+                         return_orthogonality: bool = False, threads: int = 1, top_down: bool = False):
+    """Dynamic scaling (Section 4.4.1): worker w's buffer holds ``scales[w][t]`` times its gradient
+    for tensor t.  By definition the result is the operator applied to the gradients themselves:
+    every stored value is decoded to fp64 and divided by its scale, then ``adasum_reduce`` runs on
+    those fp64 vectors.  Returns fp64."""
+    arrs = [decode(g, dtype).reshape(-1) for g in grads]
+    total = arrs[0].size
+    offs = np.asarray([0, total] if offsets is None else offsets, dtype=np.int64)
+    num_tensors = offs.size - 1
+    sc = np.asarray(scales, dtype=np.float64).reshape(len(arrs), num_tensors)
+    true = []
+    for w, a in enumerate(arrs):
+        g = a.copy()
+        for t in range(num_tensors):
+            g[offs[t]:offs[t + 1]] /= sc[w, t]
+        true.append(g)
+    return adasum_reduce(true, offsets=offs, dtype="f64", linear_order=linear_order,
+                         return_orthogonality=return_orthogonality, threads=threads, top_down=top_down)

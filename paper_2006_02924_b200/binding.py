@@ -194,6 +194,43 @@ def adasum_reduce_ex(grads, tensor_offsets=None, out=None, orthogonality=None, w
     return out, orthogonality
 
 
+_lib.adasum_reduce_scaled.restype = ctypes.c_int
+_lib.adasum_reduce_scaled.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.c_void_p, _i64p, ctypes.c_int32,
+                                      ctypes.c_int32, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
+                                      ctypes.c_void_p, ctypes.c_size_t, ctypes.c_uint32, ctypes.c_void_p]
+
+
+def adasum_reduce_scaled(grads, scales, tensor_offsets=None, out=None, orthogonality=None, workspace=None,
+                         flags: int = 0, stream=None, want_orthogonality: bool = False):
+    """``adasum_reduce_scaled`` of the C ABI: the buffers hold ``scales[w, t]`` times worker w's
+    gradient for tensor t (a CUDA fp32 tensor of shape [N, num_tensors]); returns the combination of
+    the gradients themselves (and the orthogonality measure when asked for)."""
+    grads = list(grads)
+    first = grads[0]
+    total = first.numel()
+    offs = _offsets_array(tensor_offsets, total)
+    num_tensors = offs.size - 1
+    if scales.dtype != torch.float32 or not scales.is_cuda or not scales.is_contiguous():
+        raise TypeError("scales must be a contiguous CUDA fp32 tensor")
+    if scales.numel() != len(grads) * num_tensors:
+        raise ValueError(f"scales has {scales.numel()} entries, need {len(grads)} x {num_tensors}")
+    if out is None:
+        out = torch.empty(total, dtype=torch.float32, device=first.device)
+    if orthogonality is None and want_orthogonality:
+        orthogonality = torch.empty(max(num_tensors, 1), dtype=torch.float32, device=first.device)[:num_tensors]
+    need = adasum_workspace_bytes(total, num_tensors, len(grads), first.dtype, flags)
+    workspace, ws_ptr, ws_bytes = _workspace(workspace, need, first.device)
+    ptrs = (ctypes.c_void_p * len(grads))(*[g.data_ptr() for g in grads])
+    with torch.cuda.device(first.device):
+        status = _lib.adasum_reduce_scaled(ptrs, scales.data_ptr(), offs.ctypes.data_as(_i64p), num_tensors,
+                                           len(grads), _dtype_code(first.dtype), out.data_ptr(),
+                                           orthogonality.data_ptr() if orthogonality is not None else None, ws_ptr,
+                                           ws_bytes, int(flags), _stream_handle(stream))
+    if status != ADASUM_OK:
+        raise AdasumError(status)
+    return (out, orthogonality) if orthogonality is not None else out
+
+
 _lib.adasum_sharded_gram.restype = ctypes.c_int
 _lib.adasum_sharded_gram.argtypes = [ctypes.POINTER(ctypes.c_void_p), _i64p, ctypes.c_int32, ctypes.c_int32,
                                      ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_uint32, ctypes.c_int32,

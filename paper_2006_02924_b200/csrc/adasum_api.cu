@@ -681,7 +681,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
                             void* workspace, size_t workspace_bytes, uint32_t flags, cudaStream_t stream,
                             LevelPhase phase = PHASE_WHOLE, int only_level = -1, size_t* sums_offset = nullptr,
                             int64_t* sums_count = nullptr, const void* start = nullptr,
-                            adasum_dtype_t out_dtype = ADASUM_F32)
+                            adasum_dtype_t out_dtype = ADASUM_F32, const float* leaf_scales = nullptr)
 {
     g_error[0] = '\0';
     if (dtype == ADASUM_F64)       // whole reduces of fp64 buffers go to reduce_f64_impl
@@ -692,6 +692,12 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         return fail(ADASUM_ERR_ARG, "the orthogonality measure needs at least two workers");
     if (reinterpret_cast<uintptr_t>(orthogonality) & 3u)
         return fail(ADASUM_ERR_ARG, "orthogonality is not 4-byte aligned");
+    if (leaf_scales != nullptr) {
+        if (n_workers < 2)
+            return fail(ADASUM_ERR_ARG, "the scaled reduce needs at least two workers");
+        if (reinterpret_cast<uintptr_t>(leaf_scales) & 3u)
+            return fail(ADASUM_ERR_ARG, "scales is not 4-byte aligned");
+    }
     adasum_status_t st = check_common(offsets, num_tensors, n_workers, dtype);
     if (st != ADASUM_OK)
         return st;
@@ -780,7 +786,9 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     const bool separate_finish = (flags & ADASUM_FLAG_SEPARATE_FINISH) != 0 || sharded;
     // Inputs that fit the L2 are served by one cooperative launch that needs no ticket counters.
     int small_seg_len = 0;
-    const int small_blocks = (sharded || total == 0 || num_tensors == 0) ? 0 : resident_small_blocks();
+    // (the single-launch kernel has no scaled form)
+    const int small_blocks =
+        (sharded || leaf_scales != nullptr || total == 0 || num_tensors == 0) ? 0 : resident_small_blocks();
     const bool small_candidate = small_blocks > 0 && small_input_plan(plan, total, num_tensors, offsets, n_workers, eb,
                                                                       flags, small_blocks, &small_seg_len);
     // the workspace arrives with unknown contents
@@ -828,6 +836,9 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         sa.table = short_ref->d_short;
         sa.order = tree_order(n_workers, flags);
         sa.start = start;
+        sa.leaf_scales = leaf_scales;
+        sa.num_tensors = num_tensors;
+        sa.worker_base = 0;
         sa.base_dtype = (int)dtype;
         sa.out_dtype = (int)out_dtype;
         OperandTable table;
@@ -852,6 +863,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
             for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
                 table.ptr[i] = grads[w0 + (i < here ? i : 0)];
             ShortArgs part = sa;
+            part.worker_base = w0;
             part.vec_out = vecs + (int64_t)j * lay.short_vec_stride;
             part.leaf_sum_out = sums + (int64_t)j * lay.short_sum_stride;
             ADASUM_CUDA_CHECK(launch_short_tensors((int)dtype, table, here, num_short, part, stream));
@@ -860,6 +872,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
             table.ptr[i] = vecs + (int64_t)(i < launches ? i : 0) * lay.short_vec_stride;
         sa.start = nullptr;
+        sa.leaf_scales = nullptr;        // the vectors of the earlier launches are gradients already
         sa.out = out;
         sa.base = start;
         sa.orthogonality = orthogonality;
@@ -978,6 +991,8 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         a.tree.groups_first = plan.level[0].groups;
         a.tree.leaf_norm_sums = orthogonality ? reinterpret_cast<double*>(ws + lay.leaf_sums) : nullptr;
         a.tree.orthogonality = orthogonality;
+        a.tree.leaf_scales = leaf_scales;
+        a.tree.num_tensors = num_tensors;
         a.dst = last ? out : static_cast<void*>(ws + lay.buffer[l & 1]);
         a.dst_stride = last ? 0 : lay.padded_elems;
         a.extras = last ? last_extras : kNoExtras;
@@ -1487,6 +1502,20 @@ adasum_status_t adasum_reduce_ex(const void* const* grads, const int64_t* tensor
                                        workspace, workspace_bytes, flags, static_cast<cudaStream_t>(stream), nullptr);
     return adasum::reduce_impl(grads, tensor_offsets, num_tensors, n_workers, dtype, out, orthogonality, workspace,
                                workspace_bytes, flags, static_cast<cudaStream_t>(stream));
+}
+
+adasum_status_t adasum_reduce_scaled(const void* const* grads, const float* scales, const int64_t* tensor_offsets,
+                                     int32_t num_tensors, int32_t n_workers, adasum_dtype_t dtype, float* out,
+                                     float* orthogonality, void* workspace, size_t workspace_bytes, uint32_t flags,
+                                     void* stream)
+{
+    if (!scales)
+        return adasum::fail(ADASUM_ERR_NULL, "scales is NULL");
+    if (dtype == ADASUM_F64)
+        return adasum::fail(ADASUM_ERR_DTYPE, "the scaled reduce takes fp32, fp16 or bf16 gradients");
+    return adasum::reduce_impl(grads, tensor_offsets, num_tensors, n_workers, dtype, out, orthogonality, workspace,
+                               workspace_bytes, flags, static_cast<cudaStream_t>(stream), adasum::PHASE_WHOLE, -1,
+                               nullptr, nullptr, nullptr, ADASUM_F32, scales);
 }
 
 adasum_status_t adasum_reduce_delta(const void* const* currents, const void* start,

@@ -37,6 +37,10 @@ struct ShortArgs {
     const ShortTensor* table;     // device, one entry per short tensor (= per block)
     int order;                    // 0 bottom-up pairs with carry, 1 sequential, 2 top-down halves
     const void* start;            // delta form: every leaf is (operand - start), rounded to the operands' type
+    // dynamic scaling: operand i of this launch is worker worker_base + i, whose buffer holds
+    // leaf_scales[worker * num_tensors + tensor] times its gradient; nullptr: the gradients themselves
+    const float* leaf_scales;
+    int num_tensors, worker_base;
     // destination of this launch: either the final result ...
     void* out;                    // elements of out_dtype, indexed like the inputs; nullptr: not the final launch
     const void* base;             // added to the result (the delta form's start), or nullptr

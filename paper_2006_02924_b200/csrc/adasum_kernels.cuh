@@ -347,6 +347,11 @@ struct TreeOptions {
     int groups_first;         // number of groups of the first level
     double* leaf_norm_sums;   // [tensor][groups_first]: sum of the leaves' squared norms, or nullptr
     float* orthogonality;     // [tensor]: |result|^2 / sum_i |g_i|^2 (Section 3.6), or nullptr
+    // Dynamic scaling (Section 4.4.1): worker w's buffer holds leaf_scales[w * num_tensors + t] times
+    // its gradient for tensor t; nullptr: the buffers hold the gradients themselves.  Read by the
+    // first level only.
+    const float* leaf_scales;
+    int num_tensors;
 };
 
 struct FinishArgs {
@@ -1317,8 +1322,14 @@ __device__ void tree_weights_from_gram(const double* gram, int members, W* __res
     __shared__ double weight[R], norm[R], row_dot[R], coef_a[R / 2 > 0 ? R / 2 : 1], coef_b[R / 2 > 0 ? R / 2 : 1];
     const int tid = threadIdx.x;
     if (tid < R) {
-        weight[tid] = 1.0;
-        norm[tid] = tid < members ? gram[gram_index(R, tid, tid)] : 0.0;
+        // A leaf stored as s x its gradient starts with weight 1 / s instead of 1: every product
+        // below then is the one of the gradients themselves, and the weight that comes out is the
+        // one to apply to the stored values.
+        double unit = 1.0;
+        if (opt.leaf_scales != nullptr && opt.level_is_first && tid < members)
+            unit = 1.0 / (double)opt.leaf_scales[((int64_t)group * R + tid) * opt.num_tensors + tensor];
+        weight[tid] = unit;
+        norm[tid] = tid < members ? gram[gram_index(R, tid, tid)] * unit * unit : 0.0;
     }
     __syncthreads();
     double leaf_sum = 0.0;
@@ -1419,7 +1430,7 @@ __device__ void tree_weights_from_gram(const double* gram, int members, W* __res
     } else {
         for (int k = 1; k < members; ++k) {
             if (tid < k)
-                row_dot[tid] = weight[tid] * gram[gram_index(R, tid, k)];
+                row_dot[tid] = weight[tid] * weight[k] * gram[gram_index(R, tid, k)];
             __syncthreads();
             if (tid == 0) {
                 double dot = 0.0;
@@ -1435,7 +1446,7 @@ __device__ void tree_weights_from_gram(const double* gram, int members, W* __res
             if (tid < k)
                 weight[tid] *= coef_a[0];
             else if (tid == k)
-                weight[tid] = coef_b[0];
+                weight[tid] *= coef_b[0];
             __syncthreads();
         }
     }

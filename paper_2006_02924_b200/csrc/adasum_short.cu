@@ -110,7 +110,10 @@ short_tensor_kernel(const __grid_constant__ OperandTable ops, int operands, Shor
         const int n = min(kShortChunkLeaves, operands - first);
         for (int idx = threadIdx.x; idx < n * len; idx += kShortThreads) {
             const int i = idx / len, e = idx - i * len;
-            slot[i * kShortTensorElems + e] = short_load<T>(ops.ptr[first + i], a.start, first_elem + e);
+            double x = short_load<T>(ops.ptr[first + i], a.start, first_elem + e);
+            if (a.leaf_scales != nullptr)      // the buffer holds scale x gradient (Section 4.4.1)
+                x /= (double)a.leaf_scales[(int64_t)(a.worker_base + first + i) * a.num_tensors + st.tensor];
+            slot[i * kShortTensorElems + e] = x;
         }
         __syncthreads();
         if (want_sums) {

@@ -153,3 +153,22 @@ def test_package_fails_loudly_without_the_library(tmp_path, monkeypatch):
     mod = importlib.util.module_from_spec(spec)
     with pytest.raises(ImportError, match="native library"):
         spec.loader.exec_module(mod)
+
+
+def test_scaled_reduce_argument_errors_are_caught_on_the_host(binding):
+    """adasum_reduce_scaled: a missing or misaligned scale table, a single worker and fp64 buffers
+    are refused before any CUDA call (the pointers are made-up device addresses)."""
+    lib = binding.raw()
+    s = binding.adasum_status_string
+    good = (ctypes.c_void_p * 2)(0x30000000, 0x40000000)
+    offs = np.array([0, 8], dtype=np.int64)
+
+    def call(scales=0x50000000, n=2, dtype=0):
+        return lib.adasum_reduce_scaled(good, scales, offs.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), 1, n, dtype,
+                                        0x10000000, None, 0x20000000, 1 << 40, 0, None)
+
+    assert s(call(scales=None)) == "ADASUM_ERR_NULL"
+    assert "scales" in binding.adasum_last_error()
+    assert s(call(scales=0x50000002)) == "ADASUM_ERR_ARG"
+    assert s(call(n=1)) == "ADASUM_ERR_ARG"
+    assert s(call(dtype=3)) == "ADASUM_ERR_DTYPE"

@@ -367,3 +367,73 @@ def test_delta_form_rounds_the_difference_to_the_buffer_type():
     d = (cur.astype(np.float64) - start.astype(np.float64)).astype(np.float16)
     out = oracle.adasum_reduce_delta([cur, cur], start, dtype="f16")
     assert np.allclose(out, start.astype(np.float64) + d.astype(np.float64), rtol=0, atol=1e-15)
+
+
+# ---- gradients stored with a scale (dynamic scaling, Section 4.4.1) ------------------------------
+
+def test_scaled_form_orthogonal_workers_closed_case():
+    """Orthogonal gradients add up.  The stored vectors are 4 x (1, 0) and 0.5 x (0, 1) with scales
+    (4, 0.5): the result is (1, 1); multiplying by the scales instead of dividing gives (16, 0.25)."""
+    a = np.array([4.0, 0.0])
+    b = np.array([0.0, 0.5])
+    got = oracle.adasum_reduce_scaled([a, b], [[4.0], [0.5]], dtype="f64")
+    np.testing.assert_allclose(got, [1.0, 1.0], rtol=0, atol=1e-15)
+
+
+def test_scaled_form_identical_gradients_whatever_the_scales():
+    """Adasum(g, g, ..., g) = g: workers whose gradients are the same vector stored with different
+    scales give that vector back, for every count and in every order."""
+    rng = np.random.default_rng(5)
+    g = rng.standard_normal(37)
+    for n in (2, 3, 5, 8):
+        scales = rng.uniform(0.01, 300.0, size=(n, 1))
+        stored = [g * scales[w, 0] for w in range(n)]
+        for kw in ({}, {"linear_order": True}, {"top_down": True}):
+            got = oracle.adasum_reduce_scaled(stored, scales, dtype="f64", **kw)
+            np.testing.assert_allclose(got, g, rtol=1e-13, atol=0)
+
+
+def test_scaled_form_uniform_scale_is_homogeneity():
+    """One scale s for every worker of a tensor: the operator is homogeneous of degree one, so the
+    result is the plain reduce of the stored vectors divided by s, tensor by tensor."""
+    rng = np.random.default_rng(6)
+    offs = [0, 5, 5, 40, 41]
+    n = 6
+    stored = [rng.standard_normal(41) for _ in range(n)]
+    per_tensor = np.array([3.0, 7.0, 0.125, 1000.0])
+    scales = np.tile(per_tensor, (n, 1))
+    got = oracle.adasum_reduce_scaled(stored, scales, offsets=offs, dtype="f64")
+    plain = oracle.adasum_reduce(stored, offsets=offs, dtype="f64")
+    for t in range(4):
+        np.testing.assert_allclose(got[offs[t]:offs[t + 1]], plain[offs[t]:offs[t + 1]] / per_tensor[t],
+                                   rtol=1e-13, atol=0)
+
+
+def test_scaled_form_layout_is_worker_major_and_per_tensor():
+    """Three workers, two tensors, six different power-of-two scales: the stored fp16 values are the
+    gradients times their scale exactly, so the result must be the plain reduce of the gradients.
+    Reading the table tensor-major, or applying a worker's scale to the wrong tensor, fails."""
+    rng = np.random.default_rng(7)
+    offs = [0, 9, 20]
+    g = [np.round(rng.standard_normal(20) * 64) / 64 for _ in range(3)]        # exact in fp16 after scaling
+    scales = np.array([[2.0, 0.25], [16.0, 0.5], [0.125, 8.0]])
+    stored = []
+    for w in range(3):
+        v = g[w].copy()
+        v[0:9] *= scales[w, 0]
+        v[9:20] *= scales[w, 1]
+        assert np.all(v.astype(np.float16).astype(np.float64) == v)
+        stored.append(v.astype(np.float16))
+    got = oracle.adasum_reduce_scaled(stored, scales, offsets=offs, dtype="f16")
+    want = oracle.adasum_reduce(g, offsets=offs, dtype="f64")
+    np.testing.assert_allclose(got, want, rtol=1e-13, atol=1e-15)
+
+
+def test_scaled_form_orthogonality_is_that_of_the_gradients():
+    """Mutually orthogonal gradients stored with different scales: the measure of Section 3.6 is 1."""
+    n = 4
+    stored = [np.eye(n)[w] * (w + 2.0) for w in range(n)]
+    scales = np.array([[w + 2.0] for w in range(n)]) * 10.0
+    out, ortho = oracle.adasum_reduce_scaled(stored, scales, dtype="f64", return_orthogonality=True)
+    np.testing.assert_allclose(out, np.full(n, 0.1), rtol=1e-14)
+    np.testing.assert_allclose(ortho, [1.0], rtol=1e-14)
