@@ -208,6 +208,12 @@ int64_t segment_bound(int64_t total, int32_t num_tensors, int seg_len)
     return total / seg_len + 2 * (int64_t)num_tensors + 1 + (may_taper ? 4 * kTaperSlots : 0);
 }
 
+// Upper bound of the runs of kSegmentsPerGroup segments in such a table (every tensor ends one).
+int64_t run_bound(int64_t segments, int32_t num_tensors)
+{
+    return segments / kSegmentsPerGroup + num_tensors + 1;
+}
+
 struct Layout {
     size_t partials = 0, weights = 0, weights_alt = 0, gram64 = 0, counters = 0, leaf_sums = 0, buffer[2] = {0, 0};
     size_t partials_bytes = 0, weights_bytes = 0, gram64_bytes = 0, counters_bytes = 0, leaf_sums_bytes = 0,
@@ -215,6 +221,7 @@ struct Layout {
     // short tensors of reduces with more workers than one launch carries: per launch an fp64 vector
     // over the short tensors' elements and the sum of its leaves' squared norms
     size_t short_vecs = 0, short_sums = 0, short_vecs_bytes = 0, short_sums_bytes = 0;
+    size_t run_sums = 0, run_sums_bytes = 0;       // the two-step finish: one fp64 Gram matrix per run and group
     int64_t short_vec_stride = 0, short_sum_stride = 0;      // doubles between two launches' arrays
     int64_t padded_elems = 0;
     size_t total = 0;
@@ -242,9 +249,17 @@ Layout make_layout(const LevelPlan& plan, int64_t total_elems, int32_t num_tenso
             lay.partials_bytes = p;
         if (w > lay.weights_bytes)
             lay.weights_bytes = w;
-        const size_t c = ((size_t)(num_tensors > 0 ? num_tensors : 1) * lv.groups + 1) * sizeof(int);
-        if (c > lay.counters_bytes)       // + 1: the device status word sits after the ticket counters
+        // ticket counters per (tensor, group), then per (run of segments, group); + 1: the device
+        // status word sits after them
+        const size_t runs = (size_t)run_bound(segment_bound(total_elems, num_tensors,
+                                                            min_gram_segment_length(lv.radix, total_elems)),
+                                              num_tensors);
+        const size_t c = (((size_t)(num_tensors > 0 ? num_tensors : 1) + runs) * lv.groups + 1) * sizeof(int);
+        if (c > lay.counters_bytes)
             lay.counters_bytes = c;
+        const size_t rs = runs * lv.groups * gram_entries(lv.radix) * sizeof(double);
+        if (rs > lay.run_sums_bytes)
+            lay.run_sums_bytes = rs;
         const size_t g64 = (size_t)(num_tensors > 0 ? num_tensors : 1) * lv.groups * gram_entries(lv.radix) *
                            sizeof(double);
         if (g64 > lay.gram64_bytes)
@@ -278,6 +293,8 @@ Layout make_layout(const LevelPlan& plan, int64_t total_elems, int32_t num_tenso
     off += align_up(lay.short_vecs_bytes);
     lay.short_sums = off;
     off += align_up(lay.short_sums_bytes);
+    lay.run_sums = off;
+    off += align_up(lay.run_sums_bytes);
     lay.total = off > 0 ? off : kAlign;
     return lay;
 }
@@ -356,8 +373,8 @@ void build_segments(const int64_t* offsets, int32_t num_tensors, int seg_len, bo
     for (int32_t t = 0; t < num_tensors; ++t)
         left += in_segments(t) ? offsets[t + 1] - offsets[t] : 0;
     const int64_t round = (int64_t)taper_slots * seg_len;
-    if (left < 3 * round || seg_len % 256 != 0)
-        taper_slots = 0;        // too short a launch to have a middle
+    if (left < 3 * round || seg_len < 4096)
+        taper_slots = 0;        // too short a launch to have a middle, or blocks too short to matter
     tab->taper_slots = taper_slots;
     int64_t done = 0;
     for (int32_t t : order) {
@@ -390,6 +407,16 @@ void build_segments(const int64_t* offsets, int32_t num_tensors, int seg_len, bo
             tab->max_segments_per_tensor = n;
     }
     tab->num_segments = (int32_t)tab->h_segments.size();
+    // runs of kSegmentsPerGroup segments, numbered through the tensors in their own order
+    tab->h_seg_first.resize(3 * (size_t)num_tensors + 3, 0);
+    int32_t runs = 0;
+    for (int32_t t = 0; t < num_tensors; ++t) {
+        tab->h_seg_first[2 * (size_t)num_tensors + 2 + t] = runs;
+        const int32_t n = tab->h_seg_first[2 * (size_t)t + 1] - tab->h_seg_first[2 * (size_t)t];
+        runs += (n + kSegmentsPerGroup - 1) / kSegmentsPerGroup;
+    }
+    tab->h_seg_first[3 * (size_t)num_tensors + 2] = runs;
+    tab->num_runs = runs;
 }
 
 // The table for (current device, offsets, seg_len), built and uploaded on first use.  The caller
@@ -445,6 +472,7 @@ adasum_status_t get_segment_table(const int64_t* offsets, int32_t num_tensors, i
                          sizeof(Segment) * tab->h_segments.size(), cudaMemcpyHostToDevice);
     if (err == cudaSuccess)
         err = cudaMemcpy(tab->d_seg_first, tab->h_seg_first.data(), first_bytes, cudaMemcpyHostToDevice);
+    tab->d_group_first = tab->d_seg_first ? tab->d_seg_first + 2 * (size_t)num_tensors + 2 : nullptr;
     if (err == cudaSuccess && !tab->h_warp.empty()) {
         err = cudaMalloc(&tab->d_warp, sizeof(WarpTensor) * tab->h_warp.size());
         if (err == cudaSuccess)
@@ -914,7 +942,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
             OperandTable table;
             for (int i = 0; i < kMaxOperandsPerLaunch; ++i)
                 table.ptr[i] = grads[i < n_workers ? i : 0];
-            FinishArgs fin;
+            FinishArgs fin{};
             fin.seg_first = tab->d_seg_first;
             fin.counters = nullptr;
             fin.weights = nullptr;
@@ -979,6 +1007,8 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         a.weights = reinterpret_cast<float*>(ws + ((l & 1) ? lay.weights_alt : lay.weights));
         a.gram64 = reinterpret_cast<double*>(ws + lay.gram64);
         a.counters = separate_finish ? nullptr : reinterpret_cast<int*>(ws + lay.counters);
+        a.run_counters = reinterpret_cast<int*>(ws + lay.counters) + (size_t)(num_tensors > 0 ? num_tensors : 1) * lv.groups;
+        a.run_sums = reinterpret_cast<double*>(ws + lay.run_sums);
         a.phase = phase;
         // the status word is the last int of the (zeroed) counter region
         a.tc_status = (flags & ADASUM_FLAG_NO_TCGEN05)
@@ -1403,8 +1433,9 @@ adasum_status_t pair_noalloc_impl(const void* a, const void* b, const int64_t* o
     if (!tab.h_segments.empty())
         ADASUM_CUDA_CHECK(cudaMemcpyAsync(tab.d_segments, tab.h_segments.data(),
                                           sizeof(Segment) * tab.h_segments.size(), cudaMemcpyHostToDevice, stream));
+    // (the segment ranges only: the run numbers that follow them are for the ticket finish, unused here)
     ADASUM_CUDA_CHECK(cudaMemcpyAsync(tab.d_seg_first, tab.h_seg_first.data(),
-                                      sizeof(int32_t) * tab.h_seg_first.size(), cudaMemcpyHostToDevice, stream));
+                                      sizeof(int32_t) * (2 * (size_t)num_tensors + 2), cudaMemcpyHostToDevice, stream));
     if (!tab.h_short.empty())
         ADASUM_CUDA_CHECK(cudaMemcpyAsync(short_table, tab.h_short.data(), sizeof(ShortTensor) * tab.h_short.size(),
                                           cudaMemcpyHostToDevice, stream));

@@ -83,6 +83,11 @@ struct SegmentTable {
     std::vector<int64_t> offsets;
     Segment* d_segments = nullptr;
     int32_t* d_seg_first = nullptr;
+    // d_seg_first + 2 * num_tensors + 2: per tensor the number of its first run of kSegmentsPerGroup
+    // segments (runs are numbered through the table; the two-step finish keeps a counter and a sum
+    // per run); the same allocation
+    int32_t* d_group_first = nullptr;
+    int32_t num_runs = 0;
     bool owns_device_arrays = false;    // false: the arrays belong to somebody else (static scratch)
     int32_t num_segments = 0;
     int32_t max_segments_per_tensor = 0;
@@ -141,6 +146,8 @@ struct LevelArgs {
     int32_t num_tensors;
     float* partials;
     int* counters;      // ticket counters for finishing inside pass 1, or nullptr
+    int* run_counters;  // zeroed, one per (run of segments, group): the two-step finish of long tensors
+    double* run_sums;   // [run][group][entries of the Gram matrix]
     TreeOptions tree;
     LevelPhase phase;
     int* tc_status;     // status word for the tcgen05 kernel, or nullptr to keep to mma.sync

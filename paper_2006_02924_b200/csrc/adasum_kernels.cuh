@@ -361,36 +361,90 @@ struct FinishArgs {
     TreeOptions tree;
     int selftest_timeout;       // gram_partial_tc64_kernel only: leave the last tile unmultiplied and wait briefly,
                                 // so that the epilogue's bounded wait runs out (test of the status path)
+    // Tensors of more than kSegmentsPerGroup segments are finished in two steps (nullptr: in one):
+    // the block that hands in the last partial of a run of kSegmentsPerGroup segments adds that
+    // run's partials, and the block that hands in the tensor's last run sum adds the run sums.
+    const int32_t* group_first; // [tensor]: number of the tensor's first run
+    int* group_counters;        // [run][group], zero on entry
+    double* group_sums;         // [run][group][E]
 };
 
-template <int R>
-__device__ void finish_group_in_block(const float* partials, int seg_begin, int seg_end, int tensor, int group,
-                                      int groups_total, int members, float* weights_dst, const TreeOptions& opt);
+constexpr int kSegmentsPerGroup = 16;
 
-// Called by every thread of the block after its partial matrix has been written.
+template <int R>
+__device__ void add_partials_in_block(const float* partials, int seg_begin, int seg_end, int group, int groups_total,
+                                      double* gram);
+template <int R, typename W = float>
+__device__ void tree_weights_from_gram(const double* gram, int members, W* __restrict__ dst, const TreeOptions& opt,
+                                       int tensor, int group);
+
+// Called by every thread of the block after its partial matrix (number seg_index) has been written.
 template <int R>
 __device__ __forceinline__ void finish_if_last(const FinishArgs& fin, const float* partials, int tensor, int group,
-                                               int groups_total, int members)
+                                               int groups_total, int members, int seg_index)
 {
     if (fin.counters == nullptr)
         return;
+    constexpr int E = gram_entries(R);
     __shared__ int is_last;
-    __threadfence();                       // this block's partial is visible device-wide ...
-    __syncthreads();
+    __shared__ double gram[E];
     const int s0 = fin.seg_first[2 * tensor], s1 = fin.seg_first[2 * tensor + 1];
+    const bool in_runs = fin.group_sums != nullptr && s1 - s0 > kSegmentsPerGroup;
+    const int runs = (s1 - s0 + kSegmentsPerGroup - 1) / kSegmentsPerGroup;
+    const double* run_sums = nullptr;
+    if (in_runs) {
+        const int run = (seg_index - s0) / kSegmentsPerGroup;
+        const int run_begin = s0 + run * kSegmentsPerGroup;
+        const int run_end = min(run_begin + kSegmentsPerGroup, s1);
+        const int64_t first_slot = (int64_t)fin.group_first[tensor] * groups_total + group;
+        const int64_t slot = first_slot + (int64_t)run * groups_total;
+        run_sums = fin.group_sums + first_slot * E;
+        __threadfence();                   // this block's partial is visible device-wide ...
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const int ticket = atomicAdd(fin.group_counters + slot, 1);      // ... before its ticket is drawn
+            is_last = ticket == run_end - run_begin - 1;
+            if (is_last)
+                fin.group_counters[slot] = 0;
+        }
+        __syncthreads();
+        if (!is_last)
+            return;
+        __threadfence();
+        add_partials_in_block<R>(partials, run_begin, run_end, group, groups_total, gram);
+        double* run_sum = fin.group_sums + slot * E;
+        for (int k = threadIdx.x; k < E; k += kThreads)
+            run_sum[k] = gram[k];
+    }
+    __threadfence();                       // this block's partial (or run sum) is visible device-wide ...
+    __syncthreads();
     if (threadIdx.x == 0) {
         int* counter = fin.counters + (int64_t)tensor * groups_total + group;
         const int ticket = atomicAdd(counter, 1);      // ... before its ticket is drawn
-        is_last = ticket == s1 - s0 - 1;
+        is_last = ticket == (in_runs ? runs : s1 - s0) - 1;
         if (is_last)
             *counter = 0;                  // ready for the next level / the next call
     }
     __syncthreads();
-    if (is_last) {
-        __threadfence();
-        finish_group_in_block<R>(partials, s0, s1, tensor, group, groups_total, members,
-                                 fin.weights + ((int64_t)tensor * groups_total + group) * R, fin.tree);
+    if (!is_last)
+        return;
+    __threadfence();
+    if (in_runs) {
+        // the run sums, in run order
+        const int64_t stride = (int64_t)groups_total * E;
+        for (int k = threadIdx.x; k < E; k += kThreads) {
+            double sum = 0.0;
+#pragma unroll 8
+            for (int r = 0; r < runs; ++r)
+                sum += __ldcg(run_sums + r * stride + k);
+            gram[k] = sum;
+        }
+        __syncthreads();
+    } else {
+        add_partials_in_block<R>(partials, s0, s1, group, groups_total, gram);
     }
+    tree_weights_from_gram<R>(gram, members, fin.weights + ((int64_t)tensor * groups_total + group) * R, fin.tree,
+                              tensor, group);
 }
 
 // ---- pass 1: partial Gram matrices -------------------------------------------------------------
@@ -518,7 +572,7 @@ gram_partial_kernel(const __grid_constant__ OperandTable ops, int operands,
     gram_of_segment<T, R, VEC, DELTA>(ops, first, members, seg,
                                       partials + ((int64_t)blockIdx.x * groups_total + group_base + blockIdx.y) * E,
                                       static_cast<const T*>(start));
-    finish_if_last<R>(fin, partials, seg.tensor, group_base + blockIdx.y, groups_total, members);
+    finish_if_last<R>(fin, partials, seg.tensor, group_base + blockIdx.y, groups_total, members, (int)blockIdx.x);
 }
 
 // ---- asynchronous copies into shared memory ----------------------------------------------------
@@ -1036,7 +1090,7 @@ gram_partial_mma_kernel(const __grid_constant__ OperandTable ops, int operands,
     gram_segment_mma<T, R, VEC, DELTA>(ops, first, members, seg,
                                        partials + ((int64_t)blockIdx.x * groups_total + group_base + blockIdx.y) * E,
                                        start_ptr);
-    finish_if_last<R>(fin, partials, seg.tensor, group_base + blockIdx.y, groups_total, members);
+    finish_if_last<R>(fin, partials, seg.tensor, group_base + blockIdx.y, groups_total, members, (int)blockIdx.x);
 }
 
 // ---- pass 1 for groups of 64 fp16 / bf16 rows: tcgen05 ------------------------------------------
@@ -1288,7 +1342,7 @@ gram_partial_tc64_kernel(const __grid_constant__ OperandTable ops, int operands,
     __syncthreads();
     if (warp == 0)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 64;" ::"r"(tmem_acc) : "memory");
-    finish_if_last<R>(fin, partials, seg.tensor, group_base + blockIdx.y, groups_total, R);
+    finish_if_last<R>(fin, partials, seg.tensor, group_base + blockIdx.y, groups_total, R, (int)blockIdx.x);
 }
 
 // ---- coefficients: the binary tree evaluated on a Gram matrix ---------------------------------
@@ -1315,7 +1369,7 @@ __device__ __forceinline__ void pair_coefficients(double dot, double norm_a, dou
 // Also written, when asked for: the sum of the leaves' squared norms (first level) and the
 // orthogonality measure |result|^2 / sum_i |g_i|^2 of Section 3.6 (last level; NaN when every
 // leaf is zero).
-template <int R, typename W = float>
+template <int R, typename W>
 __device__ void tree_weights_from_gram(const double* gram, int members, W* __restrict__ dst,
                                        const TreeOptions& opt, int tensor, int group)
 {
@@ -1467,16 +1521,15 @@ __device__ void tree_weights_from_gram(const double* gram, int members, W* __res
     }
 }
 
-// The tensor's partial matrices (segments seg_begin .. seg_end) added in fp64 by one block of
-// kThreads threads, then the tree.  Small groups: with Q = kThreads / E slices, slice q takes
-// segments q, q + Q, ... in order and the slices are added in order.  Partials were written by
-// other blocks of the running kernel, hence the L2 loads.
+// Partial matrices of segments seg_begin .. seg_end added in fp64 by one block of kThreads threads
+// into gram[0 .. E) (shared memory); ends with a block barrier.  Small groups: with Q = kThreads / E
+// slices, slice q takes segments q, q + Q, ... in order and the slices are added in order.
+// Partials were written by other blocks of the running kernel, hence the L2 loads.
 template <int R>
-__device__ void finish_group_in_block(const float* partials, int seg_begin, int seg_end, int tensor, int group,
-                                      int groups_total, int members, float* weights_dst, const TreeOptions& opt)
+__device__ void add_partials_in_block(const float* partials, int seg_begin, int seg_end, int group, int groups_total,
+                                      double* gram)
 {
     constexpr int E = gram_entries(R);
-    __shared__ double gram[E];
     const int64_t stride = (int64_t)groups_total * E;
     if constexpr (E <= kThreads) {
         constexpr int Q = kThreads / E;
@@ -1509,7 +1562,6 @@ __device__ void finish_group_in_block(const float* partials, int seg_begin, int 
         }
     }
     __syncthreads();
-    tree_weights_from_gram<R>(gram, members, weights_dst, opt, tensor, group);
 }
 
 constexpr int kTreeThreadsMax = 1024;
@@ -1858,7 +1910,8 @@ wsum_gram_kernel(const __grid_constant__ OperandTable ops, int operands,
             sum += warp_sums[w][k];
         dst[k] = sum;
     }
-    finish_if_last<R2>(next_fin, next_partials, seg.tensor, next_group_base + blockIdx.y, next_groups_total, members_next);
+    finish_if_last<R2>(next_fin, next_partials, seg.tensor, next_group_base + blockIdx.y, next_groups_total, members_next,
+                       (int)blockIdx.x);
 }
 
 // ---- both passes in one launch, for inputs that fit the L2 -------------------------------------

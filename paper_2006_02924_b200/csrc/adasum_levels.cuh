@@ -193,7 +193,12 @@ template <typename T, int R1, int R2>
 adasum_status_t launch_wsum_gram(const LevelArgs& a)
 {
     constexpr int kNextGroupsPerLaunch = kMaxOperandsPerLaunch / (R1 * R2);
-    const FinishArgs next_fin{a.fuse_tab->d_seg_first, a.counters, a.next_weights, a.next_tree};
+    // (the next level's ticket counters per tensor end where its counters per run begin)
+    const FinishArgs next_fin{a.fuse_tab->d_seg_first, a.counters, a.next_weights, a.next_tree, 0,
+                              a.fuse_tab->d_group_first,
+                              a.counters ? a.counters + (size_t)(a.num_tensors > 0 ? a.num_tensors : 1) * a.next_groups
+                                         : nullptr,
+                              a.run_sums};
     for (int ng0 = 0; ng0 < a.next_groups; ng0 += kNextGroupsPerLaunch) {
         const int next_here = a.next_groups - ng0 < kNextGroupsPerLaunch ? a.next_groups - ng0 : kNextGroupsPerLaunch;
         const int g0 = ng0 * R2, op0 = g0 * R1;
@@ -218,7 +223,7 @@ adasum_status_t run_level_typed(const LevelArgs& a)
     // the last block of every (tensor, group) in pass 1 also derives the weights
     const bool fused_finish = a.counters != nullptr && a.phase == PHASE_WHOLE;
     const FinishArgs fin{a.gram_tab->d_seg_first, fused_finish ? a.counters : nullptr, a.weights, a.tree,
-                         a.selftest_timeout ? 1 : 0};
+                         a.selftest_timeout ? 1 : 0, a.gram_tab->d_group_first, a.run_counters, a.run_sums};
     // pass 1
     for (int g0 = 0; g0 < a.groups && a.phase != PHASE_APPLY && !a.skip_gram; g0 += kGroupsPerLaunch) {
         const int groups_here = a.groups - g0 < kGroupsPerLaunch ? a.groups - g0 : kGroupsPerLaunch;

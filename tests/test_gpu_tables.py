@@ -102,9 +102,9 @@ def test_host_threads_share_the_library(lib):
 
 
 @pytest.mark.parametrize("n,flags,total_target,lead", [
-    (4, SIMPLE | (1 << 17), 2_600_000, 700_000),      # fp32 pipes, segments of 2048: tapered from 1.82 M elements
-    (2, 1 << 17, 2_400_000, 1_500_000),               # the pair, separate finish (no single launch)
-    (16, 0, 7_900_000, 3_000_000),                    # tensor cores, segments of 8192: tapered from 7.27 M elements
+    (4, SIMPLE | (1 << 17), 8_600_000, 2_000_000),    # fp32 pipes, segments of 8192: tapered from 7.27 M elements
+    (2, 1 << 17, 8_500_000, 4_500_000),               # the pair, separate finish (no single launch)
+    (16, 0, 7_900_000, 3_000_000),                    # tensor cores, segments of 8192
 ])
 def test_tapered_tables_cover_every_element_once(lib, n, flags, total_target, lead):
     """Pass-1 tables of buffers that fill the GPU at least three times over are cut with shorter
