@@ -97,11 +97,27 @@ int pow2_ceil(int x)
 
 // Elements per segment.  One block accumulates a whole segment in fp32 (per thread: segment /
 // 256 elements; on the tensor cores: per warp segment / 8), longer tensors are finished in fp64.
-int gram_segment_length(GramKind kind, int64_t total)
+//
+// Buffers below 8 M elements that one round of blocks can cover: the shortest power of two that
+// still needs no second round (a one-tensor buffer of 256 K elements cut at 8192 would be 32 blocks
+// on 148 SMs).  One round, not more: a pass-1 block costs 5 to 10 microseconds before its first
+// tile is multiplied, so a second round of short blocks is slower than one round of long ones.
+int filling_length(int64_t total, int slots, int shortest, int longest)
+{
+    int len = shortest;
+    while (len < longest && (total + len - 1) / len > slots)
+        len *= 2;
+    return len;
+}
+// slots: blocks of the pass-1 kernel that the GPU holds at once (two per SM; one for the kernel
+// that keeps its accumulator in tensor memory).
+int gram_segment_length(GramKind kind, int64_t total, int slots = 296)
 {
     if (kind == GRAM_MMA)
-        return total >= (int64_t(1) << 26) ? 32768 : (total >= (int64_t(1) << 23) ? 16384 : 8192);
-    return total >= (int64_t(1) << 23) ? 8192 : 2048;
+        return total >= (int64_t(1) << 26)   ? 32768
+               : total >= (int64_t(1) << 23) ? 16384
+                                             : filling_length(total, slots, 1024, 8192);
+    return total >= (int64_t(1) << 23) ? 8192 : filling_length(total, slots, 512, 2048);
 }
 int min_gram_segment_length(int radix, int64_t total)
 {
@@ -987,8 +1003,10 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
         const bool simple_kernels = (flags & ADASUM_FLAG_SIMPLE_KERNELS) != 0;
         const GramKind kind = gram_kind(lv.radix, simple_kernels);
         TableRef gram_tab, wsum_tab, fuse_tab;     // held until this level's launches are enqueued
-        st = get_segment_table(offsets, num_tensors, gram_segment_length(kind, total), skip_short, &gram_tab, 0,
-                               kTaperSlots);
+        const bool tensor_memory_kernel = kind == GRAM_MMA && lv.radix == 64 && dtype != ADASUM_F32 && l == 0 &&
+                                          !(flags & ADASUM_FLAG_NO_TCGEN05);
+        st = get_segment_table(offsets, num_tensors, gram_segment_length(kind, total, tensor_memory_kernel ? 148 : 296),
+                               skip_short, &gram_tab, 0, kTaperSlots);
         if (st != ADASUM_OK)
             return st;
         st = get_segment_table(offsets, num_tensors, wsum_segment_length(total), skip_short, &wsum_tab);

@@ -413,7 +413,7 @@ __device__ __forceinline__ void finish_if_last(const FinishArgs& fin, const floa
         __threadfence();
         add_partials_in_block<R>(partials, run_begin, run_end, group, groups_total, gram);
         double* run_sum = fin.group_sums + slot * E;
-        for (int k = threadIdx.x; k < E; k += kThreads)
+        for (int k = threadIdx.x; k < E; k += (int)blockDim.x)
             run_sum[k] = gram[k];
     }
     __threadfence();                       // this block's partial (or run sum) is visible device-wide ...
@@ -432,7 +432,7 @@ __device__ __forceinline__ void finish_if_last(const FinishArgs& fin, const floa
     if (in_runs) {
         // the run sums, in run order
         const int64_t stride = (int64_t)groups_total * E;
-        for (int k = threadIdx.x; k < E; k += kThreads) {
+        for (int k = threadIdx.x; k < E; k += (int)blockDim.x) {
             double sum = 0.0;
 #pragma unroll 8
             for (int r = 0; r < runs; ++r)
@@ -1552,7 +1552,8 @@ __device__ void add_partials_in_block(const float* partials, int seg_begin, int 
         }
     } else {
         // wide groups: every thread owns several entries and adds their partials in segment order
-        for (int k = threadIdx.x; k < E; k += kThreads) {
+        // (blocks of more than kThreads threads: all of them)
+        for (int k = threadIdx.x; k < E; k += (int)blockDim.x) {
             const float* src = partials + (int64_t)group * E + k;
             double s = 0.0;
 #pragma unroll 8
