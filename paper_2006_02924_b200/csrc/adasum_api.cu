@@ -224,10 +224,12 @@ int64_t segment_bound(int64_t total, int32_t num_tensors, int seg_len)
     return total / seg_len + 2 * (int64_t)num_tensors + 1 + (may_taper ? 4 * kTaperSlots : 0);
 }
 
-// Upper bound of the runs of kSegmentsPerGroup segments in such a table (every tensor ends one).
-int64_t run_bound(int64_t segments, int32_t num_tensors)
+// Upper bound of the runs of kSegmentsPerGroup segments in such a table.  Only tensors of more than
+// kSegmentsPerGroup segments have runs, and such a tensor of n segments has at most n / 16 + 1 <=
+// n / 8 of them.
+int64_t run_bound(int64_t segments)
 {
-    return segments / kSegmentsPerGroup + num_tensors + 1;
+    return segments / (kSegmentsPerGroup / 2) + 1;
 }
 
 struct Layout {
@@ -268,8 +270,7 @@ Layout make_layout(const LevelPlan& plan, int64_t total_elems, int32_t num_tenso
         // ticket counters per (tensor, group), then per (run of segments, group); + 1: the device
         // status word sits after them
         const size_t runs = (size_t)run_bound(segment_bound(total_elems, num_tensors,
-                                                            min_gram_segment_length(lv.radix, total_elems)),
-                                              num_tensors);
+                                                            min_gram_segment_length(lv.radix, total_elems)));
         const size_t c = (((size_t)(num_tensors > 0 ? num_tensors : 1) + runs) * lv.groups + 1) * sizeof(int);
         if (c > lay.counters_bytes)
             lay.counters_bytes = c;
@@ -429,7 +430,8 @@ void build_segments(const int64_t* offsets, int32_t num_tensors, int seg_len, bo
     for (int32_t t = 0; t < num_tensors; ++t) {
         tab->h_seg_first[2 * (size_t)num_tensors + 2 + t] = runs;
         const int32_t n = tab->h_seg_first[2 * (size_t)t + 1] - tab->h_seg_first[2 * (size_t)t];
-        runs += (n + kSegmentsPerGroup - 1) / kSegmentsPerGroup;
+        if (n > kSegmentsPerGroup)          // shorter tensors are finished in one step and need no runs
+            runs += (n + kSegmentsPerGroup - 1) / kSegmentsPerGroup;
     }
     tab->h_seg_first[3 * (size_t)num_tensors + 2] = runs;
     tab->num_runs = runs;

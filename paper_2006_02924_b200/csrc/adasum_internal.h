@@ -83,9 +83,9 @@ struct SegmentTable {
     std::vector<int64_t> offsets;
     Segment* d_segments = nullptr;
     int32_t* d_seg_first = nullptr;
-    // d_seg_first + 2 * num_tensors + 2: per tensor the number of its first run of kSegmentsPerGroup
-    // segments (runs are numbered through the table; the two-step finish keeps a counter and a sum
-    // per run); the same allocation
+    // d_seg_first + 2 * num_tensors + 2: per tensor of more than kSegmentsPerGroup segments the number
+    // of its first run of that many segments (runs are numbered through those tensors; the two-step
+    // finish keeps a counter and a sum per run); the same allocation
     int32_t* d_group_first = nullptr;
     int32_t num_runs = 0;
     bool owns_device_arrays = false;    // false: the arrays belong to somebody else (static scratch)
