@@ -18,7 +18,7 @@
  * arithmetic is fp64 on the device; intermediates between levels and the output are fp32.
  * Tensors of at most 64 elements are the exception: their result can be a small difference of
  * large terms (a one-element tensor whose workers disagree in sign), so adasum_reduce,
- * adasum_reduce_ex, adasum_reduce_delta and adasum_pair apply the operator to them literally, pair
+ * adasum_reduce_ex, adasum_reduce_scaled, adasum_reduce_delta and adasum_pair apply the operator to them literally, pair
  * by pair and level by level, in fp64 from the loads to the one rounding of the stored result (one
  * more small kernel when a buffer has such tensors, run beside the streaming passes on a stream of
  * the library's own that is forked from `stream` and joined to it again with events before the call
