@@ -230,8 +230,7 @@ adasum_status_t adasum_reduce_ex(const void* const* grads, const int64_t* tensor
  * stored values as in adasum_reduce, and the fp64 coefficient step divides entry (i, k) of a
  * tensor's Gram matrix by scales[i][t] * scales[k][t] and the weight of worker i's stored values by
  * scales[i][t] (tensors of at most 64 elements: every loaded value is divided, in fp64).  Same
- * traffic and launches as adasum_reduce_ex, except that inputs small enough for the single
- * cooperative launch take the two-pass path.
+ * traffic, launches and plans as adasum_reduce_ex.
  *
  *   scales          device, n_workers * num_tensors floats (worker-major), 4-byte aligned; every
  *                   entry finite and > 0 (not checked: anything else gives Inf or NaN in that

@@ -832,9 +832,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
     const bool separate_finish = (flags & ADASUM_FLAG_SEPARATE_FINISH) != 0 || sharded;
     // Inputs that fit the L2 are served by one cooperative launch that needs no ticket counters.
     int small_seg_len = 0;
-    // (the single-launch kernel has no scaled form)
-    const int small_blocks =
-        (sharded || leaf_scales != nullptr || total == 0 || num_tensors == 0) ? 0 : resident_small_blocks();
+    const int small_blocks = (sharded || total == 0 || num_tensors == 0) ? 0 : resident_small_blocks();
     const bool small_candidate = small_blocks > 0 && small_input_plan(plan, total, num_tensors, offsets, n_workers, eb,
                                                                       flags, small_blocks, &small_seg_len);
     // the workspace arrives with unknown contents
@@ -967,7 +965,7 @@ adasum_status_t reduce_impl(const void* const* grads, const int64_t* offsets, in
             fin.selftest_timeout = 0;
             fin.tree = TreeOptions{tree_order(n_workers, flags), 1, 1, 1,
                                    orthogonality ? reinterpret_cast<double*>(ws + lay.leaf_sums) : nullptr,
-                                   orthogonality};
+                                   orthogonality, leaf_scales, num_tensors};
             float* partials = reinterpret_cast<float*>(ws + lay.partials);
             const int radix = plan.level[0].radix;
             PassExtras ex = last_extras;

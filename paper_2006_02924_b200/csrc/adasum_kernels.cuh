@@ -1956,14 +1956,23 @@ struct WarpTensor {
 // The binary tree (or the other two orders of Section 3.4) evaluated on a packed R x R Gram matrix
 // by ONE thread, R <= 8: leaf weights w[0 .. members) and the squared norm of the result.  Same
 // recursion as tree_weights_from_gram.
+// With opt.leaf_scales (operand i holds scale x gradient) a leaf starts with weight 1 / scale, as in
+// tree_weights_from_gram.  leaf_sum: the sum of the leaves' squared norms, in the gradients' units.
 template <int R>
-__device__ void tree_weights_serial(const double* gram, int members, int order, double* w, double& root_norm)
+__device__ void tree_weights_serial(const double* gram, int members, const TreeOptions& opt, int tensor, double* w,
+                                    double& root_norm, double& leaf_sum)
 {
+    const int order = opt.linear;
     double norm[R];
+    leaf_sum = 0.0;
 #pragma unroll
     for (int i = 0; i < R; ++i) {
-        w[i] = 1.0;
-        norm[i] = i < members ? gram[gram_index(R, i, i)] : 0.0;
+        double unit = 1.0;
+        if (opt.leaf_scales != nullptr && i < members)
+            unit = 1.0 / (double)opt.leaf_scales[(int64_t)i * opt.num_tensors + tensor];
+        w[i] = unit;
+        norm[i] = i < members ? gram[gram_index(R, i, i)] * unit * unit : 0.0;
+        leaf_sum += norm[i];
     }
     // a <- Adasum(a, b) for the nodes over leaves [lo, mid) and [mid, hi); norms kept at lo / mid
     auto combine = [&](int lo, int mid, int hi) {
@@ -2118,14 +2127,10 @@ __device__ void reduce_warp_tensor(const OperandTable& ops, int members, const W
             s += __shfl_xor_sync(0xffffffffu, s, d);
         gram[k] = s;
     }
-    double w64[R], root = 0.0;
-    tree_weights_serial<R>(gram, members, opt.linear, w64, root);
-    if (lane == 0 && opt.orthogonality != nullptr) {
-        double leaf_sum = 0.0;
-        for (int i = 0; i < members; ++i)
-            leaf_sum += gram[gram_index(R, i, i)];
+    double w64[R], root = 0.0, leaf_sum = 0.0;
+    tree_weights_serial<R>(gram, members, opt, wt.tensor, w64, root, leaf_sum);
+    if (lane == 0 && opt.orthogonality != nullptr)
         opt.orthogonality[wt.tensor] = leaf_sum == 0.0 ? __int_as_float(0x7fc00000) : (float)(root / leaf_sum);
-    }
     float w[R];
 #pragma unroll
     for (int i = 0; i < R; ++i)
@@ -2184,6 +2189,8 @@ __device__ void reduce_short_tensor_warp(const OperandTable& ops, int members, c
                 x = (double)delta_one(src, static_cast<const T*>(ex.start), st.begin + e);
             else
                 x = (double)Element<T>::one(src + st.begin + e);
+            if (opt.leaf_scales != nullptr)        // the buffer holds scale x gradient
+                x /= (double)opt.leaf_scales[(int64_t)i * opt.num_tensors + st.tensor];
             slot[i * kShortSlotElems + e] = x;
             sq += x * x;
         }
@@ -2243,16 +2250,12 @@ __device__ void finish_small(const float* partials, int seg_begin, int seg_end, 
     __syncthreads();
     if constexpr (R <= 4) {
         if (threadIdx.x == 0) {
-            double w64[R], root = 0.0;
-            tree_weights_serial<R>(gram, members, opt.linear, w64, root);
+            double w64[R], root = 0.0, leaf_sum = 0.0;
+            tree_weights_serial<R>(gram, members, opt, tensor, w64, root, leaf_sum);
             for (int i = 0; i < R; ++i)
                 weights_dst[i] = i < members ? (float)w64[i] : 0.0f;
-            if (opt.orthogonality != nullptr) {
-                double leaf_sum = 0.0;
-                for (int i = 0; i < members; ++i)
-                    leaf_sum += gram[gram_index(R, i, i)];
+            if (opt.orthogonality != nullptr)
                 opt.orthogonality[tensor] = leaf_sum == 0.0 ? __int_as_float(0x7fc00000) : (float)(root / leaf_sum);
-            }
         }
     } else {
         tree_weights_from_gram<R>(gram, members, weights_dst, opt, tensor, 0);

@@ -83,6 +83,22 @@ def test_scaled_reduce_matches_the_oracle(lib, dtype, n, flags):
     assert np.all(np.isnan(got_ortho[lens == 0]))
 
 
+@pytest.mark.parametrize("n,dtype", [(2, "f16"), (4, "f32"), (8, "bf16")])
+def test_scaled_small_inputs_take_the_single_launch(lib, n, dtype):
+    """Up to 8 workers and operands that fit the L2: one cooperative launch, which reads the scales in
+    its three coefficient steps (segments, one-warp tensors, tensors of at most 64 elements)."""
+    stored, scales = _case(n, OFFSETS, dtype, seed=9500 + n)
+    lib.adasum_profile_enable(16)
+    out, ortho = lib.adasum_reduce_scaled(stored, scales, OFFSETS, want_orthogonality=True)
+    torch.cuda.synchronize()
+    assert [r["kernel"] for r in lib.adasum_profile_collect(16)] == ["fused_small"]
+    ref, ref_ortho = oracle.adasum_reduce_scaled([_np(s, dtype) for s in stored], scales.cpu().numpy(), offsets=OFFSETS,
+                                                 dtype=dtype, return_orthogonality=True, threads=0)
+    _check(out, ref, OFFSETS, TOL[dtype])
+    lens = np.diff(OFFSETS)
+    np.testing.assert_allclose(ortho.double().cpu().numpy()[lens > 0], ref_ortho[lens > 0], rtol=20 * TOL[dtype])
+
+
 def test_scaled_reduce_differs_from_the_reduce_of_the_stored_values(lib):
     """The test above would also pass if the scales were ignored and the inputs happened to be
     insensitive to them; they are not: the plain reduce of the same buffers is far from the oracle."""
@@ -96,14 +112,14 @@ def test_scaled_reduce_differs_from_the_reduce_of_the_stored_values(lib):
 
 
 def test_unit_scales_give_the_plain_reduce_bit_for_bit(lib):
-    """Scales of exactly 1 change no bit on the two-pass path (flag bit 17 keeps the plain call off
-    the single launch, which the scaled call never takes)."""
+    """Scales of exactly 1 change no bit, on the two-pass path (flag bit 17) and in the single launch."""
     stored, _ = _case(8, OFFSETS, "f32", seed=9200, spread=0.0)
     ones = torch.ones(8, len(OFFSETS) - 1, device="cuda")
-    a = lib.adasum_reduce_scaled(stored, ones, OFFSETS, flags=SEPARATE)
-    b = lib.adasum_reduce(stored, OFFSETS, flags=SEPARATE)
-    torch.cuda.synchronize()
-    assert torch.equal(a, b)
+    for flags in (SEPARATE, 0):
+        a = lib.adasum_reduce_scaled(stored, ones, OFFSETS, flags=flags)
+        b = lib.adasum_reduce(stored, OFFSETS, flags=flags)
+        torch.cuda.synchronize()
+        assert torch.equal(a, b), flags
 
 
 @pytest.mark.parametrize("n", [300, 513])
