@@ -117,3 +117,87 @@ def test_planted_mistake_is_caught(tmp_path, name):
     assert text.count(old) >= 1, f"mutation site for '{name}' not found in the oracle source"
     mutant = _compile(text.replace(old, new, 1), tmp_path, "mutant")
     assert _failed_pins(mutant), f"no pin notices: {name}"
+
+
+# ---- the scaled form (its oracle function is Python around the same C tree) -----------------------
+
+def _scaled_variant(mistake):
+    """oracle.adasum_reduce_scaled with one plausible mistake planted (None: as it stands)."""
+    from oracle import adasum_oracle as oracle
+
+    def scaled(grads, scales, offsets=None, dtype=None, **kw):
+        arrs = [oracle.decode(g, dtype).reshape(-1) for g in grads]
+        total = arrs[0].size
+        offs = np.asarray([0, total] if offsets is None else offsets, dtype=np.int64)
+        num_tensors = offs.size - 1
+        sc = np.asarray(scales, dtype=np.float64)
+        if mistake == "table read tensor-major":
+            sc = sc.reshape(-1).reshape(num_tensors, len(arrs)).T
+        else:
+            sc = sc.reshape(len(arrs), num_tensors)
+        true = []
+        for w, a in enumerate(arrs):
+            g = a.copy()
+            for t in range(num_tensors):
+                s = sc[w, 0] if mistake == "first tensor's scale for every tensor" else sc[w, t]
+                if mistake == "multiplied instead of divided":
+                    g[offs[t]:offs[t + 1]] *= s
+                elif mistake == "worker 0's scale for every worker":
+                    g[offs[t]:offs[t + 1]] /= sc[0, t]
+                else:
+                    g[offs[t]:offs[t + 1]] /= s
+            true.append(g)
+        if mistake == "scales undone on the output instead":
+            plain = oracle.adasum_reduce(arrs, offsets=offs, dtype="f64", **kw)
+            res = plain[0] if isinstance(plain, tuple) else plain
+            for t in range(num_tensors):
+                res[offs[t]:offs[t + 1]] /= sc[:, t].mean()
+            return plain
+        return oracle.adasum_reduce(true, offsets=offs, dtype="f64", **kw)
+
+    return scaled
+
+
+def _failed_scaled_pins(scaled):
+    from oracle import adasum_oracle as oracle
+
+    failed = []
+
+    def check(name, got, want, tol=1e-12):
+        if not (np.all(np.isfinite(got)) and np.linalg.norm(got - want) <= tol * max(np.linalg.norm(want), 1e-300)):
+            failed.append(name)
+
+    check("orthogonal workers add up", scaled([np.array([4.0, 0.0]), np.array([0.0, 0.5])], [[4.0], [0.5]], dtype="f64"),
+          np.array([1.0, 1.0]))
+    rng = np.random.default_rng(5)
+    g = rng.standard_normal(37)
+    sc = rng.uniform(0.01, 300.0, size=(5, 1))
+    check("identical gradients under any scales", scaled([g * sc[w, 0] for w in range(5)], sc, dtype="f64"), g)
+    offs = [0, 9, 20]
+    gs = [np.round(rng.standard_normal(20) * 64) / 64 for _ in range(3)]
+    table = np.array([[2.0, 0.25], [16.0, 0.5], [0.125, 8.0]])
+    stored = []
+    for w in range(3):
+        v = gs[w].copy()
+        v[0:9] *= table[w, 0]
+        v[9:20] *= table[w, 1]
+        stored.append(v.astype(np.float16))
+    check("six power-of-two scales, fp16 storage", scaled(stored, table, offsets=offs, dtype="f16"),
+          oracle.adasum_reduce(gs, offsets=offs, dtype="f64"))
+    return failed
+
+
+SCALED_MISTAKES = ["multiplied instead of divided", "table read tensor-major", "first tensor's scale for every tensor",
+                   "worker 0's scale for every worker", "scales undone on the output instead"]
+
+
+def test_scaled_form_as_it_stands_passes_its_pins():
+    from oracle import adasum_oracle as oracle
+
+    assert _failed_scaled_pins(oracle.adasum_reduce_scaled) == []
+    assert _failed_scaled_pins(_scaled_variant(None)) == []
+
+
+@pytest.mark.parametrize("mistake", SCALED_MISTAKES)
+def test_planted_mistake_in_the_scaled_form_is_caught(mistake):
+    assert _failed_scaled_pins(_scaled_variant(mistake)), mistake
